@@ -1,0 +1,155 @@
+"""fp64 CPU oracle for SEKA / AdaSEKA steered attention -- TEST INFRASTRUCTURE ONLY.
+
+Thin ctypes wrapper over ``seka_oracle.c`` (compiled on first use with gcc).
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import
+this package; the CUDA library never does, and this package never imports the
+CUDA library.  All tensors are packed ``[total_tokens, heads, d]`` numpy arrays
+with ``cu_seqlens`` (host list of B+1 offsets) delimiting the sequences; every
+input is upcast to float64 and nothing is rounded afterwards.
+
+Functions follow the paper: ``route`` is Eq. 6 (Section 3.3), ``edit_keys`` is
+the hook of Algorithm 1/2 with k' = k + g P k (Section 2, Eq. 7), and
+``attention_rows`` is causal softmax attention with the score of Section 2.
+The reading of the routing query under GQA (sum over the group's query heads)
+is PARITY UNPINNED: the paper does not fix it.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "seka_oracle.c")
+_LIB = os.path.join(_HERE, "libseka_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle into a shared object next to its source."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp%d" % os.getpid()
+        subprocess.check_call(["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        dp = ctypes.POINTER(ctypes.c_double)
+        u8p = ctypes.POINTER(ctypes.c_uint8)
+        i32p = ctypes.POINTER(ctypes.c_int32)
+        ci = ctypes.c_int
+        lib.seka_oracle_route.argtypes = [ci, ci, ci, ci, ci, ci, dp, dp, dp, dp]
+        lib.seka_oracle_route.restype = None
+        lib.seka_oracle_edit_keys.argtypes = [ci, ci, ci, ci, ci, dp, u8p, dp, dp, ctypes.c_double, u8p, dp]
+        lib.seka_oracle_edit_keys.restype = None
+        lib.seka_oracle_attention_rows.argtypes = [ci, ci, ci, ci, dp, dp, dp, ctypes.c_double, ci, i32p, dp, dp]
+        lib.seka_oracle_attention_rows.restype = None
+        lib.seka_oracle_threads.argtypes = []
+        lib.seka_oracle_threads.restype = ci
+        _lib = lib
+    return _lib
+
+
+def _f64(a) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(a, dtype=np.float64))
+
+
+def _dp(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(ctypes.POINTER(ctypes.c_double))
+
+
+def _u8p(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(ctypes.POINTER(ctypes.c_uint8))
+
+
+def threads() -> int:
+    """OpenMP threads the oracle uses for its independent loops."""
+    return int(_load().seka_oracle_threads())
+
+
+def route(Q, cu_seqlens: Sequence[int], U, sigma, k_route: int = 0) -> np.ndarray:
+    """AdaSEKA coefficients alpha[B, Hkv, M] from each sequence's last-token query (Eq. 6)."""
+    lib = _load()
+    Q = _f64(Q); U = _f64(U); sigma = _f64(sigma)
+    M, Hkv, d, r = U.shape
+    Hq = Q.shape[1]
+    k_route = r if k_route in (0, None) else int(k_route)
+    assert 1 <= k_route <= r and sigma.shape == (M, Hkv, r) and Hq % Hkv == 0
+    B = len(cu_seqlens) - 1
+    alpha = np.zeros((B, Hkv, M), dtype=np.float64)
+    for b in range(B):
+        last = int(cu_seqlens[b + 1]) - 1
+        q_last = np.ascontiguousarray(Q[last])
+        out = np.zeros((Hkv, M), dtype=np.float64)
+        lib.seka_oracle_route(Hq, Hkv, d, r, M, k_route, _dp(q_last), _dp(U), _dp(sigma), _dp(out))
+        alpha[b] = out
+    return alpha
+
+
+def edit_keys(K, mask, cu_seqlens: Sequence[int], U, alpha=None, gain=None, head_enable=None) -> np.ndarray:
+    """Edited keys k' = k + g * sum_m alpha_m U_m U_m^T k at highlighted tokens (Algorithm 1/2 hook)."""
+    lib = _load()
+    K = _f64(K); U = _f64(U)
+    M, Hkv, d, r = U.shape
+    assert K.shape[1:] == (Hkv, d)
+    B = len(cu_seqlens) - 1
+    mask = np.ascontiguousarray(np.asarray(mask) != 0, dtype=np.uint8)
+    gain = np.ones(B) if gain is None else np.broadcast_to(np.asarray(gain, dtype=np.float64), (B,))
+    he = None if head_enable is None else np.ascontiguousarray(np.asarray(head_enable) != 0, dtype=np.uint8)
+    out = np.empty_like(K)
+    for b in range(B):
+        s, e = int(cu_seqlens[b]), int(cu_seqlens[b + 1])
+        if e == s:
+            continue
+        Kb = np.ascontiguousarray(K[s:e]); mb = np.ascontiguousarray(mask[s:e])
+        ab = None if alpha is None else _f64(np.asarray(alpha)[b])
+        ob = np.empty_like(Kb)
+        lib.seka_oracle_edit_keys(e - s, Hkv, d, r, M, _dp(Kb), _u8p(mb), _dp(U), _dp(ab),
+                                  float(gain[b]), _u8p(he), _dp(ob))
+        out[s:e] = ob
+    return out
+
+
+def attention_rows(Q, Kp, V, cu_seqlens: Sequence[int], rows=None, scale: Optional[float] = None):
+    """Causal softmax attention over (already edited) keys for chosen query rows.
+
+    ``rows`` is None (every row) or a list with one int array of in-sequence
+    positions per sequence.  Returns ``(O, LSE, index)``: O [n, Hq, d] and
+    LSE [n, Hq] stacked over sequences, and ``index`` [n] the packed token index
+    of each returned row.
+    """
+    lib = _load()
+    Q = _f64(Q); Kp = _f64(Kp); V = _f64(V)
+    Hq, d = Q.shape[1:]
+    Hkv = Kp.shape[1]
+    scale = 1.0 / np.sqrt(d) if not scale else float(scale)
+    B = len(cu_seqlens) - 1
+    Os, Ls, idx = [], [], []
+    for b in range(B):
+        s, e = int(cu_seqlens[b]), int(cu_seqlens[b + 1])
+        rb = np.arange(e - s, dtype=np.int32) if rows is None else np.ascontiguousarray(rows[b], dtype=np.int32)
+        if rb.size == 0:
+            continue
+        assert rb.min() >= 0 and rb.max() < e - s
+        Qb = np.ascontiguousarray(Q[s:e]); Kb = np.ascontiguousarray(Kp[s:e]); Vb = np.ascontiguousarray(V[s:e])
+        O = np.empty((rb.size, Hq, d)); LSE = np.empty((rb.size, Hq))
+        lib.seka_oracle_attention_rows(e - s, Hq, Hkv, d, _dp(Qb), _dp(Kb), _dp(Vb), scale, rb.size,
+                                       rb.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)), _dp(O), _dp(LSE))
+        Os.append(O); Ls.append(LSE); idx.append(rb.astype(np.int64) + s)
+    if not Os:
+        return np.zeros((0, Hq, d)), np.zeros((0, Hq)), np.zeros((0,), dtype=np.int64)
+    return np.concatenate(Os), np.concatenate(Ls), np.concatenate(idx)
+
+
+def seka_attention(Q, K, V, mask, cu_seqlens, U, alpha=None, gain=None, head_enable=None,
+                   rows=None, scale: Optional[float] = None):
+    """The whole steered path: edit the highlighted keys, then causal attention."""
+    Kp = edit_keys(K, mask, cu_seqlens, U, alpha, gain, head_enable)
+    return attention_rows(Q, Kp, V, cu_seqlens, rows, scale)

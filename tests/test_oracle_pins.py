@@ -1,0 +1,252 @@
+"""Pins for the fp64 CPU oracle: everything the paper and the mathematics fix, none of it
+computed by the oracle itself.  CPU only."""
+import json
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import brute
+from paper_2603_01281_b200 import inputs
+
+GOLD = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "hand_cases.json")))
+
+
+def tiny(seed=1, L=48, Hq=4, Hkv=2, d=16, r=4, M=1, lens=None, mask_kind="spans", gain=0.7, highlight=0.3):
+    return inputs.make_custom(seed=seed, dtype="f32", lens=lens or [L], n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d,
+                              rank=r, n_experts=M, mask_kind=mask_kind, gain=gain, highlight=highlight)
+
+
+# ----------------------------------------------------------------- hand-derived examples
+
+def test_route_hand_case():
+    g = GOLD["route"]
+    U = np.array(g["U"], dtype=np.float64)            # [M=2, Hkv=1, d=3, r=2]
+    sigma = np.array(g["sigma"], dtype=np.float64)
+    q = np.array(g["q"], dtype=np.float64).reshape(1, 1, 3)
+    np.testing.assert_allclose(oracle.route(q, [0, 1], U, sigma, 2)[0, 0], g["alpha_K2"], atol=1e-15)
+    np.testing.assert_allclose(oracle.route(q, [0, 1], U, sigma, 1)[0, 0], g["alpha_K1"], atol=1e-15)
+    # the routing query is the LAST token of the sequence; earlier tokens must not matter
+    qq = np.concatenate([np.full((3, 1, 3), 9.0), q], axis=0)
+    np.testing.assert_allclose(oracle.route(qq, [0, 4], U, sigma, 2)[0, 0], g["alpha_K2"], atol=1e-15)
+    # GQA: the group's query heads are summed
+    qh = np.array(g["q_heads"], dtype=np.float64).reshape(1, 2, 3)
+    np.testing.assert_allclose(oracle.route(qh, [0, 1], U, sigma, 2)[0, 0], g["alpha_K2"], atol=1e-15)
+
+
+def test_edit_hand_case():
+    g = GOLD["edit"]
+    k = np.array(g["k"], dtype=np.float64).reshape(1, 1, 3)
+    U1 = np.array(g["u1"]).reshape(1, 1, 3, 1)
+    out = oracle.edit_keys(k, [1], [0, 1], U1, gain=[g["g"]])
+    np.testing.assert_allclose(out[0, 0], g["k_edit_single"], atol=1e-14)
+    U2 = np.stack([np.array(g["u1"]).reshape(1, 3, 1), np.array(g["u2"]).reshape(1, 3, 1)])
+    out = oracle.edit_keys(k, [1], [0, 1], U2, alpha=np.array(g["alpha"], dtype=float).reshape(1, 1, 2), gain=[g["g"]])
+    np.testing.assert_allclose(out[0, 0], g["k_edit_blend"], atol=1e-14)
+    # unhighlighted token: untouched
+    assert np.array_equal(oracle.edit_keys(k, [0], [0, 1], U1, gain=[g["g"]]), k)
+
+
+def test_attention_hand_case():
+    g = GOLD["attention"]
+    Q = np.zeros((2, 1, 4)); Q[:, 0, 0] = 2.0
+    K = np.zeros((2, 1, 4)); K[1, 0, 0] = math.log(3.0)
+    V = np.zeros((2, 1, 4)); V[0, 0, :] = 4.0; V[1, 0, :] = 8.0
+    O, LSE, idx = oracle.attention_rows(Q, K, V, [0, 2])
+    np.testing.assert_allclose(O[1, 0], g["o1_plain"], atol=1e-14)
+    np.testing.assert_allclose(O[0, 0], 4.0, atol=1e-14)
+    np.testing.assert_allclose(LSE[:, 0], [0.0, math.log(4.0)], atol=1e-14)
+    U = np.eye(4).reshape(1, 1, 4, 4)
+    O, LSE, _ = oracle.seka_attention(Q, K, V, [0, 1], [0, 2], U, gain=[1.0])
+    np.testing.assert_allclose(O[1, 0], g["o1_steered"], atol=1e-14)
+    np.testing.assert_allclose(LSE[1, 0], math.log(10.0), atol=1e-14)
+
+
+# ----------------------------------------------------------------- key edit: Appendix C closed forms
+
+@pytest.mark.parametrize("g", [0.5, 1.0, -0.4, -5.0, 2.0])
+def test_edit_closed_form_eq12(g):
+    w = tiny(seed=3, gain=g)
+    g = float(w.gain[0])          # the gain as stored (fp32)
+    Kp = oracle.edit_keys(w.K, w.mask, w.cu_seqlens, w.U, gain=w.gain)
+    K = w.K.astype(np.float64)
+    hl = w.mask != 0
+    assert hl.any() and (~hl).any()
+    for h in range(w.n_kv_heads):
+        U = w.U[0, h].astype(np.float64)
+        # exactly orthonormal factor for the closed form (the stored fp32 U is only nearly so)
+        Uo, _ = np.linalg.qr(U)
+        Kpo = oracle.edit_keys(w.K, w.mask, w.cu_seqlens, np.broadcast_to(Uo, (1, w.n_kv_heads) + Uo.shape), gain=w.gain)
+        par = K[hl, h] @ Uo @ Uo.T
+        perp = K[hl, h] - par
+        # Eq. 12: (I + g U U^T) x = x_perp + (1+g) x_par
+        np.testing.assert_allclose(Kpo[hl, h], perp + (1 + g) * par, atol=1e-12)
+        np.testing.assert_allclose(Kpo[hl, h] @ Uo, (1 + g) * (K[hl, h] @ Uo), atol=1e-12)
+        np.testing.assert_allclose(np.sum(Kpo[hl, h] ** 2, -1),
+                                   np.sum(perp ** 2, -1) + (1 + g) ** 2 * np.sum(par ** 2, -1), rtol=1e-12)
+        # stored-U version: U (U^T k) as written
+        np.testing.assert_allclose(Kp[hl, h], K[hl, h] + g * (K[hl, h] @ U) @ U.T, atol=1e-12)
+    # every unhighlighted key is bit-identical
+    assert np.array_equal(Kp[~hl], K[~hl])
+
+
+def test_projector_idempotent_symmetric_and_full_rank_edit():
+    rng = np.random.default_rng(0)
+    U = inputs.orthonormal_bank(rng, 1, 2, 16, 16).astype(np.float64)
+    Uq, _ = np.linalg.qr(U[0, 0])
+    P = brute.dense_projector(Uq[None, None, :, :5], 0)
+    np.testing.assert_allclose(P @ P, P, atol=1e-13)
+    np.testing.assert_allclose(P, P.T, atol=0)
+    # generated banks are orthonormal to fp32 accuracy
+    np.testing.assert_allclose(U[0, 1].T @ U[0, 1], np.eye(16), atol=1e-6)
+    # r = d with orthogonal U: k' = (1+g) k
+    K = rng.standard_normal((5, 1, 16))
+    Kp = oracle.edit_keys(K, np.ones(5), [0, 5], Uq[None, None], gain=[1.5])
+    np.testing.assert_allclose(Kp, 2.5 * K, atol=1e-12)
+
+
+def test_edit_head_enable_and_per_sequence_gain():
+    w = tiny(seed=5, lens=[20, 33, 7], gain=[0.5, -1.0, 2.0], Hkv=2)
+    he = np.array([1, 0], dtype=np.uint8)
+    Kp = oracle.edit_keys(w.K, w.mask, w.cu_seqlens, w.U, gain=w.gain, head_enable=he)
+    K = w.K.astype(np.float64)
+    assert np.array_equal(Kp[:, 1], K[:, 1])             # unselected head untouched (Section 3.4)
+    for b in range(3):
+        s, e = w.cu_seqlens[b], w.cu_seqlens[b + 1]
+        ref = brute.edited_keys(w.K[s:e], w.mask[s:e], w.U, g=float(w.gain[b]), head_enable=he)
+        np.testing.assert_allclose(Kp[s:e], ref, atol=1e-12)
+
+
+# ----------------------------------------------------------------- attention
+
+def test_g0_and_empty_mask_are_textbook_causal_attention():
+    w = tiny(seed=7, L=40, Hq=4, Hkv=2, d=16)
+    Qt = torch.from_numpy(w.Q.astype(np.float64)).permute(1, 0, 2)[None]
+    Kt = torch.from_numpy(w.K.astype(np.float64)).permute(1, 0, 2)[None].repeat_interleave(2, dim=1)
+    Vt = torch.from_numpy(w.V.astype(np.float64)).permute(1, 0, 2)[None].repeat_interleave(2, dim=1)
+    ref = torch.nn.functional.scaled_dot_product_attention(Qt, Kt, Vt, is_causal=True)[0].permute(1, 0, 2).numpy()
+    O0, _, _ = oracle.seka_attention(w.Q, w.K, w.V, w.mask, w.cu_seqlens, w.U, gain=[0.0])
+    np.testing.assert_allclose(O0, ref, atol=1e-12)
+    O1, _, _ = oracle.seka_attention(w.Q, w.K, w.V, np.zeros_like(w.mask), w.cu_seqlens, w.U, gain=[3.0])
+    np.testing.assert_allclose(O1, ref, atol=1e-12)
+    # GQA map: consecutive query heads share a KV head -- swapping which KV head a query head reads must break it
+    bad = torch.nn.functional.scaled_dot_product_attention(
+        Qt, Kt[:, [0, 2, 1, 3]], Vt[:, [0, 2, 1, 3]], is_causal=True)[0].permute(1, 0, 2).numpy()
+    assert np.abs(bad - O0).max() > 1e-3
+
+
+def test_rows_sum_to_one_first_row_and_lse():
+    w = tiny(seed=8, L=37)
+    ones = np.ones_like(w.V)
+    O, LSE, idx = oracle.seka_attention(w.Q, w.K, ones, w.mask, w.cu_seqlens, w.U, gain=w.gain)
+    np.testing.assert_allclose(O, 1.0, atol=1e-13)                    # softmax rows sum to 1
+    O, LSE, idx = oracle.seka_attention(w.Q, w.K, w.V, w.mask, w.cu_seqlens, w.U, gain=w.gain)
+    G = w.n_q_heads // w.n_kv_heads
+    np.testing.assert_allclose(O[0], np.repeat(w.V[0].astype(np.float64), G, axis=0), atol=1e-13)   # o_0 = v_0
+    # a future key must not matter (causality): perturb the last key/value, earlier rows unchanged
+    K2 = w.K.copy(); V2 = w.V.copy(); K2[-1] += 5.0; V2[-1] -= 3.0
+    O2, _, _ = oracle.seka_attention(w.Q, K2, V2, w.mask, w.cu_seqlens, w.U, gain=w.gain)
+    assert np.array_equal(O2[:-1], O[:-1]) and not np.allclose(O2[-1], O[-1])
+
+
+@pytest.mark.parametrize("M", [1, 3])
+def test_brute_force_and_logit_bias_identity(M):
+    # Eq. 5: attention over edited keys == attention over logits A + B, B the low-rank bias on highlighted columns
+    w = tiny(seed=11 + M, L=53, Hq=6, Hkv=2, d=16, r=4, M=M, gain=1.3)
+    rng = np.random.default_rng(2)
+    alpha = rng.uniform(-1, 1, size=(1, w.n_kv_heads, M)) if M > 1 else None
+    he = np.array([1, 1], dtype=np.uint8)
+    O, LSE, _ = oracle.seka_attention(w.Q, w.K, w.V, w.mask, w.cu_seqlens, w.U, alpha=alpha, gain=w.gain, head_enable=he)
+    a0 = None if alpha is None else alpha[0]
+    Ob, Lb = brute.attention_from_keys(w.Q, brute.edited_keys(w.K, w.mask, w.U, a0, float(w.gain[0])), w.V)
+    np.testing.assert_allclose(O, Ob, atol=1e-12); np.testing.assert_allclose(LSE, Lb, atol=1e-12)
+    Oc, Lc = brute.attention_logit_bias(w.Q, w.K, w.V, w.mask, w.U, a0, float(w.gain[0]))
+    np.testing.assert_allclose(O, Oc, atol=1e-12); np.testing.assert_allclose(LSE, Lc, atol=1e-12)
+
+
+def test_query_side_duality():
+    # Section 2: the same logits arise from editing the query, ((I + gP) q)^T k on highlighted columns
+    w = tiny(seed=21, L=30, Hq=2, Hkv=2, d=16, r=5, gain=0.9)
+    Kp = oracle.edit_keys(w.K, w.mask, w.cu_seqlens, w.U, gain=w.gain)
+    hl = w.mask != 0
+    for h in range(2):
+        P = brute.dense_projector(w.U, h)
+        Qe = w.Q[:, h].astype(np.float64) @ (np.eye(16) + float(w.gain[0]) * P).T
+        S_key = w.Q[:, h].astype(np.float64) @ Kp[:, h].T
+        S_dual = np.where(hl[None, :], Qe @ w.K[:, h].astype(np.float64).T, w.Q[:, h].astype(np.float64) @ w.K[:, h].astype(np.float64).T)
+        np.testing.assert_allclose(S_key, S_dual, atol=1e-12)
+
+
+def test_identity_projector_scales_highlighted_scores():
+    # P = I: the scores of highlighted columns are multiplied by (1+g), the others unchanged
+    w = tiny(seed=31, L=29, Hq=2, Hkv=1, d=8, r=8, gain=0.6)
+    U = np.eye(8).reshape(1, 1, 8, 8)
+    O, LSE, _ = oracle.seka_attention(w.Q, w.K, w.V, w.mask, w.cu_seqlens, U, gain=w.gain)
+    hl = w.mask != 0
+    for hq in range(2):
+        S = w.Q[:, hq].astype(np.float64) @ w.K[:, 0].astype(np.float64).T / math.sqrt(8)
+        S = np.where(hl[None, :], (1.0 + float(w.gain[0])) * S, S)
+        P, lse = brute._softmax_causal(S)
+        np.testing.assert_allclose(O[:, hq], P @ w.V[:, 0].astype(np.float64), atol=1e-12)
+        np.testing.assert_allclose(LSE[:, hq], lse, atol=1e-12)
+
+
+def test_varlen_sequences_are_independent_and_rows_subset():
+    w = tiny(seed=41, lens=[17, 1, 40], Hq=4, Hkv=2, d=16, gain=[0.5, 1.0, 2.0])
+    O, LSE, idx = oracle.seka_attention(w.Q, w.K, w.V, w.mask, w.cu_seqlens, w.U, gain=w.gain)
+    assert list(idx) == list(range(58))
+    for b in range(3):
+        s, e = w.cu_seqlens[b], w.cu_seqlens[b + 1]
+        Ob, _ = brute.attention_from_keys(w.Q[s:e], brute.edited_keys(w.K[s:e], w.mask[s:e], w.U, None, float(w.gain[b])), w.V[s:e])
+        np.testing.assert_allclose(O[s:e], Ob, atol=1e-12)
+    rows = [np.array([0, 16]), np.array([0]), np.array([5, 39])]
+    Os, Ls, ids = oracle.seka_attention(w.Q, w.K, w.V, w.mask, w.cu_seqlens, w.U, gain=w.gain, rows=rows)
+    np.testing.assert_allclose(Os, O[ids], atol=0); np.testing.assert_allclose(Ls, LSE[ids], atol=0)
+
+
+def test_softmax_scale_override():
+    w = tiny(seed=51, L=12, Hq=2, Hkv=2, d=16)
+    O, _, _ = oracle.attention_rows(w.Q, w.K, w.V, w.cu_seqlens, scale=0.37)
+    Ob, _ = brute.attention_from_keys(w.Q, w.K, w.V, scale=0.37)
+    np.testing.assert_allclose(O, Ob, atol=1e-12)
+
+
+# ----------------------------------------------------------------- AdaSEKA
+
+def test_single_expert_unit_alpha_is_seka():
+    w = tiny(seed=61, L=25)
+    a = oracle.edit_keys(w.K, w.mask, w.cu_seqlens, w.U, gain=w.gain)
+    b = oracle.edit_keys(w.K, w.mask, w.cu_seqlens, w.U, alpha=np.ones((1, w.n_kv_heads, 1)), gain=w.gain)
+    assert np.array_equal(a, b)
+
+
+def test_routing_invariants():
+    w = inputs.make_custom(seed=71, dtype="f32", lens=[9, 14], n_q_heads=8, n_kv_heads=2, head_dim=16, rank=6,
+                           n_experts=4, gain=1.0)
+    a = oracle.route(w.Q, w.cu_seqlens, w.U, w.sigma, 5)
+    assert a.shape == (2, 2, 4)
+    np.testing.assert_allclose(np.abs(a).max(axis=-1), 1.0, atol=1e-15)          # max_m |alpha_m| = 1
+    np.testing.assert_allclose(oracle.route(3.7 * w.Q.astype(np.float64), w.cu_seqlens, w.U, w.sigma, 5), a, atol=1e-12)
+    np.testing.assert_allclose(oracle.route(-w.Q, w.cu_seqlens, w.U, w.sigma, 5), -a, atol=1e-12)
+    # direct evaluation of Eq. 6 with matrix products
+    for b in range(2):
+        q = w.Q[w.cu_seqlens[b + 1] - 1].astype(np.float64).reshape(2, 4, 16).sum(axis=1)    # [Hkv, d]
+        for h in range(2):
+            s = np.array([(q[h] @ w.U[m, h].astype(np.float64)[:, :5]) @ w.sigma[m, h, :5].astype(np.float64) for m in range(4)])
+            np.testing.assert_allclose(a[b, h], s / np.abs(s).max(), atol=1e-12)
+    # k_route = 0 means every stored component
+    np.testing.assert_allclose(oracle.route(w.Q, w.cu_seqlens, w.U, w.sigma, 0),
+                               oracle.route(w.Q, w.cu_seqlens, w.U, w.sigma, 6), atol=0)
+    # all-zero query: alpha = 0
+    assert np.array_equal(oracle.route(np.zeros_like(w.Q), w.cu_seqlens, w.U, w.sigma, 5), np.zeros((2, 2, 4)))
+
+
+def test_blend_factor_form_equals_dense_projector():
+    w = inputs.make_custom(seed=81, dtype="f32", lens=[31], n_q_heads=4, n_kv_heads=2, head_dim=16, rank=4,
+                           n_experts=4, gain=1.1, highlight=0.4)
+    a = oracle.route(w.Q, w.cu_seqlens, w.U, w.sigma, 0)
+    Kp = oracle.edit_keys(w.K, w.mask, w.cu_seqlens, w.U, alpha=a, gain=w.gain)
+    np.testing.assert_allclose(Kp, brute.edited_keys(w.K, w.mask, w.U, a[0], float(w.gain[0])), atol=1e-12)
