@@ -1,0 +1,137 @@
+/*
+ * seka.h -- C ABI of the B200 (sm_100a) SEKA / AdaSEKA steered-attention library.
+ *
+ * The library computes prefill causal grouped-query attention in which the keys
+ * of highlighted tokens are spectrally edited before the scores are formed:
+ *     k' = k + g * P k,   P = U U^T                    (SEKA,    Section 2 / Eq. 7)
+ *     P = sum_m alpha_m U_m U_m^T                      (AdaSEKA, Section 3.3)
+ * with the routing coefficients alpha of Eq. 6, applied only where the per-token
+ * highlight mask is set and only on selected KV heads (Section 3.4), the edited
+ * keys feeding a causal softmax attention with scores q.k'/sqrt(d) (Section 2).
+ *
+ * Conventions shared by every entry point
+ *  - Pointers are DEVICE pointers unless the name starts with `h_`. The caller owns
+ *    every buffer; the library keeps none and allocates none.
+ *  - Tensors are packed token-major: Q [T, Hq, d], K and V [T, Hkv, d], O [T, Hq, d],
+ *    mask [T] (non-zero = highlighted), T = total_tokens, rows contiguous, base
+ *    pointers 16-byte aligned.  Sequence b owns tokens cu_seqlens[b] .. cu_seqlens[b+1]-1;
+ *    with cu_seqlens == NULL every sequence has max_seqlen tokens (the [B, L, H, d]
+ *    layout of the hook in Algorithm 1).
+ *  - Query head hq reads KV head hq / (Hq / Hkv).
+ *  - U is fp32 [M, Hkv, d, r] (columns assumed orthonormal but used as stored: the
+ *    kernels compute U (U^T k)).  alpha is fp32 [B, Hkv, M] or NULL (all ones).
+ *    gain is fp32 [B] (any sign, zero allowed).  head_enable is uint8 [Hkv] or NULL
+ *    (all heads steered).
+ *  - Calls are asynchronous on `cuda_stream` (a cudaStream_t passed as void*).
+ *    Argument errors are returned before anything is launched.  A device-side wait
+ *    that runs out (every wait in the kernels is bounded) records SEKA_ERR_TIMEOUT in
+ *    the first word of `workspace`; seka_poll_status reads it.
+ *  - Causal, forward only, queries and keys of equal length.  head_dim is 64 or 128.
+ */
+#ifndef SEKA_H_
+#define SEKA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SEKA_OK = 0,
+    SEKA_ERR_INVALID_ARG = 1,   /* null pointer, bad size, misaligned buffer */
+    SEKA_ERR_UNSUPPORTED = 2,   /* shape outside what the kernels cover */
+    SEKA_ERR_WORKSPACE = 3,     /* workspace missing or smaller than seka_workspace_bytes */
+    SEKA_ERR_CUDA = 4,          /* a CUDA runtime / driver call failed */
+    SEKA_ERR_TIMEOUT = 5        /* a bounded device-side wait ran out */
+} seka_status;
+
+typedef enum { SEKA_F32 = 0, SEKA_BF16 = 1 } seka_dtype;
+
+typedef struct {
+    int32_t batch;              /* number of sequences B (>= 0) */
+    int32_t max_seqlen;         /* L, or max_b L_b when cu_seqlens is given */
+    int32_t total_tokens;       /* T; 0 means batch * max_seqlen (only valid without cu_seqlens) */
+    int32_t n_q_heads;          /* Hq, a multiple of n_kv_heads */
+    int32_t n_kv_heads;         /* Hkv */
+    int32_t head_dim;           /* d: 64 or 128 */
+    int32_t rank;               /* r: columns stored per expert, 1 .. d */
+    int32_t n_experts;          /* M >= 1; M * r <= 128 */
+    int32_t dtype;              /* seka_dtype of Q, K, V, O */
+    float   softmax_scale;      /* 0 means 1/sqrt(head_dim) (Section 2) */
+    const int32_t* cu_seqlens;  /* device int32 [B+1], or NULL for fixed length */
+} seka_shape;
+
+/* Bytes of scratch the calls below need for this shape (host-only, launches nothing). */
+size_t seka_workspace_bytes(const seka_shape* shape);
+
+/*
+ * Key-editing hook of Algorithm 1 / Algorithm 2 on a key tensor in HBM (for example a
+ * KV cache): K_out[t, h, :] = K_in[t, h, :] + gain[b] * sum_m alpha[b,h,m] U_m (U_m^T K_in[t,h,:])
+ * for highlighted tokens t of enabled heads h; every other row of K_out equals K_in
+ * bit for bit.  K_out may alias K_in (in place: only edited rows are written).
+ * fp32 tensors are edited in fp32 arithmetic; bf16 tensors accumulate in fp32 and round
+ * once.  Uses `workspace` for the compacted list of highlighted tokens.
+ */
+seka_status seka_edit_keys(const seka_shape* shape, const void* K_in, void* K_out,
+                           const uint8_t* mask, const float* U, const float* alpha,
+                           const float* gain, const uint8_t* head_enable,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * AdaSEKA routing, Eq. 6 / Algorithm 2: from the query of each sequence's LAST token,
+ *   s_m = sum_{k < k_route} (q . U_m[:, k]) * sigma_m[k],   alpha_m = s_m / max_m' |s_m'|
+ * per (sequence, KV head); q is the sum of the query heads of that KV head's group; all
+ * s_m zero gives alpha = 0.  sigma is fp32 [M, Hkv, r]; k_route in 1..r, 0 means r.
+ * alpha_out is fp32 [B, Hkv, M].
+ */
+seka_status adaseka_route(const seka_shape* shape, const void* Q, const float* U,
+                          const float* sigma, int32_t k_route, float* alpha_out,
+                          void* cuda_stream);
+
+/*
+ * Fused steered attention (Algorithm 1/2 hook + the attention it feeds, Eq. 4-5 in the
+ * single-projector form): O = softmax_causal(Q K'^T * scale) V with K' the edited keys;
+ * K' and the score matrix are never written to memory, K and V are not modified.
+ * O has the dtype of the inputs.  With dtype SEKA_F32 the inputs are rounded to bf16
+ * on the way in (the contraction runs on bf16 tensor cores, fp32 accumulation).
+ * lse, if not NULL, receives log sum_j exp(score_ij) as fp32 [T, Hq].
+ * mask == NULL or U == NULL means no steering (plain causal attention).
+ */
+seka_status seka_attention_fwd(const seka_shape* shape, const void* Q, const void* K,
+                               const void* V, void* O, float* lse,
+                               const uint8_t* mask, const float* U, const float* alpha,
+                               const float* gain, const uint8_t* head_enable,
+                               void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Same computation as seka_attention_fwd for callers whose tensors live in HOST memory
+ * (pinned memory makes the copies asynchronous): h_Q, h_K, h_V, h_mask are copied to
+ * `staging` (device, seka_host_staging_bytes(shape) bytes, 256-byte aligned), the
+ * fused kernel runs, and O (and lse if h_lse != NULL) is copied back to h_O, all on
+ * `cuda_stream`.  U, alpha, gain, head_enable stay device pointers (they are per-model
+ * or per-prompt constants).
+ */
+size_t seka_host_staging_bytes(const seka_shape* shape);
+seka_status seka_attention_fwd_host(const seka_shape* shape, const void* h_Q, const void* h_K,
+                                    const void* h_V, void* h_O, float* h_lse,
+                                    const uint8_t* h_mask, const float* U, const float* alpha,
+                                    const float* gain, const uint8_t* head_enable,
+                                    void* staging, size_t staging_bytes,
+                                    void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Clears the device status word (async on the stream); call once before first use of a workspace. */
+seka_status seka_reset_status(void* workspace, void* cuda_stream);
+/* Synchronises the stream and returns the device status word (SEKA_OK if no wait ran out). */
+seka_status seka_poll_status(const void* workspace, void* cuda_stream);
+
+const char* seka_status_string(seka_status status);
+
+/* Number of kernels this library has launched in this process (for benchmark accounting). */
+uint64_t seka_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SEKA_H_ */

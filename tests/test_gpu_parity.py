@@ -1,0 +1,203 @@
+"""GPU parity: the CUDA path (through the C ABI) against the fp64 CPU oracle on identical seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2603_01281_b200 import binding, inputs
+
+import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    binding.load()          # raises if the compiled library is missing: there is no fallback
+
+
+# ----------------------------------------------------------------- routing (Eq. 6)
+
+@pytest.mark.parametrize("case", ["C3", "small_f32", "small_varlen"])
+def test_route_matches_oracle(case):
+    if case == "C3":
+        w = inputs.make_workload("C3"); k_route = 0
+    elif case == "small_f32":
+        w = inputs.make_custom(seed=5, dtype="f32", lens=[40, 40], n_q_heads=8, n_kv_heads=2, head_dim=64, rank=16,
+                               n_experts=3); k_route = 5
+    else:
+        w = inputs.make_custom(seed=6, dtype="bf16", lens=[17, 300, 1], n_q_heads=14, n_kv_heads=2, head_dim=128,
+                               rank=8, n_experts=4); k_route = 8
+    dev = H.device_tensors(w)
+    shp = H.shape_of(w, dev)
+    alpha = torch.full((w.batch, w.n_kv_heads, w.n_experts), float("nan"), device="cuda")
+    binding.adaseka_route(shp, dev["Q"], dev["U"], dev["sigma"], k_route, alpha)
+    ref = oracle.route(w.Q, w.cu_seqlens, w.U, w.sigma, k_route)
+    np.testing.assert_allclose(alpha.cpu().numpy(), ref, atol=1e-5)
+    assert np.allclose(np.abs(ref).max(-1), 1.0)
+
+
+# ----------------------------------------------------------------- standalone key edit
+
+def _check_edit(w, Kout, alpha=None, head_enable=None):
+    ref = oracle.edit_keys(w.K, w.mask, w.cu_seqlens, w.U, alpha=alpha, gain=w.gain, head_enable=head_enable)
+    got = Kout.double().cpu().numpy()
+    hl = w.mask != 0
+    # rows that are not highlighted (or belong to an unselected head) are bit-identical to the input
+    assert np.array_equal(got[~hl], w.K[~hl].astype(np.float64))
+    if head_enable is not None:
+        off = np.asarray(head_enable) == 0
+        assert np.array_equal(got[:, off], w.K[:, off].astype(np.float64))
+    rowmax = np.abs(ref).max(axis=-1, keepdims=True)
+    rel = np.abs(got - ref) / np.maximum(rowmax, 1e-30)
+    # fp32: max relative error 1e-3 of the row's largest entry; bf16: one rounding of the result (2^-8 of row max)
+    tol = 1e-3 if w.dtype == "f32" else 2.0 ** -8
+    assert rel.max() <= tol, rel.max()
+    return float(rel.max())
+
+
+@pytest.mark.parametrize("name", ["C1", "C2", "C3", "C4", "C5", "C2s100"])
+def test_edit_keys_configs(name):
+    w = inputs.make_workload(name)
+    alpha = oracle.route(w.Q, w.cu_seqlens, w.U, w.sigma, 0) if w.n_experts > 1 else None
+    dev = H.device_tensors(w)
+    _check_edit(w, H.run_edit(w, dev, alpha=alpha), alpha=alpha)
+    _check_edit(w, H.run_edit(w, dev, alpha=alpha, in_place=True), alpha=alpha)
+
+
+def test_edit_keys_edge_cases():
+    for kw in [dict(lens=[1], mask_kind="all"), dict(lens=[130, 0, 77], mask_kind="runs", highlight=0.5),
+               dict(lens=[64], mask_kind="none"), dict(lens=[200], rank=1), dict(lens=[200], rank=64, n_experts=2)]:
+        base = dict(seed=9, dtype="bf16", n_q_heads=4, n_kv_heads=2, head_dim=128, rank=16, gain=-0.5)
+        base.update(kw)
+        w = inputs.make_custom(**base)
+        alpha = None
+        if w.n_experts > 1:
+            alpha = np.random.default_rng(1).uniform(-1, 1, size=(w.batch, w.n_kv_heads, w.n_experts))
+        he = np.array([0, 1], dtype=np.uint8)
+        _check_edit(w, H.run_edit(w, alpha=alpha, head_enable=he), alpha=alpha, head_enable=he)
+    w = inputs.make_custom(seed=10, dtype="f32", lens=[50, 60], n_q_heads=2, n_kv_heads=2, head_dim=64, rank=7,
+                           gain=[2.0, -5.0], highlight=0.3)
+    assert _check_edit(w, H.run_edit(w)) < 1e-5
+
+
+# ----------------------------------------------------------------- fused attention: small and edge cases
+
+def _fused_vs_oracle(w, alpha=None, head_enable=None, rows=None, force_varlen=False, label=""):
+    O, LSE = H.run_fused(w, alpha=alpha, head_enable=head_enable, force_varlen=force_varlen)
+    Oref, Lref, idx = H.oracle_rows(w, rows, alpha=alpha, head_enable=head_enable)
+    mx, mean = H.check_attention(O[idx], Oref, label)
+    np.testing.assert_allclose(LSE[idx], Lref, atol=2e-2)
+    return mx, mean
+
+
+def test_fused_c1_full():
+    w = inputs.make_workload("C1")
+    _fused_vs_oracle(w, label="C1")
+
+
+@pytest.mark.parametrize("d,Hq,Hkv,r", [(128, 4, 1, 32), (128, 7, 1, 64), (64, 2, 2, 16), (128, 2, 2, 128),
+                                        (64, 4, 2, 1), (128, 2, 1, 8)])
+@pytest.mark.parametrize("g", [0.5, -0.5, 2.0, -5.0])
+def test_fused_small_shapes(d, Hq, Hkv, r, g):
+    w = inputs.make_custom(seed=100 + r, dtype="bf16", lens=[300], n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, rank=r,
+                           gain=g, highlight=0.2)
+    _fused_vs_oracle(w, label="d%d r%d g%g" % (d, r, g))
+
+
+@pytest.mark.parametrize("lens", [[1], [127], [128], [129], [257, 1, 0, 300], [5, 640]])
+def test_fused_ragged_lengths(lens):
+    w = inputs.make_custom(seed=7, dtype="bf16", lens=lens, n_q_heads=4, n_kv_heads=2, head_dim=128, rank=16,
+                           gain=1.0, mask_kind="runs", highlight=0.3)
+    _fused_vs_oracle(w, label=str(lens))
+
+
+def test_fused_mask_patterns_and_head_enable():
+    for kind in ["none", "all"]:
+        w = inputs.make_custom(seed=8, dtype="bf16", lens=[384], n_q_heads=4, n_kv_heads=2, head_dim=128, rank=32,
+                               gain=1.0, mask_kind=kind)
+        _fused_vs_oracle(w, label=kind)
+    w = inputs.make_custom(seed=8, dtype="bf16", lens=[384], n_q_heads=4, n_kv_heads=2, head_dim=128, rank=32,
+                           gain=1.5, mask_kind="none")
+    w.mask[127:130] = 1             # a span that straddles a key-tile boundary
+    w.mask[383] = 1                 # the very last token
+    he = np.array([1, 0], dtype=np.uint8)
+    _fused_vs_oracle(w, head_enable=he, label="straddle")
+
+
+def test_fused_unsteered_paths_are_bitwise_identical():
+    # g = 0, an empty mask and "no steering arguments" all run the same arithmetic
+    w = inputs.make_custom(seed=12, dtype="bf16", lens=[300, 200], n_q_heads=4, n_kv_heads=2, head_dim=128, rank=32,
+                           gain=1.0, highlight=0.3)
+    dev = H.device_tensors(w)
+    base, _ = H.run_fused(w, dev, steer=False)
+    w0 = inputs.make_custom(seed=12, dtype="bf16", lens=[300, 200], n_q_heads=4, n_kv_heads=2, head_dim=128, rank=32,
+                            gain=0.0, highlight=0.3)
+    dev0 = dict(dev); dev0["gain"] = torch.zeros_like(dev["gain"])
+    g0, _ = H.run_fused(w0, dev0)
+    devm = dict(dev); devm["mask"] = torch.zeros_like(dev["mask"])
+    m0, _ = H.run_fused(w, devm)
+    assert np.array_equal(base, g0) and np.array_equal(base, m0)
+    steered, _ = H.run_fused(w, dev)
+    assert not np.array_equal(base, steered)
+    # the inputs are never modified
+    assert torch.equal(dev["K"], torch.from_numpy(w.K).cuda().to(torch.bfloat16))
+
+
+def test_fused_adaseka_blend_small():
+    w = inputs.make_custom(seed=13, dtype="bf16", lens=[500, 140], n_q_heads=8, n_kv_heads=2, head_dim=128, rank=32,
+                           n_experts=4, gain=1.0, highlight=0.15)
+    dev = H.device_tensors(w)
+    shp = H.shape_of(w, dev)
+    alpha = torch.empty((w.batch, w.n_kv_heads, 4), device="cuda")
+    binding.adaseka_route(shp, dev["Q"], dev["U"], dev["sigma"], 0, alpha)
+    a = alpha.cpu().numpy().astype(np.float64)
+    _fused_vs_oracle(w, alpha=a, label="adaseka")
+
+
+def test_fused_fixed_layout_equals_packed_layout():
+    w = inputs.make_custom(seed=14, dtype="bf16", lens=[256, 256], n_q_heads=2, n_kv_heads=1, head_dim=64, rank=16,
+                           gain=1.0, highlight=0.2)
+    a, _ = H.run_fused(w)
+    b, _ = H.run_fused(w, force_varlen=True)
+    assert np.array_equal(a, b)
+
+
+def test_host_buffer_entry_point():
+    w = inputs.make_custom(seed=15, dtype="bf16", lens=[300, 300], n_q_heads=4, n_kv_heads=2, head_dim=128, rank=32,
+                           gain=1.0, highlight=0.2)
+    dev = H.device_tensors(w)
+    shp = H.shape_of(w, dev)
+    ws = binding.new_workspace(shp)
+    staging = torch.empty(binding.seka_host_staging_bytes(shp), dtype=torch.uint8, device="cuda")
+    hQ, hK, hV = (dev[k].cpu().pin_memory() for k in "QKV")
+    hmask = dev["mask"].cpu().pin_memory()
+    hO = torch.empty_like(hQ).pin_memory()
+    hlse = torch.empty((w.total_tokens, w.n_q_heads), dtype=torch.float32).pin_memory()
+    binding.seka_attention_fwd_host(shp, hQ, hK, hV, hO, hlse, hmask, dev["U"], None, dev["gain"], None, staging, ws)
+    assert binding.seka_poll_status(ws) == binding.SEKA_OK
+    ref, lse = H.run_fused(w, dev)
+    assert np.array_equal(hO.double().numpy(), ref) and np.array_equal(hlse.double().numpy(), lse)
+
+
+# ----------------------------------------------------------------- fused attention: the five configurations at full size
+
+@pytest.mark.parametrize("name,nrows", [("C2", 96), ("C3", 64), ("C4", 96), ("C5", 24), ("C2s70", 48)])
+def test_fused_full_size_sampled_rows(name, nrows):
+    w = inputs.make_workload(name)
+    alpha = None
+    dev = H.device_tensors(w)
+    if w.n_experts > 1:
+        shp = H.shape_of(w, dev)
+        a = torch.empty((w.batch, w.n_kv_heads, w.n_experts), device="cuda")
+        binding.adaseka_route(shp, dev["Q"], dev["U"], dev["sigma"], 0, a)
+        alpha = a.cpu().numpy().astype(np.float64)
+        np.testing.assert_allclose(alpha, oracle.route(w.Q, w.cu_seqlens, w.U, w.sigma, 0), atol=1e-5)
+    rows = H.sampled_rows(w, nrows, seed=1)
+    O, LSE = H.run_fused(w, dev, alpha=alpha)
+    assert np.isfinite(O).all() and np.isfinite(LSE).all()          # every row was written
+    Oref, Lref, idx = H.oracle_rows(w, rows, alpha=alpha)
+    mx, mean = H.check_attention(O[idx], Oref, name)
+    np.testing.assert_allclose(LSE[idx], Lref, atol=2e-2)
+    print("%s: rows %d max abs %.3e mean abs %.3e" % (name, len(idx), mx, mean))
