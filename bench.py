@@ -1,0 +1,282 @@
+#!/usr/bin/env python
+"""Benchmark of the SEKA fused steered-attention hot path on B200.
+
+One step = one pass of the whole path over one batch of the 8B-shaped prefill workload
+(B=4, 32 query / 8 KV heads, head_dim 128, L=4096, bf16, rank-32 projector per KV head, 10 % of
+the tokens highlighted in 1-3 spans, g=1): operand preparation + the fused steered attention
+kernel, called through the C ABI.  Prints ONE JSON line (rank 0).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank processes its own
+batch of the same shape (sequences are independent: no data-path collective, weak scaling); the
+timed region is bracketed by a barrier and a device synchronise and the maximum over ranks is used.
+``--impl reference`` times the fp64 CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "SEKA fused attention TFLOP/s (% BF16 peak); overhead vs g=0, 8B shape"
+WORKLOAD = "C2: 8B-shaped prefill layer B=4 Hq=32 Hkv=8 d=128 L=4096 bf16, rank 32, ~10% highlighted spans, g=1"
+# DRAM bytes of one fused-kernel launch on this workload from the ncu capture summarised in
+# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture exists.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"bf16_burst": d.get("bf16_tflops"), "bf16_sustained": d.get("bf16_tflops_sustained"),
+                "hbm_gbs": d.get("hbm_gbs"), "source": "measured"}
+    return {"bf16_burst": 1590.0, "bf16_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.out = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                         stdout=self.out, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self, t0: float, t1: float) -> dict:
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        self.out.flush(); self.out.seek(0)
+        rows = []
+        for line in self.out.read().splitlines():
+            p = [x.strip() for x in line.split(",")]
+            if len(p) < 8:
+                continue
+            try:
+                ts = time.mktime(time.strptime(p[0].split(".")[0], "%Y/%m/%d %H:%M:%S")) + float("0." + p[0].split(".")[1])
+                rows.append((ts, float(p[1]), float(p[2]), p[4:8]))
+            except (ValueError, IndexError):
+                continue
+        self.out.close()
+        os.unlink(self.out.name)
+        inside = [r for r in rows if t0 - 0.05 <= r[0] <= t1 + 0.05] or rows
+        if not inside:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = sorted({names[i] for r in inside for i in range(4) if r[3][i].lower() == "active"})
+        return {"sm_mhz": float(np.median([r[1] for r in inside])), "sm_max_mhz": float(inside[0][2]),
+                "reasons": reasons, "samples": len(inside)}
+
+
+def cpu_oracle_sample(w, budget_s: float, seed: int = 0):
+    """Times the fp64 oracle (as it stands) on complete query rows of the workload until the budget is spent.
+    Returns (flops done, seconds, rows)."""
+    import oracle
+    rng = np.random.default_rng(seed)
+    Kp = oracle.edit_keys(w.K, w.mask, w.cu_seqlens, w.U, gain=w.gain)
+    Q64 = w.Q.astype(np.float64); V64 = w.V.astype(np.float64)
+    flops = 0.0; secs = 0.0; nrows = 0
+    chunk = 4
+    while secs < budget_s:
+        rows = [np.sort(rng.choice(int(w.cu_seqlens[b + 1] - w.cu_seqlens[b]), size=chunk, replace=False)).astype(np.int32)
+                for b in range(w.batch)]
+        t0 = time.perf_counter()
+        oracle.attention_rows(Q64, Kp, V64, w.cu_seqlens, rows)
+        dt = time.perf_counter() - t0
+        secs += dt
+        for rb in rows:
+            flops += float(np.sum(4.0 * w.head_dim * w.n_q_heads * (rb.astype(np.float64) + 1.0)))
+            nrows += len(rb)
+        if dt < budget_s / 8:
+            chunk = min(chunk * 2, 256)
+    return flops, secs, nrows
+
+
+def run_reference(args, rank: int):
+    """The reference arm: the CPU oracle on a bounded sample of the same workload, K timed steps."""
+    if rank != 0:
+        return
+    import oracle
+    from paper_2603_01281_b200 import inputs
+    w = inputs.make_workload("C2")
+    per_step = max(0.5, min(10.0, 60.0 / max(1, args.steps + args.warmup)))
+    for i in range(args.warmup):
+        cpu_oracle_sample(w, per_step, seed=100 + i)
+    tot_f = tot_s = 0.0; rows = 0
+    for i in range(args.steps):
+        f, s, r = cpu_oracle_sample(w, per_step, seed=i)
+        tot_f += f; tot_s += s; rows += r
+    val = tot_f / tot_s / 1e12
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot_s / max(1, args.steps),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "sample": "%d complete query rows per step on average" % (rows // max(1, args.steps))},
+            "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": oracle.threads(), "kind": "oracle",
+                             "sample": "%d random complete query rows (all 32 heads) of the C2 workload" % rows},
+            "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle work for cpu_baseline")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2603_01281_b200 import binding, inputs
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    binding.load()
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None    # started early: nvidia-smi takes a while to come up
+    # every rank: its own batch of the same shape (sequences are independent units)
+    w = inputs.make_workload("C2", seed_offset=rank)
+    dt = torch.bfloat16
+    dev = {k: torch.from_numpy(getattr(w, k)).cuda().to(dt) for k in ("Q", "K", "V")}
+    mask = torch.from_numpy(w.mask).cuda(); U = torch.from_numpy(w.U).cuda(); gain = torch.from_numpy(w.gain).cuda()
+    shp = binding.make_shape(batch=w.batch, max_seqlen=w.max_seqlen, n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads,
+                             head_dim=w.head_dim, rank=w.rank, n_experts=1, dtype=dt)
+    ws = binding.new_workspace(shp)
+    O = torch.empty_like(dev["Q"])
+    flops_step = w.attention_flops()
+    tokens_step = w.total_tokens
+
+    def step(steer=True):
+        binding.seka_attention_fwd(shp, dev["Q"], dev["K"], dev["V"], O, None, mask if steer else None,
+                                   U if steer else None, None, gain, None, ws)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(nsteps, steer=True):
+        ev0 = torch.cuda.Event(enable_timing=True); ev1 = torch.cuda.Event(enable_timing=True)
+        barrier()
+        t0 = time.time()
+        ev0.record()
+        for _ in range(nsteps):
+            step(steer)
+        ev1.record()
+        barrier()
+        t1 = time.time()
+        ms = ev0.elapsed_time(ev1)
+        if world > 1:
+            t = torch.tensor([ms], device="cuda"); dist.all_reduce(t, op=dist.ReduceOp.MAX); ms = float(t.item())
+        return ms, t0, t1
+
+    for _ in range(args.warmup):
+        step(True)
+    torch.cuda.synchronize()
+    launches0 = binding.seka_launch_count()
+    ms, t0, t1 = timed(args.steps, True)
+    launches = binding.seka_launch_count() - launches0
+    clocks = sampler.stop(t0, t1) if sampler else None
+    st = binding.seka_poll_status(ws)
+    if st != binding.SEKA_OK:
+        raise SystemExit("device status: " + binding.status_string(st))
+
+    # the same kernel with steering off (g = 0 path), interleaved afterwards for the overhead figure
+    for _ in range(3):
+        step(False)
+    ms0, _, _ = timed(args.steps, False)
+    ms1, _, _ = timed(args.steps, True)
+
+    # end to end through the host-buffer entry point: H2D of Q, K, V, mask and D2H of O every step
+    staging = torch.empty(binding.seka_host_staging_bytes(shp), dtype=torch.uint8, device="cuda")
+    hQ, hK, hV = (dev[k].cpu().pin_memory() for k in ("Q", "K", "V"))
+    hmask = mask.cpu().pin_memory(); hO = torch.empty_like(hQ).pin_memory()
+    e2e_steps = max(3, min(args.steps, 20))
+
+    def e2e_step():
+        binding.seka_attention_fwd_host(shp, hQ, hK, hV, hO, None, hmask, U, None, gain, None, staging, ws)
+    for _ in range(2):
+        e2e_step()
+    ev0 = torch.cuda.Event(enable_timing=True); ev1 = torch.cuda.Event(enable_timing=True)
+    barrier(); ev0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    ev1.record(); barrier()
+    e2e_ms = ev0.elapsed_time(ev1)
+    if world > 1:
+        t = torch.tensor([e2e_ms], device="cuda"); dist.all_reduce(t, op=dist.ReduceOp.MAX); e2e_ms = float(t.item())
+    h2d = sum(t.numel() * t.element_size() for t in (hQ, hK, hV, hmask)); d2h = hO.numel() * hO.element_size()
+
+    if rank == 0:
+        peaks = measured_peaks()
+        ms_step = ms / args.steps
+        value = world * flops_step * args.steps / (ms * 1e-3) / 1e12
+        per_gpu = value / world
+        line = {
+            "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "l2": "inputs larger than L2 (Q+K+V+O = 336 MB per step vs 126 MB L2)",
+                       "batch_per_gpu": w.batch, "highlight_fraction": w.meta["highlight_fraction"]},
+            "clocks": clocks,
+            "e2e": {"value": world * flops_step * e2e_steps / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+                    "ms_per_step": e2e_ms / e2e_steps},
+            "gpu_launches": int(launches),
+            "roofline": {"bound": "tensor", "achieved": per_gpu, "peak": peaks["bf16_burst"], "unit": "TFLOP/s",
+                         "frac": per_gpu / peaks["bf16_burst"], "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
+                         "peak_source": "of %s (cuBLAS bf16 burst); sustained %.1f -> %.3f, nominal 2250 -> %.3f" % (
+                             peaks["source"], peaks["bf16_sustained"], per_gpu / peaks["bf16_sustained"], per_gpu / 2250.0)},
+            "extra": {"tokens_per_s": world * tokens_step * args.steps / (ms * 1e-3),
+                      "ms_per_step_g0": ms0 / args.steps, "ms_per_step_steered": ms1 / args.steps,
+                      "overhead_vs_g0": ms1 / ms0 - 1.0, "flops_per_step": flops_step},
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            import oracle
+            f, s, r = cpu_oracle_sample(w, args.cpu_budget)
+            line["cpu_baseline"] = {"value": f / s / 1e12, "unit": "TFLOP/s", "cores": oracle.threads(), "kind": "oracle",
+                                    "sample": "%d random complete query rows (all 32 heads) of the same workload, %.1f s" % (r, s)}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
