@@ -121,6 +121,36 @@ seka_status seka_attention_fwd_host(const seka_shape* shape, const void* h_Q, co
                                     void* staging, size_t staging_bytes,
                                     void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/*
+ * seka_edit_keys without a workspace, for callers that cannot allocate device memory.  (The paper
+ * has no counterpart for this entry point: it exists for the integration, not for the method.)
+ *
+ * Some hosts of this library may not call cudaMalloc at the point where the key cache has to be
+ * edited: an inference server that hands its whole memory budget to a pre-sized KV-cache pool at
+ * start-up, a plug-in that runs inside another framework's stream callback, or code that has
+ * already frozen its allocator.  seka_edit_keys needs a scratch buffer (the compacted list of
+ * highlighted tokens) that such a caller has nowhere to get.  This variant keeps that scratch in
+ * a fixed array inside the library's device image instead; it computes exactly what
+ * seka_edit_keys computes and takes the same tensors, minus the workspace.
+ *
+ *  - Limit: total tokens <= SEKA_STATIC_MAX_TOKENS.  A larger shape is refused with
+ *    SEKA_ERR_UNSUPPORTED before anything is launched; use seka_edit_keys with a workspace there.
+ *  - Cost: every GPU that loads the library holds the array (4 * SEKA_STATIC_MAX_TOKENS + 256
+ *    bytes) until the process exits, whether or not this entry point is ever called.
+ *  - The call itself performs no cudaMalloc / cudaFree and uses no allocating library routine.
+ *    The first call on each device looks up the array's device address (once, with that device
+ *    current); make that first call outside any stream capture.
+ *  - All calls on one device share the one array.  Its contents are whatever the previous call
+ *    left; the call clears what it needs (the list counter) on `cuda_stream` first.  Two calls
+ *    that may overlap on the GPU (different streams, or different host threads without ordering)
+ *    race on the array: serialise them, or give the overlapping ones seka_edit_keys with
+ *    separate workspaces.
+ */
+#define SEKA_STATIC_MAX_TOKENS 262144
+seka_status seka_edit_keys_static(const seka_shape* shape, const void* K_in, void* K_out,
+                                  const uint8_t* mask, const float* U, const float* alpha,
+                                  const float* gain, const uint8_t* head_enable, void* cuda_stream);
+
 /* Clears the device status word (async on the stream); call once before first use of a workspace. */
 seka_status seka_reset_status(void* workspace, void* cuda_stream);
 /* Synchronises the stream and returns the device status word (SEKA_OK if no wait ran out). */

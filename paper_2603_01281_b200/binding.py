@@ -20,7 +20,8 @@ SEKA_F32, SEKA_BF16 = 0, 1
 
 EXPORTS = ["seka_workspace_bytes", "seka_edit_keys", "adaseka_route", "seka_attention_fwd",
            "seka_host_staging_bytes", "seka_attention_fwd_host", "seka_reset_status", "seka_poll_status",
-           "seka_status_string", "seka_launch_count"]
+           "seka_status_string", "seka_launch_count", "seka_edit_keys_static"]
+SEKA_STATIC_MAX_TOKENS = 262144
 
 
 class SekaShape(ctypes.Structure):
@@ -52,6 +53,8 @@ def load() -> ctypes.CDLL:
         lib.seka_host_staging_bytes.argtypes = [sp]; lib.seka_host_staging_bytes.restype = ctypes.c_size_t
         lib.seka_edit_keys.argtypes = [sp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
         lib.seka_edit_keys.restype = ctypes.c_int
+        lib.seka_edit_keys_static.argtypes = [sp, vp, vp, vp, vp, vp, vp, vp, vp]
+        lib.seka_edit_keys_static.restype = ctypes.c_int
         lib.adaseka_route.argtypes = [sp, vp, vp, vp, ctypes.c_int32, vp, vp]
         lib.adaseka_route.restype = ctypes.c_int
         lib.seka_attention_fwd.argtypes = [sp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
@@ -121,6 +124,14 @@ def seka_edit_keys(shape: SekaShape, K_in, K_out, mask, U, alpha, gain, head_ena
     _check(load().seka_edit_keys(ctypes.byref(shape), _ptr(K_in), _ptr(K_out), _ptr(mask), _ptr(U), _ptr(alpha),
                                  _ptr(gain), _ptr(head_enable), _ptr(workspace),
                                  workspace.numel() if workspace is not None else 0, _stream()), "seka_edit_keys")
+
+
+def seka_edit_keys_static(shape: SekaShape, K_in, K_out, mask, U, alpha, gain, head_enable) -> None:
+    """seka_edit_keys for callers that cannot allocate: the scratch is a fixed array inside the library
+    (at most SEKA_STATIC_MAX_TOKENS tokens; calls that overlap on the GPU race on it)."""
+    _check(load().seka_edit_keys_static(ctypes.byref(shape), _ptr(K_in), _ptr(K_out), _ptr(mask), _ptr(U),
+                                        _ptr(alpha), _ptr(gain), _ptr(head_enable), _stream()),
+           "seka_edit_keys_static")
 
 
 def adaseka_route(shape: SekaShape, Q, U, sigma, k_route: int, alpha_out) -> None:

@@ -1,4 +1,6 @@
 // Standalone key-editing kernel (the hook of Algorithm 1 / Algorithm 2 applied to a key tensor in HBM).
+#include <mutex>
+
 #include "seka_kernels.h"
 
 namespace seka {
@@ -118,5 +120,63 @@ extern "C" seka_status seka_edit_keys(const seka_shape* shape, const void* K_in,
         launch_edit_rows<float>(shape, K_in, K_out, list, status + 2, U, alpha, gain, head_enable, st);
     else
         launch_edit_rows<__nv_bfloat16>(shape, K_in, K_out, list, status + 2, U, alpha, gain, head_enable, st);
+    return cudaGetLastError() == cudaSuccess ? SEKA_OK : SEKA_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------- allocation-free variant
+namespace seka {
+
+// Scratch of seka_edit_keys_static, resident in the device image of every GPU that loads the
+// library: a 256-byte header whose first word is the list counter, then one int32 per token.
+// In host code this name is only a handle for cudaGetSymbolAddress, never a device pointer.
+static __device__ __align__(256) unsigned char g_static_scratch[256 + (size_t)SEKA_STATIC_MAX_TOKENS * 4];
+
+// Device address of the array on the current device, looked up once per device.
+static seka_status static_scratch_of_current_device(char** out) {
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static char* table[kMaxDevices] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SEKA_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return SEKA_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(mu);
+    if (table[dev] == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return SEKA_ERR_CUDA;
+        table[dev] = static_cast<char*>(p);
+    }
+    *out = table[dev];
+    return SEKA_OK;
+}
+
+}  // namespace seka
+
+extern "C" seka_status seka_edit_keys_static(const seka_shape* shape, const void* K_in, void* K_out,
+                                             const uint8_t* mask, const float* U, const float* alpha,
+                                             const float* gain, const uint8_t* head_enable, void* cuda_stream) {
+    using namespace seka;
+    seka_status stc = validate_shape(shape);
+    if (stc != SEKA_OK) return stc;
+    const int T = shape_total_tokens(shape);
+    if (T > SEKA_STATIC_MAX_TOKENS) return SEKA_ERR_UNSUPPORTED;   // beyond the built-in scratch
+    if (T == 0) return SEKA_OK;
+    if (!K_in || !K_out || !mask || !U || !gain) return SEKA_ERR_INVALID_ARG;
+    if (((uintptr_t)K_in | (uintptr_t)K_out) & 15) return SEKA_ERR_INVALID_ARG;
+    char* scratch = nullptr;
+    stc = static_scratch_of_current_device(&scratch);
+    if (stc != SEKA_OK) return stc;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int* count = reinterpret_cast<int*>(scratch);
+    int* list = reinterpret_cast<int*>(scratch + 256);
+    const size_t esz = shape->dtype == SEKA_F32 ? 4 : 2;
+    if (K_out != K_in) {
+        const size_t bytes = (size_t)T * shape->n_kv_heads * shape->head_dim * esz;
+        if (cudaMemcpyAsync(K_out, K_in, bytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return SEKA_ERR_CUDA;
+    }
+    launch_compact_mask(mask, T, list, count, st);     // zeroes the counter on the stream first
+    if (shape->dtype == SEKA_F32)
+        launch_edit_rows<float>(shape, K_in, K_out, list, count, U, alpha, gain, head_enable, st);
+    else
+        launch_edit_rows<__nv_bfloat16>(shape, K_in, K_out, list, count, U, alpha, gain, head_enable, st);
     return cudaGetLastError() == cudaSuccess ? SEKA_OK : SEKA_ERR_CUDA;
 }
