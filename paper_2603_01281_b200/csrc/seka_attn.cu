@@ -1,14 +1,21 @@
 // Fused SEKA / AdaSEKA steered causal GQA attention forward for sm_100a.
 //
-// One CTA owns a tile of 128 queries of one query head and walks the key tiles 0 .. diagonal:
-//   TMA (128-byte swizzle) stages K and V tiles in shared memory, double buffered;
-//   key tiles that contain highlighted tokens are edited in place, k' = k + g * sum_m alpha_m U_m U_m^T k
-//     (Section 2 / Section 3.3; hook of Algorithm 1/2), by warp-level tensor-core MMAs (seka_edit_tile.cuh);
-//   S = Q K'^T runs on tcgen05 with the accumulator in tensor memory (score of Section 2);
-//   each thread owns one query row: causal mask on the diagonal tile, online softmax in base 2,
-//     P written to shared memory as bf16 in UMMA operand layout;
-//   P V runs on tcgen05 into tensor memory and is folded into the running output in registers.
-// Neither K' nor the score matrix ever reaches global memory; K and V are read only.
+// One CTA (16 warps) owns two consecutive tiles of 128 queries of one query head ("A" = lower rows,
+// "B" = upper rows) and walks the key tiles 0 .. diagonal.  Warp roles:
+//   warp 0        TMA producer: Q tiles once, then K and V tiles (128-byte swizzle) through two
+//                 shared-memory rings, throttled by "empty" mbarriers the tensor core signals;
+//   warps 12-15   key editors: for a staged K tile that contains highlighted tokens of a steered head,
+//                 k' = k + g * sum_m alpha_m U_m U_m^T k in place (Section 2 / Section 3.3, hook of
+//                 Algorithm 1/2) on warp-level MMAs (seka_edit_tile.cuh); then the tile is "ready";
+//   warp 1        MMA issuer: S_x = Q_x K'^T and O_x += P_x V on tcgen05 with all accumulators in
+//                 tensor memory (S_A, S_B, O_A, O_B = 512 columns); P_x is read from tensor memory;
+//   warps 4-7 / 8-11  softmax of tile A / B, one query row per thread: causal mask on the diagonal
+//                 tile, online softmax in base 2 with a lazily updated running maximum, P written
+//                 back as bf16 over the consumed score columns, O rescaled in tensor memory only when
+//                 the maximum moved by more than 2^8; final normalisation and store.
+// While one tile's softmax runs, the tensor core works on the other tile.  Neither K' nor the score
+// matrix ever reaches global memory; K and V are read only.  Every wait is bounded: a wait that runs
+// out raises the CTA's abort flag, every role leaves its loop, and the status word reports it.
 #include <math.h>
 
 #include "seka_edit_tile.cuh"
@@ -32,56 +39,72 @@ struct AttnParams {
 };
 
 constexpr int BM = 128, BN = 128;
+constexpr int NK = 3, NV = 2;               // K and V ring depths
+constexpr int NTHREADS = 512;
 constexpr uint32_t BLK_BYTES = 128 * 128;   // one [128 x 64] bf16 block
+constexpr float LAZY_RESCALE_LOG2 = 8.0f;   // the running maximum is only raised when it moved by more than this
 
 template <int D>
 struct SmemLayout {
     static constexpr uint32_t TILE = (D / 64) * BLK_BYTES;
-    static constexpr uint32_t Q = 0;
-    static constexpr uint32_t K = Q + TILE;          // 2 stages
-    static constexpr uint32_t V = K + 2 * TILE;      // 2 stages
-    static constexpr uint32_t P = V + 2 * TILE;      // [128 x 128] bf16
-    static constexpr uint32_t ROWFLAG = P + 2 * BLK_BYTES;   // 128 bytes
-    static constexpr uint32_t COLSCALE = ROWFLAG + 128;      // 128 floats
-    static constexpr uint32_t BARS = COLSCALE + 512;         // 8 mbarriers
-    static constexpr uint32_t MISC = BARS + 64;              // tmem holder, abort flag
+    static constexpr uint32_t Q = 0;                       // 2 tiles
+    static constexpr uint32_t K = Q + 2 * TILE;            // NK stages
+    static constexpr uint32_t V = K + NK * TILE;           // NV stages
+    static constexpr uint32_t ROWFLAG = V + NV * TILE;     // NK x 128 bytes
+    static constexpr uint32_t COLSCALE = ROWFLAG + NK * 128;   // 128 floats
+    static constexpr uint32_t BARS = COLSCALE + 512;       // mbarriers
+    static constexpr uint32_t NBARS = 2 + 3 * NK + 2 * NV + 6;
+    static constexpr uint32_t MISC = BARS + NBARS * 8;     // tmem holder, abort flag
     static constexpr uint32_t TOTAL = MISC + 16;
-    static constexpr uint32_t DYN_BYTES = TOTAL + 1024;      // slack for the 1024-byte alignment
+    static constexpr uint32_t DYN_BYTES = TOTAL + 1024;    // slack for the 1024-byte alignment
 };
 
-template <typename OutT> __device__ __forceinline__ void store_row(OutT* dst, const float* o, int n, float inv);
-template <> __device__ __forceinline__ void store_row<__nv_bfloat16>(__nv_bfloat16* dst, const float* o, int n, float inv) {
+// all lanes of a warp wait on the same barrier and then agree on the outcome
+__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status, int where) {
+    const bool ok = mbar_wait(bar, parity, abort_flag, status, where);
+    return __all_sync(0xffffffffu, ok);
+}
+
+template <typename OutT> __device__ __forceinline__ void store_chunk32(OutT* dst, const uint32_t (&v)[32], float inv);
+template <> __device__ __forceinline__ void store_chunk32<__nv_bfloat16>(__nv_bfloat16* dst, const uint32_t (&v)[32], float inv) {
     uint4* d4 = reinterpret_cast<uint4*>(dst);
 #pragma unroll
-    for (int c = 0; c < n / 8; ++c)
-        d4[c] = make_uint4(pack_bf16(o[8 * c] * inv, o[8 * c + 1] * inv), pack_bf16(o[8 * c + 2] * inv, o[8 * c + 3] * inv),
-                           pack_bf16(o[8 * c + 4] * inv, o[8 * c + 5] * inv), pack_bf16(o[8 * c + 6] * inv, o[8 * c + 7] * inv));
+    for (int c = 0; c < 4; ++c)
+        d4[c] = make_uint4(pack_bf16(__uint_as_float(v[8 * c]) * inv, __uint_as_float(v[8 * c + 1]) * inv),
+                           pack_bf16(__uint_as_float(v[8 * c + 2]) * inv, __uint_as_float(v[8 * c + 3]) * inv),
+                           pack_bf16(__uint_as_float(v[8 * c + 4]) * inv, __uint_as_float(v[8 * c + 5]) * inv),
+                           pack_bf16(__uint_as_float(v[8 * c + 6]) * inv, __uint_as_float(v[8 * c + 7]) * inv));
 }
-template <> __device__ __forceinline__ void store_row<float>(float* dst, const float* o, int n, float inv) {
+template <> __device__ __forceinline__ void store_chunk32<float>(float* dst, const uint32_t (&v)[32], float inv) {
     float4* d4 = reinterpret_cast<float4*>(dst);
 #pragma unroll
-    for (int c = 0; c < n / 4; ++c)
-        d4[c] = make_float4(o[4 * c] * inv, o[4 * c + 1] * inv, o[4 * c + 2] * inv, o[4 * c + 3] * inv);
+    for (int c = 0; c < 8; ++c)
+        d4[c] = make_float4(__uint_as_float(v[4 * c]) * inv, __uint_as_float(v[4 * c + 1]) * inv,
+                            __uint_as_float(v[4 * c + 2]) * inv, __uint_as_float(v[4 * c + 3]) * inv);
 }
 
 template <int D, typename OutT>
-__global__ void __launch_bounds__(128, 1)
+__global__ void __launch_bounds__(NTHREADS, 1)
 seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                      const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
     using SL = SmemLayout<D>;
     constexpr int NBLK = D / 64;
-    constexpr uint32_t TMEM_COLS = 256;   // S: columns [0,128), P*V: columns [128, 128 + D)
+    constexpr uint32_t TMEM_COLS = 512;
+    constexpr uint32_t COL_S = 0, COL_O = 256;     // S_x at COL_S + 128 x, O_x at COL_O + D x
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t* sQ = smem + SL::Q;
-    uint8_t* sP = smem + SL::P;
     uint8_t* rowflag = smem + SL::ROWFLAG;
     float* colscale = reinterpret_cast<float*>(smem + SL::COLSCALE);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SL::BARS);
-    uint64_t* bar_q = bars + 0;
-    uint64_t* bar_kv = bars + 1;   // [2]
-    uint64_t* bar_s = bars + 3;
-    uint64_t* bar_pv = bars + 4;
+    uint64_t* q_full = bars;                 // [2]   TMA bytes landed
+    uint64_t* k_full = q_full + 2;           // [NK]  TMA bytes landed
+    uint64_t* k_ready = k_full + NK;         // [NK]  128 editor arrivals: tile may be multiplied
+    uint64_t* k_empty = k_ready + NK;        // [NK]  tensor core finished reading the stage
+    uint64_t* v_full = k_empty + NK;         // [NV]
+    uint64_t* v_empty = v_full + NV;         // [NV]
+    uint64_t* s_full = v_empty + NV;         // [2]   scores of tile x are in tensor memory
+    uint64_t* p_full = s_full + 2;           // [2]   128 softmax arrivals: P_x written, O_x rescaled
+    uint64_t* o_full = p_full + 2;           // [2]   last P V of tile x finished
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + SL::MISC);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + SL::MISC + 4);
 
@@ -89,18 +112,26 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 
     // heaviest query tiles first; CTAs of one (sequence, KV head) are neighbours
     const int per_qt = p.B * p.Hq;
-    const int qt = p.n_qt - 1 - (int)(blockIdx.x / per_qt);
+    const int n_qt2 = (p.n_qt + 1) >> 1;
+    const int qt2 = n_qt2 - 1 - (int)(blockIdx.x / per_qt);
     const int rem = (int)(blockIdx.x % per_qt);
     const int b = rem / p.Hq, hq = rem % p.Hq;
     const int hkv = hq / (p.Hq / p.Hkv);
     const int seq0 = p.cu_seqlens ? p.cu_seqlens[b] : b * p.L;
     const int Lb = p.cu_seqlens ? (p.cu_seqlens[b + 1] - seq0) : p.L;
-    if (qt * BM >= Lb) return;                      // nothing allocated yet
-    if (*reinterpret_cast<volatile int*>(p.status) != 0) return;   // an earlier CTA gave up: do not pile on
+    if (qt2 * 2 * BM >= Lb) return;                                    // nothing allocated yet
+    if (*reinterpret_cast<volatile int*>(p.status) != 0) return;      // an earlier CTA gave up: do not pile on
+
+    const int ntiles = (Lb + BN - 1) / BN;
+    const int nA = min(2 * qt2 + 1, ntiles);                           // key tiles of query tile A (last one diagonal)
+    const int nB = ((2 * qt2 + 1) * BM < Lb) ? min(2 * qt2 + 2, ntiles) : 0;   // 0: tile B lies beyond the sequence
+    const int n_kv = max(nA, nB);
 
     if (tid == 0) {
-        mbar_init(bar_q, 1); mbar_init(bar_kv + 0, 1); mbar_init(bar_kv + 1, 1);
-        mbar_init(bar_s, 1); mbar_init(bar_pv, 1);
+        mbar_init(q_full + 0, 1); mbar_init(q_full + 1, 1);
+        for (int i = 0; i < NK; ++i) { mbar_init(k_full + i, 1); mbar_init(k_ready + i, 128); mbar_init(k_empty + i, 1); }
+        for (int i = 0; i < NV; ++i) { mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(s_full + i, 1); mbar_init(p_full + i, 128); mbar_init(o_full + i, 1); }
         *abort_flag = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
@@ -111,108 +142,153 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     // steering parameters of this (sequence, KV head)
     const float g = p.steer ? p.gain[b] : 0.f;
     const bool steer = p.steer && g != 0.f && (p.head_enable == nullptr || p.head_enable[hkv] != 0);
-    if (steer) {
-        const int j = tid;   // 128 threads cover the 128 possible stacked columns
+    if (steer && tid < 128) {
         float cs = 0.f;
-        if (j < p.M * p.rank) cs = g * (p.alpha ? p.alpha[((size_t)b * p.Hkv + hkv) * p.M + j / p.rank] : 1.f);
-        colscale[j] = cs;
+        if (tid < p.M * p.rank) cs = g * (p.alpha ? p.alpha[((size_t)b * p.Hkv + hkv) * p.M + tid / p.rank] : 1.f);
+        colscale[tid] = cs;
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_holder;
-    const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
-    const uint32_t tS = t_lane, tPV = t_lane + 128;
 
-    const int n_kv = qt + 1;
-    constexpr uint32_t KV_BYTES = 2 * SL::TILE;
-    if (tid == 0) {
-        mbar_expect_tx(bar_q, SL::TILE);
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            mbar_expect_tx(q_full + 0, SL::TILE);
 #pragma unroll
-        for (int c = 0; c < NBLK; ++c) tma_load_3d(sQ + c * BLK_BYTES, &tmQ, bar_q, c * 64, hq, seq0 + qt * BM);
-        mbar_expect_tx(bar_kv + 0, KV_BYTES);
+            for (int c = 0; c < NBLK; ++c) tma_load_3d(smem + SL::Q + c * BLK_BYTES, &tmQ, q_full + 0, c * 64, hq, seq0 + qt2 * 2 * BM);
+            if (nB > 0) {
+                mbar_expect_tx(q_full + 1, SL::TILE);
 #pragma unroll
-        for (int c = 0; c < NBLK; ++c) {
-            tma_load_3d(smem + SL::K + c * BLK_BYTES, &tmK, bar_kv + 0, c * 64, hkv, seq0);
-            tma_load_3d(smem + SL::V + c * BLK_BYTES, &tmV, bar_kv + 0, c * 64, hkv, seq0);
-        }
-    }
-    int loads_issued = 1, loads_waited = 0;   // meaningful on thread 0 only
-
-    const size_t fr_head = frag_uint4_per_head(D, p.r_pad);
-    const uint4* fragB = p.frags + (size_t)hkv * fr_head;
-    const uint4* fragA = fragB + fr_head / 2;
-    const int nR16 = p.r_pad / 16;
-
-    constexpr uint32_t IDESC_S = umma_idesc_bf16(BN, false);
-    constexpr uint32_t IDESC_PV = umma_idesc_bf16(D, true);
-
-    float o[D];
-#pragma unroll
-    for (int c = 0; c < D; ++c) o[c] = 0.f;
-    float m_run = -INFINITY, l_run = 0.f;
-    const int row = tid;
-    bool ok = true;
-
-    for (int j = 0; j < n_kv; ++j) {
-        const int s = j & 1;
-        uint8_t* sK = smem + SL::K + s * SL::TILE;
-        uint8_t* sV = smem + SL::V + s * SL::TILE;
-        if (tid == 0 && j + 1 < n_kv) {
-            const int s2 = s ^ 1;
-            mbar_expect_tx(bar_kv + s2, KV_BYTES);
-#pragma unroll
-            for (int c = 0; c < NBLK; ++c) {
-                tma_load_3d(smem + SL::K + s2 * SL::TILE + c * BLK_BYTES, &tmK, bar_kv + s2, c * 64, hkv, seq0 + (j + 1) * BN);
-                tma_load_3d(smem + SL::V + s2 * SL::TILE + c * BLK_BYTES, &tmV, bar_kv + s2, c * 64, hkv, seq0 + (j + 1) * BN);
+                for (int c = 0; c < NBLK; ++c)
+                    tma_load_3d(smem + SL::Q + SL::TILE + c * BLK_BYTES, &tmQ, q_full + 1, c * 64, hq, seq0 + (qt2 * 2 + 1) * BM);
             }
-            ++loads_issued;
-        }
-        // which keys of this tile are highlighted
-        int hl = 0;
-        if (steer) {
-            const int kpos = j * BN + tid;
-            hl = (kpos < Lb && p.mask[seq0 + kpos] != 0) ? 1 : 0;
-            rowflag[tid] = (uint8_t)hl;
-        }
-        const int any_hl = __syncthreads_or(hl);
-
-        ok = mbar_wait(bar_kv + s, (uint32_t)((j >> 1) & 1), abort_flag, p.status, 1);
-        if (tid == 0) ++loads_waited;
-        __syncwarp();
-        if (__all_sync(0xffffffffu, ok) && any_hl) {
-#pragma unroll 1
-            for (int blk = 0; blk < 2; ++blk) {
-                const int r0 = warp * 32 + blk * 16;
-                const uint32_t f4 = *reinterpret_cast<const uint32_t*>(rowflag + r0) | *reinterpret_cast<const uint32_t*>(rowflag + r0 + 4) |
-                                    *reinterpret_cast<const uint32_t*>(rowflag + r0 + 8) | *reinterpret_cast<const uint32_t*>(rowflag + r0 + 12);
-                if (f4 != 0) edit_rows16<D>(sK, BLK_BYTES, r0, rowflag, fragB, fragA, colscale, nR16, lane);
+            bool ok = true;
+            for (int j = 0; j < n_kv && ok; ++j) {
+                const int sk = j % NK, uk = j / NK, sv = j % NV, uv = j / NV;
+                if (uk > 0) ok = mbar_wait(k_empty + sk, (uint32_t)((uk - 1) & 1), abort_flag, p.status, 10);
+                if (!ok) break;
+                mbar_expect_tx(k_full + sk, SL::TILE);
+#pragma unroll
+                for (int c = 0; c < NBLK; ++c)
+                    tma_load_3d(smem + SL::K + sk * SL::TILE + c * BLK_BYTES, &tmK, k_full + sk, c * 64, hkv, seq0 + j * BN);
+                if (uv > 0) ok = mbar_wait(v_empty + sv, (uint32_t)((uv - 1) & 1), abort_flag, p.status, 11);
+                if (!ok) break;
+                mbar_expect_tx(v_full + sv, SL::TILE);
+#pragma unroll
+                for (int c = 0; c < NBLK; ++c)
+                    tma_load_3d(smem + SL::V + sv * SL::TILE + c * BLK_BYTES, &tmV, v_full + sv, c * 64, hkv, seq0 + j * BN);
             }
-            fence_proxy_async();
         }
-        if (!__syncthreads_and(ok ? 1 : 0)) { ok = false; break; }
-
-        // S = Q K'^T
-        if (tid == 0) {
-            if (j == 0) ok = mbar_wait(bar_q, 0, abort_flag, p.status, 2);
-            if (ok) {
-                tc_fence_after();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t IDESC_S = umma_idesc_bf16(BN, false);
+            constexpr uint32_t IDESC_PV = umma_idesc_bf16(D, true);
+            const uint32_t sQa = smem_u32(smem + SL::Q), sKa = smem_u32(smem + SL::K), sVa = smem_u32(smem + SL::V);
+            auto issue_S = [&](int x, int j) {
+                const uint32_t kbase = sKa + (uint32_t)(j % NK) * SL::TILE, qbase = sQa + (uint32_t)x * SL::TILE;
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     const uint32_t off = (uint32_t)(ks >> 2) * BLK_BYTES + (uint32_t)(ks & 3) * 32;
-                    umma_ss(tmem_base, umma_desc_sw128(smem_u32(sQ) + off, 16, 1024),
-                            umma_desc_sw128(smem_u32(sK) + off, 16, 1024), IDESC_S, ks > 0 ? 1u : 0u);
+                    umma_ss(tmem_base + COL_S + 128 * x, umma_desc_sw128(qbase + off, 16, 1024),
+                            umma_desc_sw128(kbase + off, 16, 1024), IDESC_S, ks > 0 ? 1u : 0u);
                 }
-                umma_commit(bar_s);
+                umma_commit(s_full + x);
+            };
+            auto issue_PV = [&](int x, int j) {
+                const uint32_t vbase = sVa + (uint32_t)(j % NV) * SL::TILE;
+#pragma unroll
+                for (int ks = 0; ks < BN / 16; ++ks)
+                    umma_ts(tmem_base + COL_O + D * x, tmem_base + COL_S + 128 * x + (uint32_t)ks * 8,
+                            umma_desc_sw128(vbase + (uint32_t)ks * 2048, BLK_BYTES, 1024), IDESC_PV, (j > 0 || ks > 0) ? 1u : 0u);
+            };
+            bool ok = mbar_wait(q_full + 0, 0, abort_flag, p.status, 20);
+            if (ok && nB > 0) ok = mbar_wait(q_full + 1, 0, abort_flag, p.status, 21);
+            if (ok) ok = mbar_wait(k_ready + 0, 0, abort_flag, p.status, 22);
+            if (ok) {
+                tc_fence_after();
+                issue_S(0, 0);
+                if (nB > 0) issue_S(1, 0);
+                umma_commit(k_empty + 0);
+            }
+            for (int j = 0; j < n_kv && ok; ++j) {
+                const int sv = j % NV, j1 = j + 1, sk1 = j1 % NK;
+                const uint32_t par_k1 = (uint32_t)((j1 / NK) & 1);
+                ok = mbar_wait(v_full + sv, (uint32_t)((j / NV) & 1), abort_flag, p.status, 23);
+                if (!ok) break;
+                if (j < nA) {
+                    ok = mbar_wait(p_full + 0, (uint32_t)(j & 1), abort_flag, p.status, 24);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_PV(0, j);
+                    if (j == nA - 1) umma_commit(o_full + 0);
+                    if (j1 < nA) {
+                        ok = mbar_wait(k_ready + sk1, par_k1, abort_flag, p.status, 25);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_S(0, j1);
+                    }
+                }
+                if (j < nB) {
+                    ok = mbar_wait(p_full + 1, (uint32_t)(j & 1), abort_flag, p.status, 26);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_PV(1, j);
+                    if (j == nB - 1) umma_commit(o_full + 1);
+                }
+                umma_commit(v_empty + sv);
+                if (j1 < nB) {
+                    ok = mbar_wait(k_ready + sk1, par_k1, abort_flag, p.status, 27);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_S(1, j1);
+                }
+                if (j1 < n_kv) umma_commit(k_empty + sk1);
             }
         }
-        ok = mbar_wait(bar_s, (uint32_t)(j & 1), abort_flag, p.status, 3) && ok;
-        __syncwarp();
-        tc_fence_after();
-
-        float corr = 1.f;
-        if (ok) {
-            const bool diag = (j == qt);
+    } else if (warp >= 12) {
+        // ------------------------------------------------------------ key editors (32 rows of every K tile per warp)
+        const int wrow = (warp - 12) * 32;
+        const size_t fr_head = frag_uint4_per_head(D, p.r_pad);
+        const uint4* fragB = p.frags + (size_t)hkv * fr_head;
+        const uint4* fragA = fragB + fr_head / 2;
+        const int nR16 = p.r_pad / 16;
+        for (int j = 0; j < n_kv; ++j) {
+            const int sk = j % NK;
+            uint8_t* flags = rowflag + sk * 128;
+            unsigned hl_mask = 0;
+            if (steer) {
+                const int kpos = j * BN + wrow + lane;
+                const bool hl = kpos < Lb && p.mask[seq0 + kpos] != 0;
+                flags[wrow + lane] = hl ? 1 : 0;
+                hl_mask = __ballot_sync(0xffffffffu, hl);
+            }
+            if (!warp_wait(k_full + sk, (uint32_t)((j / NK) & 1), abort_flag, p.status, 30)) break;
+            if (hl_mask != 0) {
+                __syncwarp();      // the flags written above are read by other lanes of this warp
+                uint8_t* sK = smem + SL::K + sk * SL::TILE;
+                if (hl_mask & 0x0000ffffu) edit_rows16<D>(sK, BLK_BYTES, wrow, flags, fragB, fragA, colscale, nR16, lane);
+                if (hl_mask & 0xffff0000u) edit_rows16<D>(sK, BLK_BYTES, wrow + 16, flags, fragB, fragA, colscale, nR16, lane);
+                fence_proxy_async();
+            }
+            mbar_arrive(k_ready + sk);
+        }
+    } else if (warp >= 4) {
+        // ------------------------------------------------------------ softmax of tile x, one query row per thread
+        const int x = (warp - 4) >> 2;
+        const int nX = x == 0 ? nA : nB;
+        const int row = (warp & 3) * 32 + lane;
+        const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+        const uint32_t tS = t_lane + COL_S + 128 * x, tO = t_lane + COL_O + D * x;
+        float m_run = -INFINITY, l_run = 0.f;
+        bool ok = true;
+        for (int j = 0; j < nX; ++j) {
+            ok = warp_wait(s_full + x, (uint32_t)(j & 1), abort_flag, p.status, 40 + x);
+            if (!ok) break;
+            tc_fence_after();
+            const bool diag = (j == nX - 1);
             uint32_t v[32];
             float mx = -INFINITY;
 #pragma unroll 1
@@ -221,87 +297,77 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                 tmem_wait_ld();
 #pragma unroll
                 for (int e = 0; e < 32; ++e) {
-                    float x = __uint_as_float(v[e]);
-                    if (diag && (c * 32 + e) > row) x = -INFINITY;
-                    mx = fmaxf(mx, x);
+                    float xv = __uint_as_float(v[e]);
+                    if (diag && (c * 32 + e) > row) xv = -INFINITY;
+                    mx = fmaxf(mx, xv);
                 }
             }
             const float m_new = fmaxf(m_run, mx * p.scale_log2);
-            corr = fast_exp2(m_run - m_new);
+            // raise the running maximum only when it moved a lot; p may then exceed 1 (up to 2^8), which is harmless
+            const bool raise = (m_new - m_run) > LAZY_RESCALE_LOG2;      // true on the first tile (m_run = -inf)
+            const float factor = raise ? fast_exp2(m_run - m_new) : 1.f;
+            if (raise) m_run = m_new;
+            if (j > 0 && __any_sync(0xffffffffu, raise)) {
+#pragma unroll 1
+                for (int c = 0; c < D / 32; ++c) {
+                    tmem_ld32(tO + c * 32, v);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * factor);
+                    tmem_st32(tO + c * 32, v);
+                }
+            }
             float psum = 0.f;
 #pragma unroll 1
             for (int c = 0; c < 4; ++c) {
                 tmem_ld32(tS + c * 32, v);
                 tmem_wait_ld();
+                uint32_t pk16[16];
 #pragma unroll
-                for (int e8 = 0; e8 < 4; ++e8) {
-                    float pv[8];
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        const int col = c * 32 + e8 * 8 + e;
-                        float x = fast_exp2(fmaf(__uint_as_float(v[e8 * 8 + e]), p.scale_log2, -m_new));
-                        if (diag && col > row) x = 0.f;
-                        pv[e] = x;
-                        psum += x;
-                    }
-                    const int col0 = c * 32 + e8 * 8;
-                    uint4 pk = make_uint4(pack_bf16(pv[0], pv[1]), pack_bf16(pv[2], pv[3]), pack_bf16(pv[4], pv[5]), pack_bf16(pv[6], pv[7]));
-                    *reinterpret_cast<uint4*>(sP + (uint32_t)(col0 >> 6) * BLK_BYTES + sw128_offset(row, col0 & 63)) = pk;
+                for (int e2 = 0; e2 < 16; ++e2) {
+                    float p0 = fast_exp2(fmaf(__uint_as_float(v[2 * e2]), p.scale_log2, -m_run));
+                    float p1 = fast_exp2(fmaf(__uint_as_float(v[2 * e2 + 1]), p.scale_log2, -m_run));
+                    if (diag && (c * 32 + 2 * e2) > row) p0 = 0.f;
+                    if (diag && (c * 32 + 2 * e2 + 1) > row) p1 = 0.f;
+                    psum += p0 + p1;
+                    pk16[e2] = pack_bf16(p0, p1);
                 }
+                tmem_st16(tS + c * 16, pk16);     // P (bf16 pairs) overwrites score columns already consumed
             }
-            l_run = l_run * corr + psum;
-            m_run = m_new;
-            fence_proxy_async();
+            l_run = l_run * factor + psum;
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(p_full + x);
         }
-        tc_fence_before();
-        if (!__syncthreads_and(ok ? 1 : 0)) { ok = false; break; }
-
-        // PV = P V
-        if (tid == 0) {
+        if (ok && nX > 0) ok = warp_wait(o_full + x, 0, abort_flag, p.status, 44 + x);
+        if (ok && nX > 0) {
             tc_fence_after();
-#pragma unroll
-            for (int ks = 0; ks < BN / 16; ++ks) {
-                const uint32_t offP = (uint32_t)(ks >> 2) * BLK_BYTES + (uint32_t)(ks & 3) * 32;
-                umma_ss(tmem_base + 128, umma_desc_sw128(smem_u32(sP) + offP, 16, 1024),
-                        umma_desc_sw128(smem_u32(sV) + (uint32_t)ks * 2048, BLK_BYTES, 1024), IDESC_PV, ks > 0 ? 1u : 0u);
-            }
-            umma_commit(bar_pv);
-        }
-        ok = mbar_wait(bar_pv, (uint32_t)(j & 1), abort_flag, p.status, 4);
-        __syncwarp();
-        tc_fence_after();
-        if (ok) {
+            const int qpos = (qt2 * 2 + x) * BM + row;
+            const bool valid = qpos < Lb;
+            const size_t orow = (size_t)(seq0 + (valid ? qpos : 0)) * p.Hq + hq;
+            const float inv = 1.f / l_run;
             uint32_t v[32];
-#pragma unroll
+#pragma unroll 1
             for (int c = 0; c < D / 32; ++c) {
-                tmem_ld32(tPV + c * 32, v);
+                tmem_ld32(tO + c * 32, v);
                 tmem_wait_ld();
-#pragma unroll
-                for (int e = 0; e < 32; ++e) o[c * 32 + e] = fmaf(o[c * 32 + e], corr, __uint_as_float(v[e]));
+                if (valid) store_chunk32<OutT>(static_cast<OutT*>(p.O) + orow * D + c * 32, v, inv);
             }
+            if (valid && p.lse != nullptr) p.lse[orow] = (m_run + log2f(l_run)) * 0.6931471805599453f;
         }
-        tc_fence_before();
-        if (!__syncthreads_and(ok ? 1 : 0)) { ok = false; break; }
     }
 
-    if (ok) {
-        const int qpos = qt * BM + row;
-        if (qpos < Lb) {
-            const size_t orow = (size_t)(seq0 + qpos) * p.Hq + hq;
-            store_row<OutT>(static_cast<OutT*>(p.O) + orow * D, o, D, 1.f / l_run);
-            if (p.lse != nullptr) p.lse[orow] = (m_run + log2f(l_run)) * 0.6931471805599453f;
-        }
-    } else if (tid == 0) {
-        // let any tile load still in flight land before the CTA's shared memory is released
-        int dummy = 0;
-        while (loads_waited < loads_issued) {
-            mbar_wait(bar_kv + (loads_waited & 1), (uint32_t)((loads_waited >> 1) & 1), &dummy, nullptr, 0);
-            ++loads_waited;
-        }
-    }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem_base, TMEM_COLS);
+    if (warp == 0) {
+        if (*abort_flag && lane == 0) {
+            // let tile loads that may still be in flight land before the shared memory is released
+            int dummy = 0;
+            for (int i = 0; i < NK; ++i) { mbar_wait(k_full + i, 0, &dummy, nullptr, 0); }
+        }
+        __syncwarp();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
 }
 
 // ---------------------------------------------------------------- host side
@@ -344,8 +410,8 @@ static seka_status launch_attn(const CUtensorMap& tq, const CUtensorMap& tk, con
                                  (int)SL::DYN_BYTES) != cudaSuccess) return SEKA_ERR_CUDA;
         configured = true;
     }
-    const unsigned grid = (unsigned)p.n_qt * p.B * p.Hq;
-    seka_attn_fwd_kernel<D, OutT><<<grid, 128, SL::DYN_BYTES, st>>>(tq, tk, tv, p);
+    const unsigned grid = (unsigned)((p.n_qt + 1) / 2) * p.B * p.Hq;
+    seka_attn_fwd_kernel<D, OutT><<<grid, NTHREADS, SL::DYN_BYTES, st>>>(tq, tk, tv, p);
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? SEKA_OK : SEKA_ERR_CUDA;
 }

@@ -47,44 +47,52 @@ __device__ __forceinline__ void edit_rows16(uint8_t* tile, uint32_t blk_stride, 
     const int g = lane >> 2, t = lane & 3;
     const uint32_t tile_s = smem_u32(tile);
 
-    float acc[8][2][4];
-#pragma unroll
-    for (int np = 0; np < 8; ++np)
-#pragma unroll
-        for (int q = 0; q < 2; ++q)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) acc[np][q][e] = 0.f;
-
-    // T = K_block * Ustack
+    // T = K_block * Ustack, 64 stacked columns at a time; the columns are scaled by gain * alpha and the
+    // accumulators repacked as the A operand of the next product
+    uint32_t ta[8][4];
     const int lrow = r0 + (lane & 7) + ((lane >> 3) & 1) * 8;
 #pragma unroll
-    for (int kb = 0; kb < KB; ++kb) {
-        const int col = kb * 16 + (lane >> 4) * 8;
-        uint32_t a[4];
-        ldmatrix_x4(a, tile_s + (uint32_t)(col >> 6) * blk_stride + sw128_offset(lrow, col & 63));
+    for (int half = 0; half < 2; ++half) {
+        if (half * 4 < nR16) {
+            float acc[4][2][4];
 #pragma unroll
-        for (int np = 0; np < 8; ++np) {
-            if (np < nR16) {
-                const uint4 f = __ldg(fragB + ((size_t)kb * nR16 + np) * 32 + lane);
-                mma_bf16_16816(acc[np][0], a, f.x, f.y);
-                mma_bf16_16816(acc[np][1], a, f.z, f.w);
+            for (int n4 = 0; n4 < 4; ++n4)
+#pragma unroll
+                for (int q = 0; q < 2; ++q)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) acc[n4][q][e] = 0.f;
+#pragma unroll
+            for (int kb = 0; kb < KB; ++kb) {
+                const int col = kb * 16 + (lane >> 4) * 8;
+                uint32_t a[4];
+                ldmatrix_x4(a, tile_s + (uint32_t)(col >> 6) * blk_stride + sw128_offset(lrow, col & 63));
+#pragma unroll
+                for (int n4 = 0; n4 < 4; ++n4) {
+                    const int np = half * 4 + n4;
+                    if (np < nR16) {
+                        const uint4 f = __ldg(fragB + ((size_t)kb * nR16 + np) * 32 + lane);
+                        mma_bf16_16816(acc[n4][0], a, f.x, f.y);
+                        mma_bf16_16816(acc[n4][1], a, f.z, f.w);
+                    }
+                }
             }
-        }
-    }
-
-    // scale the columns by gain * alpha and repack the accumulators as the next product's A operand
-    uint32_t ta[8][4];
 #pragma unroll
-    for (int np = 0; np < 8; ++np) {
-        if (np < nR16) {
-            const float2 s0 = *reinterpret_cast<const float2*>(colscale + np * 16 + 2 * t);
-            const float2 s1 = *reinterpret_cast<const float2*>(colscale + np * 16 + 8 + 2 * t);
-            ta[np][0] = pack_bf16(acc[np][0][0] * s0.x, acc[np][0][1] * s0.y);
-            ta[np][1] = pack_bf16(acc[np][0][2] * s0.x, acc[np][0][3] * s0.y);
-            ta[np][2] = pack_bf16(acc[np][1][0] * s1.x, acc[np][1][1] * s1.y);
-            ta[np][3] = pack_bf16(acc[np][1][2] * s1.x, acc[np][1][3] * s1.y);
+            for (int n4 = 0; n4 < 4; ++n4) {
+                const int np = half * 4 + n4;
+                if (np < nR16) {
+                    const float2 s0 = *reinterpret_cast<const float2*>(colscale + np * 16 + 2 * t);
+                    const float2 s1 = *reinterpret_cast<const float2*>(colscale + np * 16 + 8 + 2 * t);
+                    ta[np][0] = pack_bf16(acc[n4][0][0] * s0.x, acc[n4][0][1] * s0.y);
+                    ta[np][1] = pack_bf16(acc[n4][0][2] * s0.x, acc[n4][0][3] * s0.y);
+                    ta[np][2] = pack_bf16(acc[n4][1][0] * s1.x, acc[n4][1][1] * s1.y);
+                    ta[np][3] = pack_bf16(acc[n4][1][2] * s1.x, acc[n4][1][3] * s1.y);
+                } else {
+                    ta[np][0] = ta[np][1] = ta[np][2] = ta[np][3] = 0u;
+                }
+            }
         } else {
-            ta[np][0] = ta[np][1] = ta[np][2] = ta[np][3] = 0u;
+#pragma unroll
+            for (int n4 = 0; n4 < 4; ++n4) ta[half * 4 + n4][0] = ta[half * 4 + n4][1] = ta[half * 4 + n4][2] = ta[half * 4 + n4][3] = 0u;
         }
     }
 
