@@ -21,6 +21,10 @@
 #include "seka_edit_tile.cuh"
 #include "seka_kernels.h"
 
+#ifndef SEKA_POLY_PAIR_MASK
+#define SEKA_POLY_PAIR_MASK 0x0000u
+#endif
+
 namespace seka {
 
 struct AttnParams {
@@ -35,6 +39,7 @@ struct AttnParams {
     int* status;
     int B, L, Hq, Hkv, rank, M, r_pad, n_qt;
     int steer;
+    int pair_heads;       // 1: the two tiles of a CTA are two query heads of one KV group; 0: two consecutive query tiles
     float scale_log2;
 };
 
@@ -43,6 +48,10 @@ constexpr int NK = 3, NV = 2;               // K and V ring depths
 constexpr int NTHREADS = 512;
 constexpr uint32_t BLK_BYTES = 128 * 128;   // one [128 x 64] bf16 block
 constexpr float LAZY_RESCALE_LOG2 = 8.0f;   // the running maximum is only raised when it moved by more than this
+// registers per thread after the roles split (the CTA owns the whole register file: 4 x 128 x (48+184+184+96) = 64 Ki)
+constexpr int REGS_CTRL = 48, REGS_SOFTMAX = 184, REGS_EDIT = 96;
+// which of the 16 element pairs of every 32-key chunk take the polynomial exp2 instead of the special-function unit
+constexpr uint32_t POLY_PAIR_MASK = SEKA_POLY_PAIR_MASK;
 
 template <int D>
 struct SmemLayout {
@@ -59,10 +68,42 @@ struct SmemLayout {
     static constexpr uint32_t DYN_BYTES = TOTAL + 1024;    // slack for the 1024-byte alignment
 };
 
+// One 128-row query tile of a CTA: query head, tile index within the sequence, number of key tiles it attends
+// to (the last of them is the diagonal tile); n == 0 means the tile lies beyond the sequence.
+struct TileWork { int hq, qt, n; };
+
 // all lanes of a warp wait on the same barrier and then agree on the outcome
 __device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status, int where) {
     const bool ok = mbar_wait(bar, parity, abort_flag, status, where);
     return __all_sync(0xffffffffu, ok);
+}
+
+template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
+// 2^x for a pair of arguments on the FMA pipe: x = n + f with n = round(x), f in [-1/2, 1/2];
+// 2^f by a cubic fitted to relative error 7.5e-5 (far below the bf16 rounding of P), 2^n by adding n
+// to the exponent field.  Arguments below -126 (masked scores) give a value below 2^-125.
+__device__ __forceinline__ float2 exp2_poly2(float2 x) {
+    const float kMagic = 12582912.f;      // 1.5 * 2^23: adding it rounds to an integer in the low mantissa bits
+    x.x = fmaxf(x.x, -126.f);
+    x.y = fmaxf(x.y, -126.f);
+    const float2 t = __fadd2_rn(x, make_float2(kMagic, kMagic));
+    const float2 n = __fadd2_rn(t, make_float2(-kMagic, -kMagic));
+    const float2 f = __ffma2_rn(n, make_float2(-1.f, -1.f), x);
+    float2 q = __ffma2_rn(f, make_float2(0.05517167f, 0.05517167f), make_float2(0.24261113f, 0.24261113f));
+    q = __ffma2_rn(q, f, make_float2(0.69326097f, 0.69326097f));
+    q = __ffma2_rn(q, f, make_float2(0.99992806f, 0.99992806f));
+    float2 r;
+    r.x = __int_as_float(__float_as_int(q.x) + (__float_as_int(t.x) << 23));
+    r.y = __int_as_float(__float_as_int(q.y) + (__float_as_int(t.y) << 23));
+    return r;
 }
 
 template <typename OutT> __device__ __forceinline__ void store_chunk32(OutT* dst, const uint32_t (&v)[32], float inv);
@@ -110,21 +151,33 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-    // heaviest query tiles first; CTAs of one (sequence, KV head) are neighbours
-    const int per_qt = p.B * p.Hq;
-    const int n_qt2 = (p.n_qt + 1) >> 1;
-    const int qt2 = n_qt2 - 1 - (int)(blockIdx.x / per_qt);
-    const int rem = (int)(blockIdx.x % per_qt);
-    const int b = rem / p.Hq, hq = rem % p.Hq;
-    const int hkv = hq / (p.Hq / p.Hkv);
+    // work of this CTA: heaviest query tiles first; CTAs of one (sequence, KV head) are neighbours
+    TileWork tw[2];
+    int b;
+    if (p.pair_heads) {
+        const int per_qt = p.B * (p.Hq >> 1);
+        const int qt = p.n_qt - 1 - (int)(blockIdx.x / per_qt);
+        const int rem = (int)(blockIdx.x % per_qt);
+        b = rem / (p.Hq >> 1);
+        const int hp = rem % (p.Hq >> 1);
+        tw[0].hq = 2 * hp; tw[1].hq = 2 * hp + 1;
+        tw[0].qt = tw[1].qt = qt;
+    } else {
+        const int per_qt = p.B * p.Hq;
+        const int qt2 = ((p.n_qt + 1) >> 1) - 1 - (int)(blockIdx.x / per_qt);
+        const int rem = (int)(blockIdx.x % per_qt);
+        b = rem / p.Hq;
+        tw[0].hq = tw[1].hq = rem % p.Hq;
+        tw[0].qt = 2 * qt2; tw[1].qt = 2 * qt2 + 1;
+    }
+    const int hkv = tw[0].hq / (p.Hq / p.Hkv);
     const int seq0 = p.cu_seqlens ? p.cu_seqlens[b] : b * p.L;
     const int Lb = p.cu_seqlens ? (p.cu_seqlens[b + 1] - seq0) : p.L;
-    if (qt2 * 2 * BM >= Lb) return;                                    // nothing allocated yet
+    tw[0].n = tw[0].qt * BM < Lb ? tw[0].qt + 1 : 0;
+    tw[1].n = tw[1].qt * BM < Lb ? tw[1].qt + 1 : 0;
+    const int nA = tw[0].n, nB = tw[1].n;
+    if (nA == 0) return;                                               // nothing allocated yet (tile B starts no earlier)
     if (*reinterpret_cast<volatile int*>(p.status) != 0) return;      // an earlier CTA gave up: do not pile on
-
-    const int ntiles = (Lb + BN - 1) / BN;
-    const int nA = min(2 * qt2 + 1, ntiles);                           // key tiles of query tile A (last one diagonal)
-    const int nB = ((2 * qt2 + 1) * BM < Lb) ? min(2 * qt2 + 2, ntiles) : 0;   // 0: tile B lies beyond the sequence
     const int n_kv = max(nA, nB);
 
     if (tid == 0) {
@@ -152,17 +205,19 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     tc_fence_after();
     const uint32_t tmem_base = *tmem_holder;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
-        if (lane == 0) {
+    if (warp < 4) {
+        reg_dec<REGS_CTRL>();
+        if (warp == 0 && lane == 0) {
+            // ------------------------------------------------------------ TMA producer
             mbar_expect_tx(q_full + 0, SL::TILE);
 #pragma unroll
-            for (int c = 0; c < NBLK; ++c) tma_load_3d(smem + SL::Q + c * BLK_BYTES, &tmQ, q_full + 0, c * 64, hq, seq0 + qt2 * 2 * BM);
+            for (int c = 0; c < NBLK; ++c)
+                tma_load_3d(smem + SL::Q + c * BLK_BYTES, &tmQ, q_full + 0, c * 64, tw[0].hq, seq0 + tw[0].qt * BM);
             if (nB > 0) {
                 mbar_expect_tx(q_full + 1, SL::TILE);
 #pragma unroll
                 for (int c = 0; c < NBLK; ++c)
-                    tma_load_3d(smem + SL::Q + SL::TILE + c * BLK_BYTES, &tmQ, q_full + 1, c * 64, hq, seq0 + (qt2 * 2 + 1) * BM);
+                    tma_load_3d(smem + SL::Q + SL::TILE + c * BLK_BYTES, &tmQ, q_full + 1, c * 64, tw[1].hq, seq0 + tw[1].qt * BM);
             }
             bool ok = true;
             for (int j = 0; j < n_kv && ok; ++j) {
@@ -180,10 +235,8 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                 for (int c = 0; c < NBLK; ++c)
                     tma_load_3d(smem + SL::V + sv * SL::TILE + c * BLK_BYTES, &tmV, v_full + sv, c * 64, hkv, seq0 + j * BN);
             }
-        }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        } else if (warp == 1 && lane == 0) {
+            // ------------------------------------------------------------ MMA issuer
             constexpr uint32_t IDESC_S = umma_idesc_bf16(BN, false);
             constexpr uint32_t IDESC_PV = umma_idesc_bf16(D, true);
             const uint32_t sQa = smem_u32(smem + SL::Q), sKa = smem_u32(smem + SL::K), sVa = smem_u32(smem + SL::V);
@@ -250,6 +303,7 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         }
     } else if (warp >= 12) {
         // ------------------------------------------------------------ key editors (32 rows of every K tile per warp)
+        reg_dec<REGS_EDIT>();
         const int wrow = (warp - 12) * 32;
         const size_t fr_head = frag_uint4_per_head(D, p.r_pad);
         const uint4* fragB = p.frags + (size_t)hkv * fr_head;
@@ -269,72 +323,84 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             if (hl_mask != 0) {
                 __syncwarp();      // the flags written above are read by other lanes of this warp
                 uint8_t* sK = smem + SL::K + sk * SL::TILE;
-                if (hl_mask & 0x0000ffffu) edit_rows16<D>(sK, BLK_BYTES, wrow, flags, fragB, fragA, colscale, nR16, lane);
-                if (hl_mask & 0xffff0000u) edit_rows16<D>(sK, BLK_BYTES, wrow + 16, flags, fragB, fragA, colscale, nR16, lane);
+                if (hl_mask & 0x0000ffffu) edit_rows16_any<D>(sK, BLK_BYTES, wrow, flags, fragB, fragA, colscale, nR16, lane);
+                if (hl_mask & 0xffff0000u) edit_rows16_any<D>(sK, BLK_BYTES, wrow + 16, flags, fragB, fragA, colscale, nR16, lane);
                 fence_proxy_async();
             }
             mbar_arrive(k_ready + sk);
         }
-    } else if (warp >= 4) {
+    } else {
         // ------------------------------------------------------------ softmax of tile x, one query row per thread
+        reg_inc<REGS_SOFTMAX>();
         const int x = (warp - 4) >> 2;
-        const int nX = x == 0 ? nA : nB;
+        const int nX = x ? nB : nA;
+        const int hqX = x ? tw[1].hq : tw[0].hq, qtX = x ? tw[1].qt : tw[0].qt;
         const int row = (warp & 3) * 32 + lane;
         const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
         const uint32_t tS = t_lane + COL_S + 128 * x, tO = t_lane + COL_O + D * x;
+        const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
         float m_run = -INFINITY, l_run = 0.f;
         bool ok = true;
         for (int j = 0; j < nX; ++j) {
             ok = warp_wait(s_full + x, (uint32_t)(j & 1), abort_flag, p.status, 40 + x);
             if (!ok) break;
             tc_fence_after();
-            const bool diag = (j == nX - 1);
-            uint32_t v[32];
-            float mx = -INFINITY;
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                tmem_ld32(tS + c * 32, v);
-                tmem_wait_ld();
+            // the whole score row of this thread: 128 fp32 values in registers
+            uint32_t v[128];
 #pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    float xv = __uint_as_float(v[e]);
-                    if (diag && (c * 32 + e) > row) xv = -INFINITY;
-                    mx = fmaxf(mx, xv);
-                }
+            for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, reinterpret_cast<uint32_t(&)[32]>(v[32 * c]));
+            tmem_wait_ld();
+            if (j == nX - 1) {       // diagonal tile: keys after the query are masked
+#pragma unroll
+                for (int e = 0; e < 128; ++e)
+                    if (e > row) v[e] = 0xff800000u;
             }
-            const float m_new = fmaxf(m_run, mx * p.scale_log2);
+            float mx[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                mx[q] = fmaxf(__uint_as_float(v[32 * q]), __uint_as_float(v[32 * q + 1]));
+#pragma unroll
+                for (int e = 2; e < 32; e += 2) mx[q] = max3(mx[q], __uint_as_float(v[32 * q + e]), __uint_as_float(v[32 * q + e + 1]));
+            }
+            const float m_new = fmaxf(m_run, fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale_log2);
             // raise the running maximum only when it moved a lot; p may then exceed 1 (up to 2^8), which is harmless
             const bool raise = (m_new - m_run) > LAZY_RESCALE_LOG2;      // true on the first tile (m_run = -inf)
             const float factor = raise ? fast_exp2(m_run - m_new) : 1.f;
             if (raise) m_run = m_new;
             if (j > 0 && __any_sync(0xffffffffu, raise)) {
+                uint32_t o[32];
 #pragma unroll 1
                 for (int c = 0; c < D / 32; ++c) {
-                    tmem_ld32(tO + c * 32, v);
+                    tmem_ld32(tO + c * 32, o);
                     tmem_wait_ld();
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * factor);
-                    tmem_st32(tO + c * 32, v);
+                    for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * factor);
+                    tmem_st32(tO + c * 32, o);
                 }
             }
-            float psum = 0.f;
-#pragma unroll 1
+            const float2 nm2 = make_float2(-m_run, -m_run);
+            float2 sum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+#pragma unroll
             for (int c = 0; c < 4; ++c) {
-                tmem_ld32(tS + c * 32, v);
-                tmem_wait_ld();
                 uint32_t pk16[16];
 #pragma unroll
                 for (int e2 = 0; e2 < 16; ++e2) {
-                    float p0 = fast_exp2(fmaf(__uint_as_float(v[2 * e2]), p.scale_log2, -m_run));
-                    float p1 = fast_exp2(fmaf(__uint_as_float(v[2 * e2 + 1]), p.scale_log2, -m_run));
-                    if (diag && (c * 32 + 2 * e2) > row) p0 = 0.f;
-                    if (diag && (c * 32 + 2 * e2 + 1) > row) p1 = 0.f;
-                    psum += p0 + p1;
-                    pk16[e2] = pack_bf16(p0, p1);
+                    const int e = 32 * c + 2 * e2;
+                    const float2 arg = __ffma2_rn(make_float2(__uint_as_float(v[e]), __uint_as_float(v[e + 1])), sc2, nm2);
+                    float2 pe;
+                    if ((POLY_PAIR_MASK >> e2) & 1u) {
+                        pe = exp2_poly2(arg);
+                    } else {
+                        pe.x = fast_exp2(arg.x);
+                        pe.y = fast_exp2(arg.y);
+                    }
+                    sum[e2 & 1] = __fadd2_rn(sum[e2 & 1], pe);
+                    pk16[e2] = pack_bf16(pe.x, pe.y);
                 }
-                tmem_st16(tS + c * 16, pk16);     // P (bf16 pairs) overwrites score columns already consumed
+                tmem_st16(tS + c * 16, pk16);     // P (bf16 pairs) over score columns that are already in registers
             }
-            l_run = l_run * factor + psum;
+            const float2 s2 = __fadd2_rn(sum[0], sum[1]);
+            l_run = l_run * factor + (s2.x + s2.y);
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(p_full + x);
@@ -342,16 +408,16 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         if (ok && nX > 0) ok = warp_wait(o_full + x, 0, abort_flag, p.status, 44 + x);
         if (ok && nX > 0) {
             tc_fence_after();
-            const int qpos = (qt2 * 2 + x) * BM + row;
+            const int qpos = qtX * BM + row;
             const bool valid = qpos < Lb;
-            const size_t orow = (size_t)(seq0 + (valid ? qpos : 0)) * p.Hq + hq;
+            const size_t orow = (size_t)(seq0 + (valid ? qpos : 0)) * p.Hq + hqX;
             const float inv = 1.f / l_run;
-            uint32_t v[32];
+            uint32_t o[32];
 #pragma unroll 1
             for (int c = 0; c < D / 32; ++c) {
-                tmem_ld32(tO + c * 32, v);
+                tmem_ld32(tO + c * 32, o);
                 tmem_wait_ld();
-                if (valid) store_chunk32<OutT>(static_cast<OutT*>(p.O) + orow * D + c * 32, v, inv);
+                if (valid) store_chunk32<OutT>(static_cast<OutT*>(p.O) + orow * D + c * 32, o, inv);
             }
             if (valid && p.lse != nullptr) p.lse[orow] = (m_run + log2f(l_run)) * 0.6931471805599453f;
         }
@@ -410,7 +476,7 @@ static seka_status launch_attn(const CUtensorMap& tq, const CUtensorMap& tk, con
                                  (int)SL::DYN_BYTES) != cudaSuccess) return SEKA_ERR_CUDA;
         configured = true;
     }
-    const unsigned grid = (unsigned)((p.n_qt + 1) / 2) * p.B * p.Hq;
+    const unsigned grid = p.pair_heads ? (unsigned)p.n_qt * p.B * (p.Hq / 2) : (unsigned)((p.n_qt + 1) / 2) * p.B * p.Hq;
     seka_attn_fwd_kernel<D, OutT><<<grid, NTHREADS, SL::DYN_BYTES, st>>>(tq, tk, tv, p);
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? SEKA_OK : SEKA_ERR_CUDA;
@@ -460,6 +526,7 @@ extern "C" seka_status seka_attention_fwd(const seka_shape* shape, const void* Q
     p.cu_seqlens = shape->cu_seqlens; p.frags = frags; p.status = reinterpret_cast<int*>(ws);
     p.B = shape->batch; p.L = shape->max_seqlen; p.Hq = Hq; p.Hkv = Hkv; p.rank = shape->rank; p.M = shape->n_experts;
     p.r_pad = w.r_pad; p.n_qt = (shape->max_seqlen + BM - 1) / BM; p.steer = steer ? 1 : 0;
+    p.pair_heads = ((Hq / Hkv) % 2 == 0) ? 1 : 0;
     const float scale = shape->softmax_scale > 0.f ? shape->softmax_scale : 1.f / sqrtf((float)D);
     p.scale_log2 = scale * 1.4426950408889634f;
 

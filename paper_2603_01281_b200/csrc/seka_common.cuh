@@ -24,7 +24,7 @@ struct WorkspaceLayout {
     size_t list_off, list_bytes;      // int32 [total_tokens]
     size_t cvt_off, cvt_bytes;        // bf16 copies of Q, K, V (fp32 inputs only)
     size_t total;
-    int r_pad;                        // M * r rounded up to 16
+    int r_pad;                        // M * r rounded up to 16, 32, 64 or 128
 };
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -36,7 +36,8 @@ static inline int shape_total_tokens(const seka_shape* s) {
 static inline WorkspaceLayout workspace_layout(const seka_shape* s) {
     WorkspaceLayout w;
     const size_t T = (size_t)shape_total_tokens(s);
-    w.r_pad = (s->n_experts * s->rank + 15) / 16 * 16;
+    w.r_pad = 16;
+    while (w.r_pad < s->n_experts * s->rank) w.r_pad *= 2;
     w.frag_off = kStatusBytes;
     w.frag_bytes = align_up((size_t)s->n_kv_heads * 2 * (size_t)s->head_dim * w.r_pad * 2, 256);
     w.list_off = w.frag_off + w.frag_bytes;

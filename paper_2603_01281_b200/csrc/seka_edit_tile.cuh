@@ -39,60 +39,58 @@ __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t smem_addr
 __host__ __device__ inline size_t frag_uint4_per_head(int D, int r_pad) { return (size_t)2 * (D / 16) * (r_pad / 16) * 32; }
 
 // Edits one block of 16 rows (rows r0 .. r0+15 of the tile); called by a whole warp.
-template <int D>
+// NR16 = stacked rank / 16 (1, 2, 4 or 8: the stacked rank is padded to a power of two with zero columns).
+template <int D, int NR16>
 __device__ __forceinline__ void edit_rows16(uint8_t* tile, uint32_t blk_stride, int r0, const uint8_t* rowflag,
                                             const uint4* __restrict__ fragB, const uint4* __restrict__ fragA,
-                                            const float* colscale, int nR16, int lane) {
+                                            const float* colscale, int lane) {
     constexpr int KB = D / 16;
+    constexpr int nR16 = NR16;
     const int g = lane >> 2, t = lane & 3;
     const uint32_t tile_s = smem_u32(tile);
 
-    // T = K_block * Ustack, 64 stacked columns at a time; the columns are scaled by gain * alpha and the
+    // T = K_block * Ustack, 32 stacked columns at a time (keeps the accumulators small: this routine runs in
+    // warps that gave most of their registers away); the columns are scaled by gain * alpha and the
     // accumulators repacked as the A operand of the next product
-    uint32_t ta[8][4];
+    uint32_t ta[NR16][4];
     const int lrow = r0 + (lane & 7) + ((lane >> 3) & 1) * 8;
 #pragma unroll
-    for (int half = 0; half < 2; ++half) {
-        if (half * 4 < nR16) {
-            float acc[4][2][4];
+    for (int np0 = 0; np0 < NR16; np0 += 2) {
+        {
+            float acc[2][2][4];
 #pragma unroll
-            for (int n4 = 0; n4 < 4; ++n4)
+            for (int n2 = 0; n2 < 2; ++n2)
 #pragma unroll
                 for (int q = 0; q < 2; ++q)
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) acc[n4][q][e] = 0.f;
+                    for (int e = 0; e < 4; ++e) acc[n2][q][e] = 0.f;
 #pragma unroll
             for (int kb = 0; kb < KB; ++kb) {
                 const int col = kb * 16 + (lane >> 4) * 8;
                 uint32_t a[4];
                 ldmatrix_x4(a, tile_s + (uint32_t)(col >> 6) * blk_stride + sw128_offset(lrow, col & 63));
 #pragma unroll
-                for (int n4 = 0; n4 < 4; ++n4) {
-                    const int np = half * 4 + n4;
+                for (int n2 = 0; n2 < 2; ++n2) {
+                    const int np = np0 + n2;
                     if (np < nR16) {
                         const uint4 f = __ldg(fragB + ((size_t)kb * nR16 + np) * 32 + lane);
-                        mma_bf16_16816(acc[n4][0], a, f.x, f.y);
-                        mma_bf16_16816(acc[n4][1], a, f.z, f.w);
+                        mma_bf16_16816(acc[n2][0], a, f.x, f.y);
+                        mma_bf16_16816(acc[n2][1], a, f.z, f.w);
                     }
                 }
             }
 #pragma unroll
-            for (int n4 = 0; n4 < 4; ++n4) {
-                const int np = half * 4 + n4;
+            for (int n2 = 0; n2 < 2; ++n2) {
+                const int np = np0 + n2;
                 if (np < nR16) {
                     const float2 s0 = *reinterpret_cast<const float2*>(colscale + np * 16 + 2 * t);
                     const float2 s1 = *reinterpret_cast<const float2*>(colscale + np * 16 + 8 + 2 * t);
-                    ta[np][0] = pack_bf16(acc[n4][0][0] * s0.x, acc[n4][0][1] * s0.y);
-                    ta[np][1] = pack_bf16(acc[n4][0][2] * s0.x, acc[n4][0][3] * s0.y);
-                    ta[np][2] = pack_bf16(acc[n4][1][0] * s1.x, acc[n4][1][1] * s1.y);
-                    ta[np][3] = pack_bf16(acc[n4][1][2] * s1.x, acc[n4][1][3] * s1.y);
-                } else {
-                    ta[np][0] = ta[np][1] = ta[np][2] = ta[np][3] = 0u;
+                    ta[np][0] = pack_bf16(acc[n2][0][0] * s0.x, acc[n2][0][1] * s0.y);
+                    ta[np][1] = pack_bf16(acc[n2][0][2] * s0.x, acc[n2][0][3] * s0.y);
+                    ta[np][2] = pack_bf16(acc[n2][1][0] * s1.x, acc[n2][1][1] * s1.y);
+                    ta[np][3] = pack_bf16(acc[n2][1][2] * s1.x, acc[n2][1][3] * s1.y);
                 }
             }
-        } else {
-#pragma unroll
-            for (int n4 = 0; n4 < 4; ++n4) ta[half * 4 + n4][0] = ta[half * 4 + n4][1] = ta[half * 4 + n4][2] = ta[half * 4 + n4][3] = 0u;
         }
     }
 
@@ -107,12 +105,10 @@ __device__ __forceinline__ void edit_rows16(uint8_t* tile, uint32_t blk_stride, 
 #pragma unroll
             for (int e = 0; e < 4; ++e) c[q][e] = 0.f;
 #pragma unroll
-        for (int kb2 = 0; kb2 < 8; ++kb2) {
-            if (kb2 < nR16) {
-                const uint4 f = __ldg(fragA + ((size_t)kb2 * KB + np2) * 32 + lane);
-                mma_bf16_16816(c[0], ta[kb2], f.x, f.y);
-                mma_bf16_16816(c[1], ta[kb2], f.z, f.w);
-            }
+        for (int kb2 = 0; kb2 < NR16; ++kb2) {
+            const uint4 f = __ldg(fragA + ((size_t)kb2 * KB + np2) * 32 + lane);
+            mma_bf16_16816(c[0], ta[kb2], f.x, f.y);
+            mma_bf16_16816(c[1], ta[kb2], f.z, f.w);
         }
 #pragma unroll
         for (int q = 0; q < 2; ++q) {
@@ -129,6 +125,19 @@ __device__ __forceinline__ void edit_rows16(uint8_t* tile, uint32_t blk_stride, 
                 *p = __floats2bfloat162_rn(k.x + c[q][2], k.y + c[q][3]);
             }
         }
+    }
+}
+
+// Run-time dispatch on the padded stacked rank.
+template <int D>
+__device__ __forceinline__ void edit_rows16_any(uint8_t* tile, uint32_t blk_stride, int r0, const uint8_t* rowflag,
+                                                const uint4* __restrict__ fragB, const uint4* __restrict__ fragA,
+                                                const float* colscale, int nR16, int lane) {
+    switch (nR16) {
+        case 1: edit_rows16<D, 1>(tile, blk_stride, r0, rowflag, fragB, fragA, colscale, lane); break;
+        case 2: edit_rows16<D, 2>(tile, blk_stride, r0, rowflag, fragB, fragA, colscale, lane); break;
+        case 4: edit_rows16<D, 4>(tile, blk_stride, r0, rowflag, fragB, fragA, colscale, lane); break;
+        default: edit_rows16<D, 8>(tile, blk_stride, r0, rowflag, fragB, fragA, colscale, lane); break;
     }
 }
 
