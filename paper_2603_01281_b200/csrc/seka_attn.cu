@@ -62,7 +62,7 @@ struct SmemLayout {
     static constexpr uint32_t ROWFLAG = V + NV * TILE;     // NK x 128 bytes
     static constexpr uint32_t COLSCALE = ROWFLAG + NK * 128;   // 128 floats
     static constexpr uint32_t BARS = COLSCALE + 512;       // mbarriers
-    static constexpr uint32_t NBARS = 2 + 3 * NK + 2 * NV + 6;
+    static constexpr uint32_t NBARS = 2 + 3 * NK + 2 * NV + 8;
     static constexpr uint32_t MISC = BARS + NBARS * 8;     // tmem holder, abort flag
     static constexpr uint32_t TOTAL = MISC + 16;
     static constexpr uint32_t DYN_BYTES = TOTAL + 1024;    // slack for the 1024-byte alignment
@@ -76,6 +76,13 @@ struct TileWork { int hq, qt, n; };
 __device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status, int where) {
     const bool ok = mbar_wait(bar, parity, abort_flag, status, where);
     return __all_sync(0xffffffffu, ok);
+}
+
+// true in exactly one lane of a fully active warp
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+    return pred != 0;
 }
 
 template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
@@ -139,13 +146,14 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SL::BARS);
     uint64_t* q_full = bars;                 // [2]   TMA bytes landed
     uint64_t* k_full = q_full + 2;           // [NK]  TMA bytes landed
-    uint64_t* k_ready = k_full + NK;         // [NK]  128 editor arrivals: tile may be multiplied
+    uint64_t* k_ready = k_full + NK;         // [NK]  4 editor-warp arrivals: tile may be multiplied
     uint64_t* k_empty = k_ready + NK;        // [NK]  tensor core finished reading the stage
     uint64_t* v_full = k_empty + NK;         // [NV]
     uint64_t* v_empty = v_full + NV;         // [NV]
     uint64_t* s_full = v_empty + NV;         // [2]   scores of tile x are in tensor memory
-    uint64_t* p_full = s_full + 2;           // [2]   128 softmax arrivals: P_x written, O_x rescaled
-    uint64_t* o_full = p_full + 2;           // [2]   last P V of tile x finished
+    uint64_t* p_full = s_full + 2;           // [2]   4 softmax-warp arrivals: O_x rescaled, keys 0-95 of P_x written
+    uint64_t* p_last = p_full + 2;           // [2]   4 softmax-warp arrivals: keys 96-127 of P_x written
+    uint64_t* o_full = p_last + 2;           // [2]   last P V of tile x finished
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + SL::MISC);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + SL::MISC + 4);
 
@@ -182,9 +190,9 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 
     if (tid == 0) {
         mbar_init(q_full + 0, 1); mbar_init(q_full + 1, 1);
-        for (int i = 0; i < NK; ++i) { mbar_init(k_full + i, 1); mbar_init(k_ready + i, 128); mbar_init(k_empty + i, 1); }
+        for (int i = 0; i < NK; ++i) { mbar_init(k_full + i, 1); mbar_init(k_ready + i, 4); mbar_init(k_empty + i, 1); }
         for (int i = 0; i < NV; ++i) { mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(s_full + i, 1); mbar_init(p_full + i, 128); mbar_init(o_full + i, 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(s_full + i, 1); mbar_init(p_full + i, 4); mbar_init(p_last + i, 4); mbar_init(o_full + i, 1); }
         *abort_flag = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
@@ -207,98 +215,121 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 
     if (warp < 4) {
         reg_dec<REGS_CTRL>();
-        if (warp == 0 && lane == 0) {
+        // Both control warps run their loops with all 32 lanes and elect one lane only around the issuing
+        // instructions: addresses, descriptors and barrier phases then stay warp-uniform values.
+        const bool leader = elect_one();
+        if (warp == 0) {
             // ------------------------------------------------------------ TMA producer
-            mbar_expect_tx(q_full + 0, SL::TILE);
-#pragma unroll
-            for (int c = 0; c < NBLK; ++c)
-                tma_load_3d(smem + SL::Q + c * BLK_BYTES, &tmQ, q_full + 0, c * 64, tw[0].hq, seq0 + tw[0].qt * BM);
-            if (nB > 0) {
-                mbar_expect_tx(q_full + 1, SL::TILE);
+            if (leader) {
+                mbar_expect_tx(q_full + 0, SL::TILE);
 #pragma unroll
                 for (int c = 0; c < NBLK; ++c)
-                    tma_load_3d(smem + SL::Q + SL::TILE + c * BLK_BYTES, &tmQ, q_full + 1, c * 64, tw[1].hq, seq0 + tw[1].qt * BM);
+                    tma_load_3d(smem + SL::Q + c * BLK_BYTES, &tmQ, q_full + 0, c * 64, tw[0].hq, seq0 + tw[0].qt * BM);
+                if (nB > 0) {
+                    mbar_expect_tx(q_full + 1, SL::TILE);
+#pragma unroll
+                    for (int c = 0; c < NBLK; ++c)
+                        tma_load_3d(smem + SL::Q + SL::TILE + c * BLK_BYTES, &tmQ, q_full + 1, c * 64, tw[1].hq, seq0 + tw[1].qt * BM);
+                }
             }
-            bool ok = true;
-            for (int j = 0; j < n_kv && ok; ++j) {
+            __syncwarp();
+            for (int j = 0; j < n_kv; ++j) {
                 const int sk = j % NK, uk = j / NK, sv = j % NV, uv = j / NV;
-                if (uk > 0) ok = mbar_wait(k_empty + sk, (uint32_t)((uk - 1) & 1), abort_flag, p.status, 10);
-                if (!ok) break;
-                mbar_expect_tx(k_full + sk, SL::TILE);
+                if (uk > 0 && !warp_wait(k_empty + sk, (uint32_t)((uk - 1) & 1), abort_flag, p.status, 10)) break;
+                if (leader) {
+                    mbar_expect_tx(k_full + sk, SL::TILE);
 #pragma unroll
-                for (int c = 0; c < NBLK; ++c)
-                    tma_load_3d(smem + SL::K + sk * SL::TILE + c * BLK_BYTES, &tmK, k_full + sk, c * 64, hkv, seq0 + j * BN);
-                if (uv > 0) ok = mbar_wait(v_empty + sv, (uint32_t)((uv - 1) & 1), abort_flag, p.status, 11);
-                if (!ok) break;
-                mbar_expect_tx(v_full + sv, SL::TILE);
+                    for (int c = 0; c < NBLK; ++c)
+                        tma_load_3d(smem + SL::K + sk * SL::TILE + c * BLK_BYTES, &tmK, k_full + sk, c * 64, hkv, seq0 + j * BN);
+                }
+                __syncwarp();
+                if (uv > 0 && !warp_wait(v_empty + sv, (uint32_t)((uv - 1) & 1), abort_flag, p.status, 11)) break;
+                if (leader) {
+                    mbar_expect_tx(v_full + sv, SL::TILE);
 #pragma unroll
-                for (int c = 0; c < NBLK; ++c)
-                    tma_load_3d(smem + SL::V + sv * SL::TILE + c * BLK_BYTES, &tmV, v_full + sv, c * 64, hkv, seq0 + j * BN);
+                    for (int c = 0; c < NBLK; ++c)
+                        tma_load_3d(smem + SL::V + sv * SL::TILE + c * BLK_BYTES, &tmV, v_full + sv, c * 64, hkv, seq0 + j * BN);
+                }
+                __syncwarp();
             }
-        } else if (warp == 1 && lane == 0) {
+        } else if (warp == 1) {
             // ------------------------------------------------------------ MMA issuer
             constexpr uint32_t IDESC_S = umma_idesc_bf16(BN, false);
             constexpr uint32_t IDESC_PV = umma_idesc_bf16(D, true);
-            const uint32_t sQa = smem_u32(smem + SL::Q), sKa = smem_u32(smem + SL::K), sVa = smem_u32(smem + SL::V);
+            constexpr uint32_t DESC_HI = umma_desc_hi_sw128(1024);
+            const uint32_t dQ = umma_desc_lo(smem_u32(smem + SL::Q), 16), dK = umma_desc_lo(smem_u32(smem + SL::K), 16);
+            const uint32_t dV = umma_desc_lo(smem_u32(smem + SL::V), BLK_BYTES);
             auto issue_S = [&](int x, int j) {
-                const uint32_t kbase = sKa + (uint32_t)(j % NK) * SL::TILE, qbase = sQa + (uint32_t)x * SL::TILE;
-#pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint32_t off = (uint32_t)(ks >> 2) * BLK_BYTES + (uint32_t)(ks & 3) * 32;
-                    umma_ss(tmem_base + COL_S + 128 * x, umma_desc_sw128(qbase + off, 16, 1024),
-                            umma_desc_sw128(kbase + off, 16, 1024), IDESC_S, ks > 0 ? 1u : 0u);
-                }
-                umma_commit(s_full + x);
-            };
-            auto issue_PV = [&](int x, int j) {
-                const uint32_t vbase = sVa + (uint32_t)(j % NV) * SL::TILE;
-#pragma unroll
-                for (int ks = 0; ks < BN / 16; ++ks)
-                    umma_ts(tmem_base + COL_O + D * x, tmem_base + COL_S + 128 * x + (uint32_t)ks * 8,
-                            umma_desc_sw128(vbase + (uint32_t)ks * 2048, BLK_BYTES, 1024), IDESC_PV, (j > 0 || ks > 0) ? 1u : 0u);
-            };
-            bool ok = mbar_wait(q_full + 0, 0, abort_flag, p.status, 20);
-            if (ok && nB > 0) ok = mbar_wait(q_full + 1, 0, abort_flag, p.status, 21);
-            if (ok) ok = mbar_wait(k_ready + 0, 0, abort_flag, p.status, 22);
-            if (ok) {
+                const uint32_t kd = dK + (uint32_t)(j % NK) * (SL::TILE >> 4), qd = dQ + (uint32_t)x * (SL::TILE >> 4);
+                const uint32_t dst = tmem_base + COL_S + 128 * x;
                 tc_fence_after();
+                if (leader) {
+#pragma unroll
+                    for (int ks = 0; ks < D / 16; ++ks) {
+                        // 16 elements along the contraction = 32 bytes inside a 64-element block
+                        const uint32_t off = ((uint32_t)(ks >> 2) * BLK_BYTES + (uint32_t)(ks & 3) * 32) >> 4;
+                        umma_ss(dst, qd + off, DESC_HI, kd + off, DESC_HI, IDESC_S, ks > 0 ? 1u : 0u);
+                    }
+                    umma_commit(s_full + x);
+                }
+                __syncwarp();
+            };
+            // P V of tile x and key tile j, key blocks [ks0, ks1) of 16 keys (2048 bytes of the V tile, 8 columns of P)
+            auto issue_PV = [&](int x, int j, int ks0, int ks1, bool last) {
+                const uint32_t vd = dV + (uint32_t)(j % NV) * (SL::TILE >> 4);
+                const uint32_t dst = tmem_base + COL_O + D * x, src = tmem_base + COL_S + 128 * x;
+                tc_fence_after();
+                if (leader) {
+#pragma unroll
+                    for (int ks = 0; ks < BN / 16; ++ks)
+                        if (ks >= ks0 && ks < ks1)
+                            umma_ts(dst, src + (uint32_t)ks * 8, vd + (uint32_t)ks * (2048 >> 4), DESC_HI, IDESC_PV,
+                                    (j > 0 || ks > 0) ? 1u : 0u);
+                    if (last) umma_commit(o_full + x);
+                }
+                __syncwarp();
+            };
+            auto commit = [&](uint64_t* bar) {
+                if (leader) umma_commit(bar);
+                __syncwarp();
+            };
+            // One thread issues for both tiles, in a fixed order: the in-order tensor pipe then keeps the two
+            // tiles half a period apart (softmax of one tile under the MMAs of the other).
+            bool ok = warp_wait(q_full + 0, 0, abort_flag, p.status, 20);
+            if (ok && nB > 0) ok = warp_wait(q_full + 1, 0, abort_flag, p.status, 21);
+            if (ok) ok = warp_wait(k_ready + 0, 0, abort_flag, p.status, 22);
+            if (ok) {
                 issue_S(0, 0);
                 if (nB > 0) issue_S(1, 0);
-                umma_commit(k_empty + 0);
+                commit(k_empty + 0);
             }
             for (int j = 0; j < n_kv && ok; ++j) {
                 const int sv = j % NV, j1 = j + 1, sk1 = j1 % NK;
-                const uint32_t par_k1 = (uint32_t)((j1 / NK) & 1);
-                ok = mbar_wait(v_full + sv, (uint32_t)((j / NV) & 1), abort_flag, p.status, 23);
+                // operands of this step and of the next score product: these waits end long before P arrives,
+                // so they are taken here, off the path between "P is ready" and the MMAs that consume it
+                ok = warp_wait(v_full + sv, (uint32_t)((j / NV) & 1), abort_flag, p.status, 23);
+                if (ok && j1 < n_kv) ok = warp_wait(k_ready + sk1, (uint32_t)((j1 / NK) & 1), abort_flag, p.status, 25);
                 if (!ok) break;
                 if (j < nA) {
-                    ok = mbar_wait(p_full + 0, (uint32_t)(j & 1), abort_flag, p.status, 24);
+                    ok = warp_wait(p_full + 0, (uint32_t)(j & 1), abort_flag, p.status, 24);
                     if (!ok) break;
-                    tc_fence_after();
-                    issue_PV(0, j);
-                    if (j == nA - 1) umma_commit(o_full + 0);
-                    if (j1 < nA) {
-                        ok = mbar_wait(k_ready + sk1, par_k1, abort_flag, p.status, 25);
-                        if (!ok) break;
-                        tc_fence_after();
-                        issue_S(0, j1);
-                    }
+                    issue_PV(0, j, 0, 6, false);
+                    ok = warp_wait(p_last + 0, (uint32_t)(j & 1), abort_flag, p.status, 28);
+                    if (!ok) break;
+                    issue_PV(0, j, 6, 8, j == nA - 1);
+                    if (j1 < nA) issue_S(0, j1);
                 }
                 if (j < nB) {
-                    ok = mbar_wait(p_full + 1, (uint32_t)(j & 1), abort_flag, p.status, 26);
+                    ok = warp_wait(p_full + 1, (uint32_t)(j & 1), abort_flag, p.status, 26);
                     if (!ok) break;
-                    tc_fence_after();
-                    issue_PV(1, j);
-                    if (j == nB - 1) umma_commit(o_full + 1);
-                }
-                umma_commit(v_empty + sv);
-                if (j1 < nB) {
-                    ok = mbar_wait(k_ready + sk1, par_k1, abort_flag, p.status, 27);
+                    issue_PV(1, j, 0, 6, false);
+                    ok = warp_wait(p_last + 1, (uint32_t)(j & 1), abort_flag, p.status, 29);
                     if (!ok) break;
-                    tc_fence_after();
-                    issue_S(1, j1);
+                    issue_PV(1, j, 6, 8, j == nB - 1);
                 }
-                if (j1 < n_kv) umma_commit(k_empty + sk1);
+                commit(v_empty + sv);
+                if (j1 < nB) issue_S(1, j1);
+                if (j1 < n_kv) commit(k_empty + sk1);
             }
         }
     } else if (warp >= 12) {
@@ -327,7 +358,8 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                 if (hl_mask & 0xffff0000u) edit_rows16_any<D>(sK, BLK_BYTES, wrow + 16, flags, fragB, fragA, colscale, nR16, lane);
                 fence_proxy_async();
             }
-            mbar_arrive(k_ready + sk);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(k_ready + sk);
         }
     } else {
         // ------------------------------------------------------------ softmax of tile x, one query row per thread
@@ -355,14 +387,15 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                 for (int e = 0; e < 128; ++e)
                     if (e > row) v[e] = 0xff800000u;
             }
-            float mx[4];
+            float mx[8];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                mx[q] = fmaxf(__uint_as_float(v[32 * q]), __uint_as_float(v[32 * q + 1]));
+            for (int q = 0; q < 8; ++q) {
+                mx[q] = fmaxf(__uint_as_float(v[16 * q]), __uint_as_float(v[16 * q + 1]));
 #pragma unroll
-                for (int e = 2; e < 32; e += 2) mx[q] = max3(mx[q], __uint_as_float(v[32 * q + e]), __uint_as_float(v[32 * q + e + 1]));
+                for (int e = 2; e < 16; e += 2) mx[q] = max3(mx[q], __uint_as_float(v[16 * q + e]), __uint_as_float(v[16 * q + e + 1]));
             }
-            const float m_new = fmaxf(m_run, fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale_log2);
+            const float mx_all = fmaxf(max3(mx[0], mx[1], mx[2]), max3(mx[3], mx[4], max3(mx[5], mx[6], mx[7])));
+            const float m_new = fmaxf(m_run, mx_all * p.scale_log2);
             // raise the running maximum only when it moved a lot; p may then exceed 1 (up to 2^8), which is harmless
             const bool raise = (m_new - m_run) > LAZY_RESCALE_LOG2;      // true on the first tile (m_run = -inf)
             const float factor = raise ? fast_exp2(m_run - m_new) : 1.f;
@@ -398,12 +431,19 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     pk16[e2] = pack_bf16(pe.x, pe.y);
                 }
                 tmem_st16(tS + c * 16, pk16);     // P (bf16 pairs) over score columns that are already in registers
+                if (c == 2) {                     // keys 0-95 are in place: the tensor core may start on them
+                    tmem_wait_st();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(p_full + x);
+                }
             }
-            const float2 s2 = __fadd2_rn(sum[0], sum[1]);
-            l_run = l_run * factor + (s2.x + s2.y);
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(p_full + x);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(p_last + x);
+            const float2 s2 = __fadd2_rn(sum[0], sum[1]);
+            l_run = l_run * factor + (s2.x + s2.y);
         }
         if (ok && nX > 0) ok = warp_wait(o_full + x, 0, abort_flag, p.status, 44 + x);
         if (ok && nX > 0) {
