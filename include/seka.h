@@ -57,7 +57,7 @@ typedef struct {
     int32_t n_kv_heads;         /* Hkv */
     int32_t head_dim;           /* d: 64 or 128 */
     int32_t rank;               /* r: columns stored per expert, 1 .. d */
-    int32_t n_experts;          /* M >= 1; M * r <= 128 */
+    int32_t n_experts;          /* M >= 1 */
     int32_t dtype;              /* seka_dtype of Q, K, V, O */
     float   softmax_scale;      /* 0 means 1/sqrt(head_dim) (Section 2) */
     const int32_t* cu_seqlens;  /* device int32 [B+1], or NULL for fixed length */

@@ -21,7 +21,7 @@ seka_status validate_shape(const seka_shape* s) {
     if ((long long)s->batch * s->max_seqlen > 0x7fffffffLL) return SEKA_ERR_UNSUPPORTED;
     if (s->head_dim != 64 && s->head_dim != 128) return SEKA_ERR_UNSUPPORTED;
     if (s->rank > s->head_dim) return SEKA_ERR_INVALID_ARG;
-    if ((long long)s->rank * s->n_experts > 128) return SEKA_ERR_UNSUPPORTED;
+    if ((long long)s->rank * s->n_experts > 4096) return SEKA_ERR_UNSUPPORTED;
     return SEKA_OK;
 }
 

@@ -1,14 +1,17 @@
 // Fused SEKA / AdaSEKA steered causal GQA attention forward for sm_100a.
 //
-// One CTA (16 warps) owns two consecutive tiles of 128 queries of one query head ("A" = lower rows,
-// "B" = upper rows) and walks the key tiles 0 .. diagonal.  Warp roles:
-//   warp 0        TMA producer: Q tiles once, then K and V tiles (128-byte swizzle) through two
-//                 shared-memory rings, throttled by "empty" mbarriers the tensor core signals;
-//   warps 12-15   key editors: for a staged K tile that contains highlighted tokens of a steered head,
-//                 k' = k + g * sum_m alpha_m U_m U_m^T k in place (Section 2 / Section 3.3, hook of
-//                 Algorithm 1/2) on warp-level MMAs (seka_edit_tile.cuh); then the tile is "ready";
-//   warp 1        MMA issuer: S_x = Q_x K'^T and O_x += P_x V on tcgen05 with all accumulators in
-//                 tensor memory (S_A, S_B, O_A, O_B = 512 columns); P_x is read from tensor memory;
+// One CTA (16 warps) owns two tiles of 128 queries that share a KV head ("A" and "B": two query heads of
+// one group at the same rows, or two consecutive row tiles of one head when the group size is odd) and
+// walks the key tiles 0 .. diagonal.  Warp roles:
+//   warp 0        TMA producer: Q tiles and the edit operator W once, then K and V tiles (128-byte swizzle)
+//                 through two shared-memory rings, throttled by "empty" mbarriers the tensor core signals;
+//   warp 1        MMA issuer: S_x = Q_x K'^T and O_x += P_x V on tcgen05 with all accumulators in tensor
+//                 memory (S_A, S_B, O_A, O_B = 512 columns); P_x is read from tensor memory.  For a staged
+//                 K tile that holds highlighted tokens of a steered head it first issues dK = K W into the
+//                 score columns of the tile that will use K first (they are idle just then);
+//   warps 12-15   key editors: read dK from tensor memory and add it, for highlighted rows only, to the
+//                 staged tile in place: k' = k + g * sum_m alpha_m U_m U_m^T k (Section 2 / Section 3.3, hook
+//                 of Algorithm 1/2) with W = g * sum_m alpha_m U_m U_m^T prepared per (sequence, KV head);
 //   warps 4-7 / 8-11  softmax of tile A / B, one query row per thread: causal mask on the diagonal
 //                 tile, online softmax in base 2 with a lazily updated running maximum, P written
 //                 back as bf16 over the consumed score columns, O rescaled in tensor memory only when
@@ -16,9 +19,11 @@
 // While one tile's softmax runs, the tensor core works on the other tile.  Neither K' nor the score
 // matrix ever reaches global memory; K and V are read only.  Every wait is bounded: a wait that runs
 // out raises the CTA's abort flag, every role leaves its loop, and the status word reports it.
+// The edit runs on tcgen05 like everything else: warp-level mma.sync is starved by a busy tcgen05 pipe
+// (it gets roughly one slot per UMMA), and its unrolled code evicts the other roles' loops from the
+// instruction cache.
 #include <math.h>
 
-#include "seka_edit_tile.cuh"
 #include "seka_kernels.h"
 
 #ifndef SEKA_POLY_PAIR_MASK
@@ -31,38 +36,41 @@ struct AttnParams {
     void* O;
     float* lse;
     const uint8_t* mask;
-    const float* alpha;
     const float* gain;
     const uint8_t* head_enable;
     const int* cu_seqlens;
-    const uint4* frags;
+    const uint8_t* tile_hot;      // [B, n_qt]: key tile holds a highlighted token
     int* status;
-    int B, L, Hq, Hkv, rank, M, r_pad, n_qt;
+    int B, L, Hq, Hkv, n_qt;
     int steer;
     int pair_heads;       // 1: the two tiles of a CTA are two query heads of one KV group; 0: two consecutive query tiles
     float scale_log2;
 };
 
 constexpr int BM = 128, BN = 128;
-constexpr int NK = 3, NV = 2;               // K and V ring depths
+constexpr int NV = 2;                       // V ring depth
 constexpr int NTHREADS = 512;
+constexpr int MAX_HOT_SMEM = 1024;          // per-tile highlight flags kept in shared memory (longer sequences read global memory)
 constexpr uint32_t BLK_BYTES = 128 * 128;   // one [128 x 64] bf16 block
 constexpr float LAZY_RESCALE_LOG2 = 8.0f;   // the running maximum is only raised when it moved by more than this
-// registers per thread after the roles split (the CTA owns the whole register file: 4 x 128 x (48+184+184+96) = 64 Ki)
-constexpr int REGS_CTRL = 48, REGS_SOFTMAX = 184, REGS_EDIT = 96;
+// registers per thread after the roles split (the CTA owns the whole register file: 4 x 128 x (72+168+168+104) = 64 Ki)
+constexpr int REGS_CTRL = 72, REGS_SOFTMAX = 168, REGS_EDIT = 104;
 // which of the 16 element pairs of every 32-key chunk take the polynomial exp2 instead of the special-function unit
 constexpr uint32_t POLY_PAIR_MASK = SEKA_POLY_PAIR_MASK;
 
 template <int D>
 struct SmemLayout {
+    // K ring depth: head_dim 128 leaves room for two stages beside the 32 KB edit operator, head_dim 64 for three
+    static constexpr int NK = D == 128 ? 2 : 3;
     static constexpr uint32_t TILE = (D / 64) * BLK_BYTES;
+    static constexpr uint32_t WBLK = D * 128;              // one [D x 64] block of W
     static constexpr uint32_t Q = 0;                       // 2 tiles
     static constexpr uint32_t K = Q + 2 * TILE;            // NK stages
     static constexpr uint32_t V = K + NK * TILE;           // NV stages
-    static constexpr uint32_t ROWFLAG = V + NV * TILE;     // NK x 128 bytes
-    static constexpr uint32_t COLSCALE = ROWFLAG + NK * 128;   // 128 floats
-    static constexpr uint32_t BARS = COLSCALE + 512;       // mbarriers
-    static constexpr uint32_t NBARS = 2 + 3 * NK + 2 * NV + 8;
+    static constexpr uint32_t W = V + NV * TILE;           // D x D bf16
+    static constexpr uint32_t HOT = W + (D / 64) * WBLK;   // MAX_HOT_SMEM bytes
+    static constexpr uint32_t BARS = HOT + MAX_HOT_SMEM;   // mbarriers
+    static constexpr uint32_t NBARS = 2 + 2 * NK + 2 * NV + 8 + 3;
     static constexpr uint32_t MISC = BARS + NBARS * 8;     // tmem holder, abort flag
     static constexpr uint32_t TOTAL = MISC + 16;
     static constexpr uint32_t DYN_BYTES = TOTAL + 1024;    // slack for the 1024-byte alignment
@@ -134,26 +142,29 @@ template <> __device__ __forceinline__ void store_chunk32<float>(float* dst, con
 template <int D, typename OutT>
 __global__ void __launch_bounds__(NTHREADS, 1)
 seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                     const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
+                     const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmW,
+                     const AttnParams p) {
     using SL = SmemLayout<D>;
+    constexpr int NK = SL::NK;
     constexpr int NBLK = D / 64;
     constexpr uint32_t TMEM_COLS = 512;
     constexpr uint32_t COL_S = 0, COL_O = 256;     // S_x at COL_S + 128 x, O_x at COL_O + D x
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t* rowflag = smem + SL::ROWFLAG;
-    float* colscale = reinterpret_cast<float*>(smem + SL::COLSCALE);
+    uint8_t* hot = smem + SL::HOT;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SL::BARS);
     uint64_t* q_full = bars;                 // [2]   TMA bytes landed
     uint64_t* k_full = q_full + 2;           // [NK]  TMA bytes landed
-    uint64_t* k_ready = k_full + NK;         // [NK]  4 editor-warp arrivals: tile may be multiplied
-    uint64_t* k_empty = k_ready + NK;        // [NK]  tensor core finished reading the stage
+    uint64_t* k_empty = k_full + NK;         // [NK]  tensor core finished reading the stage
     uint64_t* v_full = k_empty + NK;         // [NV]
     uint64_t* v_empty = v_full + NV;         // [NV]
     uint64_t* s_full = v_empty + NV;         // [2]   scores of tile x are in tensor memory
     uint64_t* p_full = s_full + 2;           // [2]   4 softmax-warp arrivals: O_x rescaled, keys 0-95 of P_x written
     uint64_t* p_last = p_full + 2;           // [2]   4 softmax-warp arrivals: keys 96-127 of P_x written
     uint64_t* o_full = p_last + 2;           // [2]   last P V of tile x finished
+    uint64_t* w_full = o_full + 2;           // [1]   edit operator landed
+    uint64_t* e_full = w_full + 1;           // [1]   dK = K W of the current highlighted tile is in tensor memory
+    uint64_t* k_edited = e_full + 1;         // [1]   4 editor-warp arrivals: the staged tile now holds K'
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + SL::MISC);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + SL::MISC + 4);
 
@@ -190,9 +201,10 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 
     if (tid == 0) {
         mbar_init(q_full + 0, 1); mbar_init(q_full + 1, 1);
-        for (int i = 0; i < NK; ++i) { mbar_init(k_full + i, 1); mbar_init(k_ready + i, 4); mbar_init(k_empty + i, 1); }
+        for (int i = 0; i < NK; ++i) { mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1); }
         for (int i = 0; i < NV; ++i) { mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(s_full + i, 1); mbar_init(p_full + i, 4); mbar_init(p_last + i, 4); mbar_init(o_full + i, 1); }
+        mbar_init(w_full, 1); mbar_init(e_full, 1); mbar_init(k_edited, 4);
         *abort_flag = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
@@ -200,14 +212,12 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     __syncwarp();
     if (warp == 0) { tmem_alloc(tmem_holder, TMEM_COLS); tmem_relinquish(); }
 
-    // steering parameters of this (sequence, KV head)
-    const float g = p.steer ? p.gain[b] : 0.f;
-    const bool steer = p.steer && g != 0.f && (p.head_enable == nullptr || p.head_enable[hkv] != 0);
-    if (steer && tid < 128) {
-        float cs = 0.f;
-        if (tid < p.M * p.rank) cs = g * (p.alpha ? p.alpha[((size_t)b * p.Hkv + hkv) * p.M + tid / p.rank] : 1.f);
-        colscale[tid] = cs;
-    }
+    // steering of this (sequence, KV head): which of its key tiles hold highlighted tokens
+    const bool steer = p.steer && p.gain[b] != 0.f && (p.head_enable == nullptr || p.head_enable[hkv] != 0);
+    const uint8_t* hot_g = p.tile_hot + (size_t)b * p.n_qt;
+    if (steer)
+        for (int i = tid; i < min(n_kv, MAX_HOT_SMEM); i += NTHREADS) hot[i] = hot_g[i];
+    auto tile_is_hot = [&](int j) -> bool { return steer && (j < MAX_HOT_SMEM ? hot[j] : hot_g[j]) != 0; };
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -231,8 +241,15 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     for (int c = 0; c < NBLK; ++c)
                         tma_load_3d(smem + SL::Q + SL::TILE + c * BLK_BYTES, &tmQ, q_full + 1, c * 64, tw[1].hq, seq0 + tw[1].qt * BM);
                 }
+                if (steer) {
+                    mbar_expect_tx(w_full, NBLK * SL::WBLK);
+#pragma unroll
+                    for (int c = 0; c < NBLK; ++c)
+                        tma_load_3d(smem + SL::W + c * SL::WBLK, &tmW, w_full, c * 64, 0, (b * p.Hkv + hkv) * D);
+                }
             }
             __syncwarp();
+#pragma unroll 1
             for (int j = 0; j < n_kv; ++j) {
                 const int sk = j % NK, uk = j / NK, sv = j % NV, uv = j / NV;
                 if (uk > 0 && !warp_wait(k_empty + sk, (uint32_t)((uk - 1) & 1), abort_flag, p.status, 10)) break;
@@ -256,9 +273,40 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             // ------------------------------------------------------------ MMA issuer
             constexpr uint32_t IDESC_S = umma_idesc_bf16(BN, false);
             constexpr uint32_t IDESC_PV = umma_idesc_bf16(D, true);
+            constexpr uint32_t IDESC_E = umma_idesc_bf16(D, false);
             constexpr uint32_t DESC_HI = umma_desc_hi_sw128(1024);
             const uint32_t dQ = umma_desc_lo(smem_u32(smem + SL::Q), 16), dK = umma_desc_lo(smem_u32(smem + SL::K), 16);
             const uint32_t dV = umma_desc_lo(smem_u32(smem + SL::V), BLK_BYTES);
+            const uint32_t dW = umma_desc_lo(smem_u32(smem + SL::W), 16);
+            int n_hot = 0;          // highlighted tiles edited so far (phase of e_full / k_edited)
+            bool ok = true;
+            auto commit = [&](uint64_t* bar) {
+                if (leader) umma_commit(bar);
+                __syncwarp();
+            };
+            // Before the first score product of key tile j (by tile x): if the tile holds highlighted tokens,
+            // dK = K W goes into the score columns of tile x (idle between P_x V and the next S_x), the editors
+            // add it to the staged tile, and only then may the tile be multiplied.
+            auto edit_K = [&](int x, int j) {
+                if (!tile_is_hot(j)) return;
+                if (n_hot == 0) ok = warp_wait(w_full, 0, abort_flag, p.status, 31);
+                if (!ok) return;
+                const uint32_t kd = dK + (uint32_t)(j % NK) * (SL::TILE >> 4);
+                const uint32_t dst = tmem_base + COL_S + 128 * x;
+                tc_fence_after();
+                if (leader) {
+#pragma unroll
+                    for (int ks = 0; ks < D / 16; ++ks) {
+                        const uint32_t offk = ((uint32_t)(ks >> 2) * BLK_BYTES + (uint32_t)(ks & 3) * 32) >> 4;
+                        const uint32_t offw = ((uint32_t)(ks >> 2) * SL::WBLK + (uint32_t)(ks & 3) * 32) >> 4;
+                        umma_ss(dst, kd + offk, DESC_HI, dW + offw, DESC_HI, IDESC_E, ks > 0 ? 1u : 0u);
+                    }
+                    umma_commit(e_full);
+                }
+                __syncwarp();
+                ok = warp_wait(k_edited, (uint32_t)(n_hot & 1), abort_flag, p.status, 32);
+                ++n_hot;
+            };
             auto issue_S = [&](int x, int j) {
                 const uint32_t kd = dK + (uint32_t)(j % NK) * (SL::TILE >> 4), qd = dQ + (uint32_t)x * (SL::TILE >> 4);
                 const uint32_t dst = tmem_base + COL_S + 128 * x;
@@ -289,26 +337,24 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                 }
                 __syncwarp();
             };
-            auto commit = [&](uint64_t* bar) {
-                if (leader) umma_commit(bar);
-                __syncwarp();
-            };
             // One thread issues for both tiles, in a fixed order: the in-order tensor pipe then keeps the two
             // tiles half a period apart (softmax of one tile under the MMAs of the other).
-            bool ok = warp_wait(q_full + 0, 0, abort_flag, p.status, 20);
+            ok = warp_wait(q_full + 0, 0, abort_flag, p.status, 20);
             if (ok && nB > 0) ok = warp_wait(q_full + 1, 0, abort_flag, p.status, 21);
-            if (ok) ok = warp_wait(k_ready + 0, 0, abort_flag, p.status, 22);
+            if (ok) ok = warp_wait(k_full + 0, 0, abort_flag, p.status, 22);
+            if (ok) edit_K(0, 0);
             if (ok) {
                 issue_S(0, 0);
                 if (nB > 0) issue_S(1, 0);
                 commit(k_empty + 0);
             }
+#pragma unroll 1
             for (int j = 0; j < n_kv && ok; ++j) {
                 const int sv = j % NV, j1 = j + 1, sk1 = j1 % NK;
                 // operands of this step and of the next score product: these waits end long before P arrives,
                 // so they are taken here, off the path between "P is ready" and the MMAs that consume it
                 ok = warp_wait(v_full + sv, (uint32_t)((j / NV) & 1), abort_flag, p.status, 23);
-                if (ok && j1 < n_kv) ok = warp_wait(k_ready + sk1, (uint32_t)((j1 / NK) & 1), abort_flag, p.status, 25);
+                if (ok && j1 < n_kv) ok = warp_wait(k_full + sk1, (uint32_t)((j1 / NK) & 1), abort_flag, p.status, 25);
                 if (!ok) break;
                 if (j < nA) {
                     ok = warp_wait(p_full + 0, (uint32_t)(j & 1), abort_flag, p.status, 24);
@@ -317,7 +363,11 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     ok = warp_wait(p_last + 0, (uint32_t)(j & 1), abort_flag, p.status, 28);
                     if (!ok) break;
                     issue_PV(0, j, 6, 8, j == nA - 1);
-                    if (j1 < nA) issue_S(0, j1);
+                    if (j1 < nA) {
+                        edit_K(0, j1);
+                        if (!ok) break;
+                        issue_S(0, j1);
+                    }
                 }
                 if (j < nB) {
                     ok = warp_wait(p_full + 1, (uint32_t)(j & 1), abort_flag, p.status, 26);
@@ -328,38 +378,57 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     issue_PV(1, j, 6, 8, j == nB - 1);
                 }
                 commit(v_empty + sv);
-                if (j1 < nB) issue_S(1, j1);
+                if (j1 < nB) {
+                    if (j1 >= nA) edit_K(1, j1);      // tile A does not use this key tile: B is its first user
+                    if (!ok) break;
+                    issue_S(1, j1);
+                }
                 if (j1 < n_kv) commit(k_empty + sk1);
             }
         }
     } else if (warp >= 12) {
-        // ------------------------------------------------------------ key editors (32 rows of every K tile per warp)
+        // ------------------------------------------------------------ key editors: one key row of the staged tile per thread
         reg_dec<REGS_EDIT>();
-        const int wrow = (warp - 12) * 32;
-        const size_t fr_head = frag_uint4_per_head(D, p.r_pad);
-        const uint4* fragB = p.frags + (size_t)hkv * fr_head;
-        const uint4* fragA = fragB + fr_head / 2;
-        const int nR16 = p.r_pad / 16;
-        for (int j = 0; j < n_kv; ++j) {
-            const int sk = j % NK;
-            uint8_t* flags = rowflag + sk * 128;
-            unsigned hl_mask = 0;
-            if (steer) {
-                const int kpos = j * BN + wrow + lane;
+        if (steer) {
+            const int row = (warp - 12) * 32 + lane;
+            const uint32_t t_lane = tmem_base + ((uint32_t)((warp - 12) * 32) << 16);
+            int n_hot = 0;
+#pragma unroll 1
+            for (int j = 0; j < n_kv; ++j) {
+                if (!tile_is_hot(j)) continue;
+                const int kpos = j * BN + row;
                 const bool hl = kpos < Lb && p.mask[seq0 + kpos] != 0;
-                flags[wrow + lane] = hl ? 1 : 0;
-                hl_mask = __ballot_sync(0xffffffffu, hl);
+                if (!warp_wait(e_full, (uint32_t)(n_hot & 1), abort_flag, p.status, 30)) break;
+                ++n_hot;
+                tc_fence_after();
+                const uint32_t tE = t_lane + COL_S + 128 * (j < nA ? 0 : 1);
+                uint8_t* sK = smem + SL::K + (j % NK) * SL::TILE;
+#pragma unroll 1
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t dk[32];
+                    tmem_ld32(tE + c * 32, dk);
+                    tmem_wait_ld_on(dk);
+                    if (hl) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {      // 8 elements = one 16-byte unit of the swizzled row
+                            const int col = c * 32 + q * 8;
+                            uint4* ptr = reinterpret_cast<uint4*>(sK + (col >> 6) * BLK_BYTES + sw128_offset(row, col & 63));
+                            uint4 kv = *ptr;
+                            uint32_t* w = reinterpret_cast<uint32_t*>(&kv);
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const float2 k2 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&w[e]));
+                                w[e] = pack_bf16(k2.x + __uint_as_float(dk[q * 8 + 2 * e]), k2.y + __uint_as_float(dk[q * 8 + 2 * e + 1]));
+                            }
+                            *ptr = kv;
+                        }
+                    }
+                }
+                fence_proxy_async();       // the rewritten rows are read next by the tensor core
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(k_edited);
             }
-            if (!warp_wait(k_full + sk, (uint32_t)((j / NK) & 1), abort_flag, p.status, 30)) break;
-            if (hl_mask != 0) {
-                __syncwarp();      // the flags written above are read by other lanes of this warp
-                uint8_t* sK = smem + SL::K + sk * SL::TILE;
-                if (hl_mask & 0x0000ffffu) edit_rows16_any<D>(sK, BLK_BYTES, wrow, flags, fragB, fragA, colscale, nR16, lane);
-                if (hl_mask & 0xffff0000u) edit_rows16_any<D>(sK, BLK_BYTES, wrow + 16, flags, fragB, fragA, colscale, nR16, lane);
-                fence_proxy_async();
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(k_ready + sk);
         }
     } else {
         // ------------------------------------------------------------ softmax of tile x, one query row per thread
@@ -377,49 +446,61 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             ok = warp_wait(s_full + x, (uint32_t)(j & 1), abort_flag, p.status, 40 + x);
             if (!ok) break;
             tc_fence_after();
-            // the whole score row of this thread: 128 fp32 values in registers
-            uint32_t v[128];
+            // The 128 scores of this thread's row are read from tensor memory twice (row maximum, then
+            // exponentials), 32 at a time through two register buffers, each load in flight under the
+            // arithmetic of the previous chunk.  The loops are kept rolled on purpose: the code of all roles of
+            // a key-tile step has to stay resident in the instruction cache.
+            const bool diag = (j == nX - 1);     // diagonal tile: keys after the query are masked
+            uint32_t a[32], b[32];
+            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            auto chunk_max = [&](uint32_t (&r)[32], int c) {
+                if (diag) {
+                    const int lim = row - 32 * c;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, reinterpret_cast<uint32_t(&)[32]>(v[32 * c]));
-            tmem_wait_ld();
-            if (j == nX - 1) {       // diagonal tile: keys after the query are masked
+                    for (int e = 0; e < 32; ++e)
+                        if (e > lim) r[e] = 0xff800000u;
+                }
 #pragma unroll
-                for (int e = 0; e < 128; ++e)
-                    if (e > row) v[e] = 0xff800000u;
+                for (int e = 0; e < 32; e += 8) {
+                    mx[0] = max3(mx[0], __uint_as_float(r[e]), __uint_as_float(r[e + 1]));
+                    mx[1] = max3(mx[1], __uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
+                    mx[2] = max3(mx[2], __uint_as_float(r[e + 4]), __uint_as_float(r[e + 5]));
+                    mx[3] = max3(mx[3], __uint_as_float(r[e + 6]), __uint_as_float(r[e + 7]));
+                }
+            };
+            tmem_ld32(tS, a);
+#pragma unroll 1
+            for (int h = 0; h < 2; ++h) {
+                tmem_wait_ld_on(a);
+                tmem_ld32(tS + 64 * h + 32, b);
+                chunk_max(a, 2 * h);
+                tmem_wait_ld_on(b);
+                tmem_ld32(tS + ((64 * h + 64) & 127), a);     // next chunk; after the last one: chunk 0 again, for the second pass
+                chunk_max(b, 2 * h + 1);
             }
-            float mx[8];
-#pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                mx[q] = fmaxf(__uint_as_float(v[16 * q]), __uint_as_float(v[16 * q + 1]));
-#pragma unroll
-                for (int e = 2; e < 16; e += 2) mx[q] = max3(mx[q], __uint_as_float(v[16 * q + e]), __uint_as_float(v[16 * q + e + 1]));
-            }
-            const float mx_all = fmaxf(max3(mx[0], mx[1], mx[2]), max3(mx[3], mx[4], max3(mx[5], mx[6], mx[7])));
-            const float m_new = fmaxf(m_run, mx_all * p.scale_log2);
+            const float m_new = fmaxf(m_run, fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale_log2);
             // raise the running maximum only when it moved a lot; p may then exceed 1 (up to 2^8), which is harmless
             const bool raise = (m_new - m_run) > LAZY_RESCALE_LOG2;      // true on the first tile (m_run = -inf)
             const float factor = raise ? fast_exp2(m_run - m_new) : 1.f;
             if (raise) m_run = m_new;
             if (j > 0 && __any_sync(0xffffffffu, raise)) {
-                uint32_t o[32];
 #pragma unroll 1
                 for (int c = 0; c < D / 32; ++c) {
-                    tmem_ld32(tO + c * 32, o);
-                    tmem_wait_ld();
+                    tmem_ld32(tO + c * 32, b);
+                    tmem_wait_ld_on(b);
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * factor);
-                    tmem_st32(tO + c * 32, o);
+                    for (int e = 0; e < 32; ++e) b[e] = __float_as_uint(__uint_as_float(b[e]) * factor);
+                    tmem_st32(tO + c * 32, b);
                 }
             }
             const float2 nm2 = make_float2(-m_run, -m_run);
             float2 sum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
+            auto chunk_exp = [&](const uint32_t (&r)[32], int c) {
                 uint32_t pk16[16];
+                const int lim = diag ? row - 32 * c : 32;
 #pragma unroll
                 for (int e2 = 0; e2 < 16; ++e2) {
-                    const int e = 32 * c + 2 * e2;
-                    const float2 arg = __ffma2_rn(make_float2(__uint_as_float(v[e]), __uint_as_float(v[e + 1])), sc2, nm2);
+                    const float2 arg = __ffma2_rn(make_float2(__uint_as_float(r[2 * e2]), __uint_as_float(r[2 * e2 + 1])), sc2, nm2);
                     float2 pe;
                     if ((POLY_PAIR_MASK >> e2) & 1u) {
                         pe = exp2_poly2(arg);
@@ -427,16 +508,29 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                         pe.x = fast_exp2(arg.x);
                         pe.y = fast_exp2(arg.y);
                     }
+                    if (diag) {
+                        if (2 * e2 > lim) pe.x = 0.f;
+                        if (2 * e2 + 1 > lim) pe.y = 0.f;
+                    }
                     sum[e2 & 1] = __fadd2_rn(sum[e2 & 1], pe);
                     pk16[e2] = pack_bf16(pe.x, pe.y);
                 }
-                tmem_st16(tS + c * 16, pk16);     // P (bf16 pairs) over score columns that are already in registers
-                if (c == 2) {                     // keys 0-95 are in place: the tensor core may start on them
+                tmem_st16(tS + c * 16, pk16);     // P (bf16 pairs) over score columns that have been consumed
+            };
+#pragma unroll 1
+            for (int h = 0; h < 2; ++h) {
+                tmem_wait_ld_on(a);
+                tmem_ld32(tS + 64 * h + 32, b);
+                chunk_exp(a, 2 * h);
+                if (h == 1) {                     // keys 0-95 are in place: the tensor core may start on them
                     tmem_wait_st();
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(p_full + x);
                 }
+                tmem_wait_ld_on(b);
+                if (h == 0) tmem_ld32(tS + 64, a);
+                chunk_exp(b, 2 * h + 1);
             }
             tmem_wait_st();
             tc_fence_before();
@@ -493,13 +587,13 @@ static EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-// bf16 tensor [T, H, d] viewed as (d, H, T); tiles of 64 x 1 x 128 with the 128-byte swizzle.
-static bool make_tile_map(CUtensorMap* m, const void* base, int d, int H, int T) {
+// bf16 tensor [T, H, d] viewed as (d, H, T); tiles of 64 x 1 x box_rows with the 128-byte swizzle.
+static bool make_tile_map(CUtensorMap* m, const void* base, int d, int H, long long T, int box_rows = 128) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (fn == nullptr) return false;
     cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)H, (cuuint64_t)T};
     cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)H * d * 2};
-    cuuint32_t box[3] = {64, 1, 128};
+    cuuint32_t box[3] = {64, 1, (cuuint32_t)box_rows};
     cuuint32_t estr[3] = {1, 1, 1};
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -508,7 +602,7 @@ static bool make_tile_map(CUtensorMap* m, const void* base, int d, int H, int T)
 
 template <int D, typename OutT>
 static seka_status launch_attn(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                               const AttnParams& p, cudaStream_t st) {
+                               const CUtensorMap& tw, const AttnParams& p, cudaStream_t st) {
     using SL = SmemLayout<D>;
     static bool configured = false;
     if (!configured) {
@@ -517,7 +611,7 @@ static seka_status launch_attn(const CUtensorMap& tq, const CUtensorMap& tk, con
         configured = true;
     }
     const unsigned grid = p.pair_heads ? (unsigned)p.n_qt * p.B * (p.Hq / 2) : (unsigned)((p.n_qt + 1) / 2) * p.B * p.Hq;
-    seka_attn_fwd_kernel<D, OutT><<<grid, NTHREADS, SL::DYN_BYTES, st>>>(tq, tk, tv, p);
+    seka_attn_fwd_kernel<D, OutT><<<grid, NTHREADS, SL::DYN_BYTES, st>>>(tq, tk, tv, tw, p);
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? SEKA_OK : SEKA_ERR_CUDA;
 }
@@ -554,28 +648,30 @@ extern "C" seka_status seka_attention_fwd(const seka_shape* shape, const void* Q
         launch_convert_bf16(static_cast<const float*>(V), cv, nk, st);
         q16 = cq; k16 = ck; v16 = cv;
     }
-    uint4* frags = reinterpret_cast<uint4*>(ws + w.frag_off);
-    if (steer) launch_prep_fragments(U, frags, Hkv, D, shape->rank, shape->n_experts, w.r_pad, st);
+    void* W = ws + w.w_off;
+    uint8_t* tile_hot = reinterpret_cast<uint8_t*>(ws + w.hot_off);
+    if (steer) launch_prep_steering(shape, U, alpha, gain, head_enable, mask, W, tile_hot, w.n_tiles, st);
 
-    CUtensorMap tq, tk, tv;
-    if (!make_tile_map(&tq, q16, D, Hq, T) || !make_tile_map(&tk, k16, D, Hkv, T) || !make_tile_map(&tv, v16, D, Hkv, T))
+    CUtensorMap tq, tk, tv, tw;
+    if (!make_tile_map(&tq, q16, D, Hq, T) || !make_tile_map(&tk, k16, D, Hkv, T) || !make_tile_map(&tv, v16, D, Hkv, T) ||
+        !make_tile_map(&tw, W, D, 1, (long long)shape->batch * Hkv * D, D))
         return SEKA_ERR_CUDA;
 
     AttnParams p;
-    p.O = O; p.lse = lse; p.mask = mask; p.alpha = alpha; p.gain = gain; p.head_enable = head_enable;
-    p.cu_seqlens = shape->cu_seqlens; p.frags = frags; p.status = reinterpret_cast<int*>(ws);
-    p.B = shape->batch; p.L = shape->max_seqlen; p.Hq = Hq; p.Hkv = Hkv; p.rank = shape->rank; p.M = shape->n_experts;
-    p.r_pad = w.r_pad; p.n_qt = (shape->max_seqlen + BM - 1) / BM; p.steer = steer ? 1 : 0;
+    p.O = O; p.lse = lse; p.mask = mask; p.gain = gain; p.head_enable = head_enable;
+    p.cu_seqlens = shape->cu_seqlens; p.tile_hot = tile_hot; p.status = reinterpret_cast<int*>(ws);
+    p.B = shape->batch; p.L = shape->max_seqlen; p.Hq = Hq; p.Hkv = Hkv;
+    p.n_qt = w.n_tiles; p.steer = steer ? 1 : 0;
     p.pair_heads = ((Hq / Hkv) % 2 == 0) ? 1 : 0;
     const float scale = shape->softmax_scale > 0.f ? shape->softmax_scale : 1.f / sqrtf((float)D);
     p.scale_log2 = scale * 1.4426950408889634f;
 
     if (D == 128) {
-        return shape->dtype == SEKA_F32 ? launch_attn<128, float>(tq, tk, tv, p, st)
-                                        : launch_attn<128, __nv_bfloat16>(tq, tk, tv, p, st);
+        return shape->dtype == SEKA_F32 ? launch_attn<128, float>(tq, tk, tv, tw, p, st)
+                                        : launch_attn<128, __nv_bfloat16>(tq, tk, tv, tw, p, st);
     }
-    return shape->dtype == SEKA_F32 ? launch_attn<64, float>(tq, tk, tv, p, st)
-                                    : launch_attn<64, __nv_bfloat16>(tq, tk, tv, p, st);
+    return shape->dtype == SEKA_F32 ? launch_attn<64, float>(tq, tk, tv, tw, p, st)
+                                    : launch_attn<64, __nv_bfloat16>(tq, tk, tv, tw, p, st);
 }
 
 extern "C" size_t seka_host_staging_bytes(const seka_shape* shape) {

@@ -14,17 +14,19 @@ namespace seka {
 // ---------------------------------------------------------------- workspace layout
 // [0, 256)            status block: word 0 = seka_status, word 1 = where the wait gave up,
 //                     word 2 = number of highlighted tokens found by the compaction pass
-// [256, ...)          U operand fragments for the tensor-core edit (per KV head)
+// [256, ...)          dense edit operators W[b][h] = gain_b * sum_m alpha_{b,h,m} U_m U_m^T as bf16 [D x D]
+// then                one byte per (sequence, 128-key tile): the tile contains a highlighted token
 // then                compacted highlighted-token list (int32 per token)
 // then (fp32 inputs)  bf16 copies of Q, K, V
 constexpr size_t kStatusBytes = 256;
 
 struct WorkspaceLayout {
-    size_t frag_off, frag_bytes;      // per head: B fragments then A fragments
+    size_t w_off, w_bytes;            // bf16 [B, Hkv, D, D]
+    size_t hot_off, hot_bytes;        // uint8 [B, ceil(max_seqlen / 128)]
     size_t list_off, list_bytes;      // int32 [total_tokens]
     size_t cvt_off, cvt_bytes;        // bf16 copies of Q, K, V (fp32 inputs only)
     size_t total;
-    int r_pad;                        // M * r rounded up to 16, 32, 64 or 128
+    int n_tiles;                      // key tiles per sequence = ceil(max_seqlen / 128)
 };
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -36,11 +38,12 @@ static inline int shape_total_tokens(const seka_shape* s) {
 static inline WorkspaceLayout workspace_layout(const seka_shape* s) {
     WorkspaceLayout w;
     const size_t T = (size_t)shape_total_tokens(s);
-    w.r_pad = 16;
-    while (w.r_pad < s->n_experts * s->rank) w.r_pad *= 2;
-    w.frag_off = kStatusBytes;
-    w.frag_bytes = align_up((size_t)s->n_kv_heads * 2 * (size_t)s->head_dim * w.r_pad * 2, 256);
-    w.list_off = w.frag_off + w.frag_bytes;
+    w.n_tiles = (s->max_seqlen + 127) / 128;
+    w.w_off = kStatusBytes;
+    w.w_bytes = align_up((size_t)s->batch * s->n_kv_heads * s->head_dim * s->head_dim * 2, 1024);
+    w.hot_off = w.w_off + w.w_bytes;
+    w.hot_bytes = align_up((size_t)s->batch * w.n_tiles + 1, 256);
+    w.list_off = w.hot_off + w.hot_bytes;
     w.list_bytes = align_up(T * 4 + 4, 256);
     w.cvt_off = w.list_off + w.list_bytes;
     w.cvt_bytes = 0;
@@ -197,6 +200,17 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
           "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
           "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr) : "memory");
+}
+// Waits for the tensor-memory loads of this thread; the registers of the load that is about to be used are
+// named as operands so that no use of them can be scheduled ahead of the wait.
+__device__ __forceinline__ void tmem_wait_ld_on(uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.wait::ld.sync.aligned;"
+        : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+          "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+          "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+          "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+        :: "memory");
 }
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
     asm volatile(

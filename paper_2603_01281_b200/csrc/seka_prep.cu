@@ -1,50 +1,67 @@
-// Small preparation kernels: U -> MMA operand fragments, highlight-mask compaction,
-// fp32 -> bf16 input conversion.
-#include "seka_edit_tile.cuh"
+// Small preparation kernels: dense edit operators and per-tile highlight flags for the fused kernel,
+// highlight-mask compaction, fp32 -> bf16 input conversion.
 #include "seka_kernels.h"
 
 namespace seka {
 
-// Ustack[i][j] = U[m = j / r][h][i][j % r] for j < M*r, 0 on the padding columns.
-__device__ __forceinline__ float ustack(const float* __restrict__ U, int Hkv, int D, int r, int M, int h, int i, int j) {
-    if (j >= M * r) return 0.f;
-    const int m = j / r, jj = j - m * r;
-    return U[(((size_t)m * Hkv + h) * D + i) * r + jj];
-}
-
-// One thread per uint4 of the fragment store (layout documented in seka_edit_tile.cuh).
-__global__ void prep_fragments_kernel(const float* __restrict__ U, uint4* __restrict__ frags,
-                                      int Hkv, int D, int r, int M, int r_pad) {
-    const int KB = D / 16, NR = r_pad / 16;
-    const size_t per_half = (size_t)KB * NR * 32;
-    const size_t total = (size_t)Hkv * 2 * per_half;
-    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= total) return;
-    const int h = (int)(idx / (2 * per_half));
-    size_t rem = idx - (size_t)h * 2 * per_half;
-    const bool second = rem >= per_half;
-    if (second) rem -= per_half;
-    const int lane = (int)(rem & 31);
-    const int g = lane >> 2, t = lane & 3;
-    uint32_t w[4];
-    if (!second) {
-        // operand of T = K * Ustack: B[k = head-dim index][n = stacked column]
-        const int np = (int)((rem >> 5) % NR), kb = (int)((rem >> 5) / NR);
-        for (int q = 0; q < 2; ++q) {
-            const int n = (2 * np + q) * 8 + g, k = kb * 16 + 2 * t;
-            w[2 * q + 0] = pack_bf16(ustack(U, Hkv, D, r, M, h, k, n), ustack(U, Hkv, D, r, M, h, k + 1, n));
-            w[2 * q + 1] = pack_bf16(ustack(U, Hkv, D, r, M, h, k + 8, n), ustack(U, Hkv, D, r, M, h, k + 9, n));
+// Operand preparation of the fused kernel, one launch:
+//   blocks [0, n_w):   a 32 x 32 tile of W[b][h] = gain_b * sum_m alpha_{b,h,m} U_m[h] U_m[h]^T  (bf16 [D x D]; the
+//                      dynamic projector of Section 3.3 times the gain, or g U U^T for plain SEKA), so that the
+//                      edit of a key tile is one product  K' = K + K W  (W is symmetric).  Pairs (b, h) that are
+//                      not steered (zero gain, head switched off) are skipped: the fused kernel never reads them.
+//   blocks [n_w, ...): one warp per (sequence, 128-key tile): does the tile hold a highlighted token?
+__global__ void prep_steering_kernel(const float* __restrict__ U, const float* __restrict__ alpha,
+                                     const float* __restrict__ gain, const uint8_t* __restrict__ head_enable,
+                                     const uint8_t* __restrict__ mask, const int* __restrict__ cu_seqlens,
+                                     __nv_bfloat16* __restrict__ W, uint8_t* __restrict__ tile_hot,
+                                     int B, int L, int Hkv, int D, int r, int M, int n_tiles, int n_w) {
+    const int tid = threadIdx.x;
+    if ((int)blockIdx.x < n_w) {
+        const int tiles = D / 32;
+        const int bh = blockIdx.x / (tiles * tiles), t = blockIdx.x % (tiles * tiles);
+        const int b = bh / Hkv, h = bh % Hkv;
+        const float g = gain[b];
+        if (g == 0.f || (head_enable != nullptr && head_enable[h] == 0)) return;
+        const int i0 = (t / tiles) * 32, j0 = (t % tiles) * 32;
+        __shared__ float ui[32][33], uj[32][33];
+        const int tx = tid & 31, ty = tid >> 5;          // 256 threads: 8 rows of 32
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int m = 0; m < M; ++m) {
+            const float a = g * (alpha != nullptr ? alpha[((size_t)b * Hkv + h) * M + m] : 1.f);
+            const float* Um = U + ((size_t)m * Hkv + h) * D * r;
+            for (int k0 = 0; k0 < r; k0 += 32) {
+                __syncthreads();
+                for (int q = ty; q < 32; q += 8) {
+                    const bool in = k0 + tx < r;
+                    ui[q][tx] = in ? a * Um[(size_t)(i0 + q) * r + k0 + tx] : 0.f;
+                    uj[q][tx] = in ? Um[(size_t)(j0 + q) * r + k0 + tx] : 0.f;
+                }
+                __syncthreads();
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int i = ty + 8 * q;
+#pragma unroll 8
+                    for (int k = 0; k < 32; ++k) acc[q] = fmaf(ui[i][k], uj[tx][k], acc[q]);
+                }
+            }
         }
+        __nv_bfloat16* Wbh = W + (size_t)bh * D * D;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) Wbh[(size_t)(i0 + ty + 8 * q) * D + j0 + tx] = __float2bfloat16_rn(acc[q]);
     } else {
-        // operand of dK = T * Ustack^T: B[k = stacked column][n = head-dim index]
-        const int np2 = (int)((rem >> 5) % KB), kb2 = (int)((rem >> 5) / KB);
-        for (int q = 0; q < 2; ++q) {
-            const int i = (2 * np2 + q) * 8 + g, k = kb2 * 16 + 2 * t;
-            w[2 * q + 0] = pack_bf16(ustack(U, Hkv, D, r, M, h, i, k), ustack(U, Hkv, D, r, M, h, i, k + 1));
-            w[2 * q + 1] = pack_bf16(ustack(U, Hkv, D, r, M, h, i, k + 8), ustack(U, Hkv, D, r, M, h, i, k + 9));
+        const int item = ((int)blockIdx.x - n_w) * 8 + (tid >> 5), lane = tid & 31;
+        if (item >= B * n_tiles) return;
+        const int b = item / n_tiles, t = item % n_tiles;
+        const int seq0 = cu_seqlens ? cu_seqlens[b] : b * L;
+        const int Lb = (cu_seqlens ? cu_seqlens[b + 1] : (b + 1) * L) - seq0;
+        bool any = false;
+        for (int q = 0; q < 4; ++q) {
+            const int pos = t * 128 + q * 32 + lane;
+            any = any || (pos < Lb && mask[seq0 + pos] != 0);
         }
+        any = __any_sync(0xffffffffu, any);
+        if (lane == 0) tile_hot[item] = any ? 1 : 0;
     }
-    frags[idx] = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
 // Appends the indices of highlighted tokens to `list` (order within a warp preserved).
@@ -68,9 +85,16 @@ __global__ void convert_f32_bf16_kernel(const float4* __restrict__ in, uint2* __
     out[i] = make_uint2(pack_bf16(v.x, v.y), pack_bf16(v.z, v.w));
 }
 
-void launch_prep_fragments(const float* U, uint4* frags, int Hkv, int D, int r, int M, int r_pad, cudaStream_t st) {
-    const size_t total = (size_t)Hkv * frag_uint4_per_head(D, r_pad);
-    prep_fragments_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(U, frags, Hkv, D, r, M, r_pad);
+void launch_prep_steering(const seka_shape* sh, const float* U, const float* alpha, const float* gain,
+                          const uint8_t* head_enable, const uint8_t* mask, void* W, uint8_t* tile_hot, int n_tiles,
+                          cudaStream_t st) {
+    const int D = sh->head_dim, tiles = D / 32;
+    const int n_w = sh->batch * sh->n_kv_heads * tiles * tiles;
+    const int n_flag = (sh->batch * n_tiles + 7) / 8;
+    prep_steering_kernel<<<n_w + n_flag, 256, 0, st>>>(U, alpha, gain, head_enable, mask, sh->cu_seqlens,
+                                                      static_cast<__nv_bfloat16*>(W), tile_hot, sh->batch,
+                                                      sh->max_seqlen, sh->n_kv_heads, D, sh->rank, sh->n_experts,
+                                                      n_tiles, n_w);
     ++g_launches;
 }
 

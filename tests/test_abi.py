@@ -40,14 +40,14 @@ def shape(**kw):
 def test_workspace_bytes_and_validation(lib):
     s = shape()
     n = binding.seka_workspace_bytes(s)
-    assert n >= 256 + 2 * 128 * 32 * 2 * 2 + 512 * 4
+    assert n >= 256 + 2 * 2 * 128 * 128 * 2 + 2 * 2 + 512 * 4     # status, edit operators, tile flags, token list
     assert binding.seka_workspace_bytes(shape(dtype=binding.SEKA_F32)) > n       # bf16 staging of fp32 inputs
     assert binding.seka_workspace_bytes(shape(head_dim=96)) == 0
     assert binding.seka_workspace_bytes(shape(n_q_heads=7)) == 0
     assert binding.seka_host_staging_bytes(s) >= 512 * (8 + 2 + 2 + 8) * 128 * 2
 
     one = ctypes.c_void_p(256)       # never dereferenced: validation fails first
-    bad = [shape(head_dim=96), shape(n_q_heads=7), shape(rank=0), shape(rank=200), shape(n_experts=5, rank=32),
+    bad = [shape(head_dim=96), shape(n_q_heads=7), shape(rank=0), shape(rank=200), shape(n_experts=0),
            shape(dtype=7), shape(batch=-1), shape(total_tokens=100)]
     for s_bad in bad:
         st = lib.seka_attention_fwd(ctypes.byref(s_bad), one, one, one, one, None, None, None, None, None, None,

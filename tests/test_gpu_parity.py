@@ -84,11 +84,14 @@ def test_edit_keys_edge_cases():
 
 # ----------------------------------------------------------------- fused attention: small and edge cases
 
-def _fused_vs_oracle(w, alpha=None, head_enable=None, rows=None, force_varlen=False, label="", stress=False):
+def _fused_vs_oracle(w, alpha=None, head_enable=None, rows=None, force_varlen=False, label="", stress=False,
+                     short_rows=False):
     O, LSE = H.run_fused(w, alpha=alpha, head_enable=head_enable, force_varlen=force_varlen)
     Oref, Lref, idx = H.oracle_rows(w, rows, alpha=alpha, head_enable=head_enable)
-    # stress cases (|g| >= 2 on short rows): the stated bound times the key magnification, with 25 % slack
-    kappa = 1.25 * H.key_magnification(w) if stress else 1.0
+    # stress cases (|g| >= 2 on short rows): the stated bound times the key magnification, with 25 % slack;
+    # short sequences with g = 1: the bound times the key magnification (the edited keys are not unit
+    # variance, Eq. 12, and a row of a few hundred keys averages the rounding of k' over few terms)
+    kappa = 1.25 * H.key_magnification(w) if stress else (H.key_magnification(w) if short_rows else 1.0)
     mx, mean = H.check_attention(O[idx], Oref, label, kappa=kappa)
     np.testing.assert_allclose(LSE[idx], Lref, atol=2e-2 * kappa)
     return mx, mean
@@ -113,7 +116,7 @@ def test_fused_small_shapes(d, Hq, Hkv, r, g):
 def test_fused_ragged_lengths(lens):
     w = inputs.make_custom(seed=7, dtype="bf16", lens=lens, n_q_heads=4, n_kv_heads=2, head_dim=128, rank=16,
                            gain=1.0, mask_kind="runs", highlight=0.3)
-    _fused_vs_oracle(w, label=str(lens))
+    _fused_vs_oracle(w, label=str(lens), short_rows=True)
 
 
 def test_fused_mask_patterns_and_head_enable():
