@@ -53,8 +53,8 @@ constexpr int NTHREADS = 512;
 constexpr int MAX_HOT_SMEM = 1024;          // per-tile highlight flags kept in shared memory (longer sequences read global memory)
 constexpr uint32_t BLK_BYTES = 128 * 128;   // one [128 x 64] bf16 block
 constexpr float LAZY_RESCALE_LOG2 = 8.0f;   // the running maximum is only raised when it moved by more than this
-// registers per thread after the roles split (the CTA owns the whole register file: 4 x 128 x (72+168+168+104) = 64 Ki)
-constexpr int REGS_CTRL = 72, REGS_SOFTMAX = 168, REGS_EDIT = 104;
+// registers per thread after the roles split (the CTA owns the whole register file: 4 x 128 x (56+184+184+88) = 64 Ki)
+constexpr int REGS_CTRL = 56, REGS_SOFTMAX = 184, REGS_EDIT = 88;
 // which of the 16 element pairs of every 32-key chunk take the polynomial exp2 instead of the special-function unit
 constexpr uint32_t POLY_PAIR_MASK = SEKA_POLY_PAIR_MASK;
 
@@ -159,7 +159,7 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     uint64_t* v_full = k_empty + NK;         // [NV]
     uint64_t* v_empty = v_full + NV;         // [NV]
     uint64_t* s_full = v_empty + NV;         // [2]   scores of tile x are in tensor memory
-    uint64_t* p_full = s_full + 2;           // [2]   4 softmax-warp arrivals: O_x rescaled, keys 0-95 of P_x written
+    uint64_t* p_full = s_full + 2;           // [2]   4 softmax-warp arrivals (O_x rescaled, keys 0-95 of P_x written) + 1 from the operand relay
     uint64_t* p_last = p_full + 2;           // [2]   4 softmax-warp arrivals: keys 96-127 of P_x written
     uint64_t* o_full = p_last + 2;           // [2]   last P V of tile x finished
     uint64_t* w_full = o_full + 2;           // [1]   edit operator landed
@@ -203,7 +203,7 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         mbar_init(q_full + 0, 1); mbar_init(q_full + 1, 1);
         for (int i = 0; i < NK; ++i) { mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1); }
         for (int i = 0; i < NV; ++i) { mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(s_full + i, 1); mbar_init(p_full + i, 4); mbar_init(p_last + i, 4); mbar_init(o_full + i, 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(s_full + i, 1); mbar_init(p_full + i, 5); mbar_init(p_last + i, 4); mbar_init(o_full + i, 1); }
         mbar_init(w_full, 1); mbar_init(e_full, 1); mbar_init(k_edited, 4);
         *abort_flag = 0;
         mbar_fence_init();
@@ -351,11 +351,9 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 #pragma unroll 1
             for (int j = 0; j < n_kv && ok; ++j) {
                 const int sv = j % NV, j1 = j + 1, sk1 = j1 % NK;
-                // operands of this step and of the next score product: these waits end long before P arrives,
-                // so they are taken here, off the path between "P is ready" and the MMAs that consume it
-                ok = warp_wait(v_full + sv, (uint32_t)((j / NV) & 1), abort_flag, p.status, 23);
-                if (ok && j1 < n_kv) ok = warp_wait(k_full + sk1, (uint32_t)((j1 / NK) & 1), abort_flag, p.status, 25);
-                if (!ok) break;
+                // V of this step and K of the next have landed once p_full completes: the relay warp vouches for
+                // them there, so this warp has no waits of its own for operands (every wait here is a bubble in
+                // the tensor pipe: its queue is only a couple of MMAs deep)
                 if (j < nA) {
                     ok = warp_wait(p_full + 0, (uint32_t)(j & 1), abort_flag, p.status, 24);
                     if (!ok) break;
@@ -384,6 +382,22 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     issue_S(1, j1);
                 }
                 if (j1 < n_kv) commit(k_empty + sk1);
+            }
+        } else if (warp == 2) {
+            // ------------------------------------------------------------ operand relay: "V(j) and K(j+1) have landed" as a
+            // fifth arrival on p_full of step j, so that the MMA issuer waits on one barrier per hand-off
+#pragma unroll 1
+            for (int j = 0; j < n_kv; ++j) {
+                if (!warp_wait(v_full + j % NV, (uint32_t)((j / NV) & 1), abort_flag, p.status, 23)) break;
+                if (j + 1 < n_kv && !warp_wait(k_full + (j + 1) % NK, (uint32_t)(((j + 1) / NK) & 1), abort_flag, p.status, 25)) break;
+                if (lane == 0) {
+                    if (j < nA) mbar_arrive(p_full + 0);
+                    if (j < nB) mbar_arrive(p_full + 1);
+                }
+                __syncwarp();
+                // stay within the phase: the next arrival may only come after this phase has completed
+                if (j < nA && !warp_wait(p_full + 0, (uint32_t)(j & 1), abort_flag, p.status, 33)) break;
+                if (j < nB && !warp_wait(p_full + 1, (uint32_t)(j & 1), abort_flag, p.status, 34)) break;
             }
         }
     } else if (warp >= 12) {
@@ -446,61 +460,49 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             ok = warp_wait(s_full + x, (uint32_t)(j & 1), abort_flag, p.status, 40 + x);
             if (!ok) break;
             tc_fence_after();
-            // The 128 scores of this thread's row are read from tensor memory twice (row maximum, then
-            // exponentials), 32 at a time through two register buffers, each load in flight under the
-            // arithmetic of the previous chunk.  The loops are kept rolled on purpose: the code of all roles of
-            // a key-tile step has to stay resident in the instruction cache.
-            const bool diag = (j == nX - 1);     // diagonal tile: keys after the query are masked
-            uint32_t a[32], b[32];
-            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-            auto chunk_max = [&](uint32_t (&r)[32], int c) {
-                if (diag) {
-                    const int lim = row - 32 * c;
+            // the whole score row of this thread: 128 fp32 values in registers
+            uint32_t v[128];
 #pragma unroll
-                    for (int e = 0; e < 32; ++e)
-                        if (e > lim) r[e] = 0xff800000u;
-                }
+            for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, reinterpret_cast<uint32_t(&)[32]>(v[32 * c]));
+            tmem_wait_ld();
+            if (j == nX - 1) {       // diagonal tile: keys after the query are masked
 #pragma unroll
-                for (int e = 0; e < 32; e += 8) {
-                    mx[0] = max3(mx[0], __uint_as_float(r[e]), __uint_as_float(r[e + 1]));
-                    mx[1] = max3(mx[1], __uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
-                    mx[2] = max3(mx[2], __uint_as_float(r[e + 4]), __uint_as_float(r[e + 5]));
-                    mx[3] = max3(mx[3], __uint_as_float(r[e + 6]), __uint_as_float(r[e + 7]));
-                }
-            };
-            tmem_ld32(tS, a);
-#pragma unroll 1
-            for (int h = 0; h < 2; ++h) {
-                tmem_wait_ld_on(a);
-                tmem_ld32(tS + 64 * h + 32, b);
-                chunk_max(a, 2 * h);
-                tmem_wait_ld_on(b);
-                tmem_ld32(tS + ((64 * h + 64) & 127), a);     // next chunk; after the last one: chunk 0 again, for the second pass
-                chunk_max(b, 2 * h + 1);
+                for (int e = 0; e < 128; ++e)
+                    if (e > row) v[e] = 0xff800000u;
             }
-            const float m_new = fmaxf(m_run, fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale_log2);
+            float mx[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                mx[q] = fmaxf(__uint_as_float(v[16 * q]), __uint_as_float(v[16 * q + 1]));
+#pragma unroll
+                for (int e = 2; e < 16; e += 2) mx[q] = max3(mx[q], __uint_as_float(v[16 * q + e]), __uint_as_float(v[16 * q + e + 1]));
+            }
+            const float mx_all = fmaxf(max3(mx[0], mx[1], mx[2]), max3(mx[3], mx[4], max3(mx[5], mx[6], mx[7])));
+            const float m_new = fmaxf(m_run, mx_all * p.scale_log2);
             // raise the running maximum only when it moved a lot; p may then exceed 1 (up to 2^8), which is harmless
             const bool raise = (m_new - m_run) > LAZY_RESCALE_LOG2;      // true on the first tile (m_run = -inf)
             const float factor = raise ? fast_exp2(m_run - m_new) : 1.f;
             if (raise) m_run = m_new;
             if (j > 0 && __any_sync(0xffffffffu, raise)) {
+                uint32_t o[32];
 #pragma unroll 1
                 for (int c = 0; c < D / 32; ++c) {
-                    tmem_ld32(tO + c * 32, b);
-                    tmem_wait_ld_on(b);
+                    tmem_ld32(tO + c * 32, o);
+                    tmem_wait_ld();
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) b[e] = __float_as_uint(__uint_as_float(b[e]) * factor);
-                    tmem_st32(tO + c * 32, b);
+                    for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * factor);
+                    tmem_st32(tO + c * 32, o);
                 }
             }
             const float2 nm2 = make_float2(-m_run, -m_run);
             float2 sum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-            auto chunk_exp = [&](const uint32_t (&r)[32], int c) {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
                 uint32_t pk16[16];
-                const int lim = diag ? row - 32 * c : 32;
 #pragma unroll
                 for (int e2 = 0; e2 < 16; ++e2) {
-                    const float2 arg = __ffma2_rn(make_float2(__uint_as_float(r[2 * e2]), __uint_as_float(r[2 * e2 + 1])), sc2, nm2);
+                    const int e = 32 * c + 2 * e2;
+                    const float2 arg = __ffma2_rn(make_float2(__uint_as_float(v[e]), __uint_as_float(v[e + 1])), sc2, nm2);
                     float2 pe;
                     if ((POLY_PAIR_MASK >> e2) & 1u) {
                         pe = exp2_poly2(arg);
@@ -508,29 +510,16 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                         pe.x = fast_exp2(arg.x);
                         pe.y = fast_exp2(arg.y);
                     }
-                    if (diag) {
-                        if (2 * e2 > lim) pe.x = 0.f;
-                        if (2 * e2 + 1 > lim) pe.y = 0.f;
-                    }
                     sum[e2 & 1] = __fadd2_rn(sum[e2 & 1], pe);
                     pk16[e2] = pack_bf16(pe.x, pe.y);
                 }
-                tmem_st16(tS + c * 16, pk16);     // P (bf16 pairs) over score columns that have been consumed
-            };
-#pragma unroll 1
-            for (int h = 0; h < 2; ++h) {
-                tmem_wait_ld_on(a);
-                tmem_ld32(tS + 64 * h + 32, b);
-                chunk_exp(a, 2 * h);
-                if (h == 1) {                     // keys 0-95 are in place: the tensor core may start on them
+                tmem_st16(tS + c * 16, pk16);     // P (bf16 pairs) over score columns that are already in registers
+                if (c == 2) {                     // keys 0-95 are in place: the tensor core may start on them
                     tmem_wait_st();
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(p_full + x);
                 }
-                tmem_wait_ld_on(b);
-                if (h == 0) tmem_ld32(tS + 64, a);
-                chunk_exp(b, 2 * h + 1);
             }
             tmem_wait_st();
             tc_fence_before();
