@@ -48,7 +48,6 @@ struct AttnParams {
 };
 
 constexpr int BM = 128, BN = 128;
-constexpr int NV = 2;                       // V ring depth
 constexpr int NTHREADS = 512;
 constexpr int MAX_HOT_SMEM = 1024;          // per-tile highlight flags kept in shared memory (longer sequences read global memory)
 constexpr uint32_t BLK_BYTES = 128 * 128;   // one [128 x 64] bf16 block
@@ -60,17 +59,17 @@ constexpr uint32_t POLY_PAIR_MASK = SEKA_POLY_PAIR_MASK;
 
 template <int D>
 struct SmemLayout {
-    // K ring depth: head_dim 128 leaves room for two stages beside the 32 KB edit operator, head_dim 64 for three
+    // K and V ring depth: head_dim 128 leaves room for two stages beside the 32 KB edit operator, head_dim 64 for three
     static constexpr int NK = D == 128 ? 2 : 3;
     static constexpr uint32_t TILE = (D / 64) * BLK_BYTES;
     static constexpr uint32_t WBLK = D * 128;              // one [D x 64] block of W
     static constexpr uint32_t Q = 0;                       // 2 tiles
     static constexpr uint32_t K = Q + 2 * TILE;            // NK stages
-    static constexpr uint32_t V = K + NK * TILE;           // NV stages
-    static constexpr uint32_t W = V + NV * TILE;           // D x D bf16
+    static constexpr uint32_t V = K + NK * TILE;           // NK stages
+    static constexpr uint32_t W = V + NK * TILE;           // D x D bf16
     static constexpr uint32_t HOT = W + (D / 64) * WBLK;   // MAX_HOT_SMEM bytes
     static constexpr uint32_t BARS = HOT + MAX_HOT_SMEM;   // mbarriers
-    static constexpr uint32_t NBARS = 2 + 2 * NK + 2 * NV + 8 + 3;
+    static constexpr uint32_t NBARS = 3 + 2 * NK + 8 + 3;
     static constexpr uint32_t MISC = BARS + NBARS * 8;     // tmem holder, abort flag
     static constexpr uint32_t TOTAL = MISC + 16;
     static constexpr uint32_t DYN_BYTES = TOTAL + 1024;    // slack for the 1024-byte alignment
@@ -154,11 +153,10 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     uint8_t* hot = smem + SL::HOT;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SL::BARS);
     uint64_t* q_full = bars;                 // [2]   TMA bytes landed
-    uint64_t* k_full = q_full + 2;           // [NK]  TMA bytes landed
-    uint64_t* k_empty = k_full + NK;         // [NK]  tensor core finished reading the stage
-    uint64_t* v_full = k_empty + NK;         // [NV]
-    uint64_t* v_empty = v_full + NV;         // [NV]
-    uint64_t* s_full = v_empty + NV;         // [2]   scores of tile x are in tensor memory
+    uint64_t* k0_full = q_full + 2;          // [1]   first key tile landed
+    uint64_t* kv_full = k0_full + 1;         // [NK]  slot t % NK: V(t) and K(t+1) landed (they are loaded as a pair)
+    uint64_t* kv_free = kv_full + NK;        // [NK]  slot i % NK: the tensor core is done with K(i) and V(i-1)
+    uint64_t* s_full = kv_free + NK;         // [2]   scores of tile x are in tensor memory
     uint64_t* p_full = s_full + 2;           // [2]   4 softmax-warp arrivals (O_x rescaled, keys 0-95 of P_x written) + 1 from the operand relay
     uint64_t* p_last = p_full + 2;           // [2]   4 softmax-warp arrivals: keys 96-127 of P_x written
     uint64_t* o_full = p_last + 2;           // [2]   last P V of tile x finished
@@ -201,8 +199,8 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 
     if (tid == 0) {
         mbar_init(q_full + 0, 1); mbar_init(q_full + 1, 1);
-        for (int i = 0; i < NK; ++i) { mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1); }
-        for (int i = 0; i < NV; ++i) { mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1); }
+        mbar_init(k0_full, 1);
+        for (int i = 0; i < NK; ++i) { mbar_init(kv_full + i, 1); mbar_init(kv_free + i, 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(s_full + i, 1); mbar_init(p_full + i, 5); mbar_init(p_last + i, 4); mbar_init(o_full + i, 1); }
         mbar_init(w_full, 1); mbar_init(e_full, 1); mbar_init(k_edited, 4);
         *abort_flag = 0;
@@ -241,6 +239,10 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     for (int c = 0; c < NBLK; ++c)
                         tma_load_3d(smem + SL::Q + SL::TILE + c * BLK_BYTES, &tmQ, q_full + 1, c * 64, tw[1].hq, seq0 + tw[1].qt * BM);
                 }
+                mbar_expect_tx(k0_full, SL::TILE);
+#pragma unroll
+                for (int c = 0; c < NBLK; ++c)
+                    tma_load_3d(smem + SL::K + c * BLK_BYTES, &tmK, k0_full, c * 64, hkv, seq0);
                 if (steer) {
                     mbar_expect_tx(w_full, NBLK * SL::WBLK);
 #pragma unroll
@@ -249,23 +251,24 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                 }
             }
             __syncwarp();
+            // V(t) and K(t+1) travel as a pair: both of their stages are released by the same event, the end of
+            // step t - NK of the MMA issuer (kv_free slot (t - NK + 1) % NK).
 #pragma unroll 1
-            for (int j = 0; j < n_kv; ++j) {
-                const int sk = j % NK, uk = j / NK, sv = j % NV, uv = j / NV;
-                if (uk > 0 && !warp_wait(k_empty + sk, (uint32_t)((uk - 1) & 1), abort_flag, p.status, 10)) break;
+            for (int t = 0; t < n_kv; ++t) {
+                const int i = t - NK + 1;
+                if (i >= 0 && !warp_wait(kv_free + i % NK, (uint32_t)((i / NK) & 1), abort_flag, p.status, 10)) break;
                 if (leader) {
-                    mbar_expect_tx(k_full + sk, SL::TILE);
+                    const bool more = t + 1 < n_kv;
+                    mbar_expect_tx(kv_full + t % NK, more ? 2 * SL::TILE : SL::TILE);
 #pragma unroll
                     for (int c = 0; c < NBLK; ++c)
-                        tma_load_3d(smem + SL::K + sk * SL::TILE + c * BLK_BYTES, &tmK, k_full + sk, c * 64, hkv, seq0 + j * BN);
-                }
-                __syncwarp();
-                if (uv > 0 && !warp_wait(v_empty + sv, (uint32_t)((uv - 1) & 1), abort_flag, p.status, 11)) break;
-                if (leader) {
-                    mbar_expect_tx(v_full + sv, SL::TILE);
+                        tma_load_3d(smem + SL::V + (t % NK) * SL::TILE + c * BLK_BYTES, &tmV, kv_full + t % NK, c * 64, hkv, seq0 + t * BN);
+                    if (more) {
 #pragma unroll
-                    for (int c = 0; c < NBLK; ++c)
-                        tma_load_3d(smem + SL::V + sv * SL::TILE + c * BLK_BYTES, &tmV, v_full + sv, c * 64, hkv, seq0 + j * BN);
+                        for (int c = 0; c < NBLK; ++c)
+                            tma_load_3d(smem + SL::K + ((t + 1) % NK) * SL::TILE + c * BLK_BYTES, &tmK, kv_full + t % NK, c * 64, hkv,
+                                        seq0 + (t + 1) * BN);
+                    }
                 }
                 __syncwarp();
             }
@@ -324,7 +327,7 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             };
             // P V of tile x and key tile j, key blocks [ks0, ks1) of 16 keys (2048 bytes of the V tile, 8 columns of P)
             auto issue_PV = [&](int x, int j, int ks0, int ks1, bool last) {
-                const uint32_t vd = dV + (uint32_t)(j % NV) * (SL::TILE >> 4);
+                const uint32_t vd = dV + (uint32_t)(j % NK) * (SL::TILE >> 4);
                 const uint32_t dst = tmem_base + COL_O + D * x, src = tmem_base + COL_S + 128 * x;
                 tc_fence_after();
                 if (leader) {
@@ -341,16 +344,16 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             // tiles half a period apart (softmax of one tile under the MMAs of the other).
             ok = warp_wait(q_full + 0, 0, abort_flag, p.status, 20);
             if (ok && nB > 0) ok = warp_wait(q_full + 1, 0, abort_flag, p.status, 21);
-            if (ok) ok = warp_wait(k_full + 0, 0, abort_flag, p.status, 22);
+            if (ok) ok = warp_wait(k0_full, 0, abort_flag, p.status, 22);
             if (ok) edit_K(0, 0);
             if (ok) {
                 issue_S(0, 0);
                 if (nB > 0) issue_S(1, 0);
-                commit(k_empty + 0);
+                commit(kv_free + 0);
             }
 #pragma unroll 1
             for (int j = 0; j < n_kv && ok; ++j) {
-                const int sv = j % NV, j1 = j + 1, sk1 = j1 % NK;
+                const int j1 = j + 1;
                 // V of this step and K of the next have landed once p_full completes: the relay warp vouches for
                 // them there, so this warp has no waits of its own for operands (every wait here is a bubble in
                 // the tensor pipe: its queue is only a couple of MMAs deep)
@@ -375,21 +378,19 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     if (!ok) break;
                     issue_PV(1, j, 6, 8, j == nB - 1);
                 }
-                commit(v_empty + sv);
                 if (j1 < nB) {
                     if (j1 >= nA) edit_K(1, j1);      // tile A does not use this key tile: B is its first user
                     if (!ok) break;
                     issue_S(1, j1);
                 }
-                if (j1 < n_kv) commit(k_empty + sk1);
+                commit(kv_free + j1 % NK);      // K(j+1) and V(j) may be overwritten
             }
         } else if (warp == 2) {
             // ------------------------------------------------------------ operand relay: "V(j) and K(j+1) have landed" as a
             // fifth arrival on p_full of step j, so that the MMA issuer waits on one barrier per hand-off
 #pragma unroll 1
             for (int j = 0; j < n_kv; ++j) {
-                if (!warp_wait(v_full + j % NV, (uint32_t)((j / NV) & 1), abort_flag, p.status, 23)) break;
-                if (j + 1 < n_kv && !warp_wait(k_full + (j + 1) % NK, (uint32_t)(((j + 1) / NK) & 1), abort_flag, p.status, 25)) break;
+                if (!warp_wait(kv_full + j % NK, (uint32_t)((j / NK) & 1), abort_flag, p.status, 23)) break;
                 if (lane == 0) {
                     if (j < nA) mbar_arrive(p_full + 0);
                     if (j < nB) mbar_arrive(p_full + 1);
@@ -552,7 +553,7 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         if (*abort_flag && lane == 0) {
             // let tile loads that may still be in flight land before the shared memory is released
             int dummy = 0;
-            for (int i = 0; i < NK; ++i) { mbar_wait(k_full + i, 0, &dummy, nullptr, 0); }
+            for (int i = 0; i < NK; ++i) { mbar_wait(kv_full + i, 0, &dummy, nullptr, 0); }
         }
         __syncwarp();
         tmem_dealloc(tmem_base, TMEM_COLS);
