@@ -42,6 +42,7 @@ struct AttnParams {
     const uint8_t* tile_hot;      // [B, n_qt]: key tile holds a highlighted token
     int* status;
     int B, L, Hq, Hkv, n_qt;
+    long long n_items;    // work items (pairs of query tiles) of the launch
     int steer;
     int pair_heads;       // 1: the two tiles of a CTA are two query heads of one KV group; 0: two consecutive query tiles
     float scale_log2;
@@ -49,7 +50,6 @@ struct AttnParams {
 
 constexpr int BM = 128, BN = 128;
 constexpr int NTHREADS = 512;
-constexpr int MAX_HOT_SMEM = 1024;          // per-tile highlight flags kept in shared memory (longer sequences read global memory)
 constexpr uint32_t BLK_BYTES = 128 * 128;   // one [128 x 64] bf16 block
 constexpr float LAZY_RESCALE_LOG2 = 8.0f;   // the running maximum is only raised when it moved by more than this
 // registers per thread after the roles split (the CTA owns the whole register file: 4 x 128 x (56+184+184+88) = 64 Ki)
@@ -67,8 +67,7 @@ struct SmemLayout {
     static constexpr uint32_t K = Q + 2 * TILE;            // NK stages
     static constexpr uint32_t V = K + NK * TILE;           // NK stages
     static constexpr uint32_t W = V + NK * TILE;           // D x D bf16
-    static constexpr uint32_t HOT = W + (D / 64) * WBLK;   // MAX_HOT_SMEM bytes
-    static constexpr uint32_t BARS = HOT + MAX_HOT_SMEM;   // mbarriers
+    static constexpr uint32_t BARS = W + (D / 64) * WBLK;  // mbarriers
     static constexpr uint32_t NBARS = 3 + 2 * NK + 8 + 3;
     static constexpr uint32_t MISC = BARS + NBARS * 8;     // tmem holder, abort flag
     static constexpr uint32_t TOTAL = MISC + 16;
@@ -138,6 +137,14 @@ template <> __device__ __forceinline__ void store_chunk32<float>(float* dst, con
                             __uint_as_float(v[4 * c + 2]) * inv, __uint_as_float(v[4 * c + 3]) * inv);
 }
 
+// One unit of work of a CTA: two 128-row query tiles that share a KV head of one sequence.
+struct Item {
+    int b, hkv, seq0, Lb;
+    int hqA, hqB, qtA, qtB;     // query head and row-tile index of tile A / B
+    int nA, nB, n_kv;           // key tiles of A / B (0: the tile lies beyond the sequence) and of the item
+    bool steer;
+};
+
 template <int D, typename OutT>
 __global__ void __launch_bounds__(NTHREADS, 1)
 seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -150,12 +157,11 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     constexpr uint32_t COL_S = 0, COL_O = 256;     // S_x at COL_S + 128 x, O_x at COL_O + D x
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t* hot = smem + SL::HOT;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SL::BARS);
     uint64_t* q_full = bars;                 // [2]   TMA bytes landed
-    uint64_t* k0_full = q_full + 2;          // [1]   first key tile landed
-    uint64_t* kv_full = k0_full + 1;         // [NK]  slot t % NK: V(t) and K(t+1) landed (they are loaded as a pair)
-    uint64_t* kv_free = kv_full + NK;        // [NK]  slot i % NK: the tensor core is done with K(i) and V(i-1)
+    uint64_t* k0_full = q_full + 2;          // [1]   first key tile of the item landed
+    uint64_t* kv_full = k0_full + 1;         // [NK]  V(t) and K(t+1) landed (they are loaded as a pair)
+    uint64_t* kv_free = kv_full + NK;        // [NK]  one event per step: the tensor core is done with K(j+1) and V(j)
     uint64_t* s_full = kv_free + NK;         // [2]   scores of tile x are in tensor memory
     uint64_t* p_full = s_full + 2;           // [2]   4 softmax-warp arrivals (O_x rescaled, keys 0-95 of P_x written) + 1 from the operand relay
     uint64_t* p_last = p_full + 2;           // [2]   4 softmax-warp arrivals: keys 96-127 of P_x written
@@ -167,39 +173,47 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + SL::MISC + 4);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // an earlier launch (or CTA) gave up on this workspace: all threads agree on leaving
+    if (__syncthreads_or(*reinterpret_cast<volatile int*>(p.status) != 0)) return;
 
-    // work of this CTA: heaviest query tiles first; CTAs of one (sequence, KV head) are neighbours
-    TileWork tw[2];
-    int b;
-    if (p.pair_heads) {
-        const int per_qt = p.B * (p.Hq >> 1);
-        const int qt = p.n_qt - 1 - (int)(blockIdx.x / per_qt);
-        const int rem = (int)(blockIdx.x % per_qt);
-        b = rem / (p.Hq >> 1);
-        const int hp = rem % (p.Hq >> 1);
-        tw[0].hq = 2 * hp; tw[1].hq = 2 * hp + 1;
-        tw[0].qt = tw[1].qt = qt;
-    } else {
-        const int per_qt = p.B * p.Hq;
-        const int qt2 = ((p.n_qt + 1) >> 1) - 1 - (int)(blockIdx.x / per_qt);
-        const int rem = (int)(blockIdx.x % per_qt);
-        b = rem / p.Hq;
-        tw[0].hq = tw[1].hq = rem % p.Hq;
-        tw[0].qt = 2 * qt2; tw[1].qt = 2 * qt2 + 1;
-    }
-    const int hkv = tw[0].hq / (p.Hq / p.Hkv);
-    const int seq0 = p.cu_seqlens ? p.cu_seqlens[b] : b * p.L;
-    const int Lb = p.cu_seqlens ? (p.cu_seqlens[b + 1] - seq0) : p.L;
-    tw[0].n = tw[0].qt * BM < Lb ? tw[0].qt + 1 : 0;
-    tw[1].n = tw[1].qt * BM < Lb ? tw[1].qt + 1 : 0;
-    const int nA = tw[0].n, nB = tw[1].n;
-    if (nA == 0) return;                                               // nothing allocated yet (tile B starts no earlier)
-    if (*reinterpret_cast<volatile int*>(p.status) != 0) return;      // an earlier CTA gave up: do not pile on
-    const int n_kv = max(nA, nB);
+    // The CTA is persistent: it walks its share of the items (heaviest first; odd rounds run the CTAs in
+    // reverse so that the shares come out even).  Every role decodes the same sequence of items by itself.
+    auto next_item = [&](int& round, Item& it) -> bool {
+        while (true) {
+            const long long G = gridDim.x;
+            const long long idx = (long long)round * G + ((round & 1) ? (G - 1 - blockIdx.x) : blockIdx.x);
+            ++round;
+            if (idx >= p.n_items) return false;
+            if (p.pair_heads) {
+                const int per_qt = p.B * (p.Hq >> 1);
+                const int qt = p.n_qt - 1 - (int)(idx / per_qt);
+                const int rem = (int)(idx % per_qt);
+                it.b = rem / (p.Hq >> 1);
+                const int hp = rem % (p.Hq >> 1);
+                it.hqA = 2 * hp; it.hqB = 2 * hp + 1;
+                it.qtA = it.qtB = qt;
+            } else {
+                const int per_qt = p.B * p.Hq;
+                const int qt2 = ((p.n_qt + 1) >> 1) - 1 - (int)(idx / per_qt);
+                const int rem = (int)(idx % per_qt);
+                it.b = rem / p.Hq;
+                it.hqA = it.hqB = rem % p.Hq;
+                it.qtA = 2 * qt2; it.qtB = 2 * qt2 + 1;
+            }
+            it.hkv = it.hqA / (p.Hq / p.Hkv);
+            it.seq0 = p.cu_seqlens ? p.cu_seqlens[it.b] : it.b * p.L;
+            it.Lb = p.cu_seqlens ? (p.cu_seqlens[it.b + 1] - it.seq0) : p.L;
+            it.nA = it.qtA * BM < it.Lb ? it.qtA + 1 : 0;
+            it.nB = it.qtB * BM < it.Lb ? it.qtB + 1 : 0;
+            if (it.nA == 0) continue;                       // beyond the sequence (tile B starts no earlier)
+            it.n_kv = max(it.nA, it.nB);
+            it.steer = p.steer && p.gain[it.b] != 0.f && (p.head_enable == nullptr || p.head_enable[it.hkv] != 0);
+            return true;
+        }
+    };
 
     if (tid == 0) {
-        mbar_init(q_full + 0, 1); mbar_init(q_full + 1, 1);
-        mbar_init(k0_full, 1);
+        mbar_init(q_full + 0, 1); mbar_init(q_full + 1, 1); mbar_init(k0_full, 1);
         for (int i = 0; i < NK; ++i) { mbar_init(kv_full + i, 1); mbar_init(kv_free + i, 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(s_full + i, 1); mbar_init(p_full + i, 5); mbar_init(p_last + i, 4); mbar_init(o_full + i, 1); }
         mbar_init(w_full, 1); mbar_init(e_full, 1); mbar_init(k_edited, 4);
@@ -209,69 +223,93 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     }
     __syncwarp();
     if (warp == 0) { tmem_alloc(tmem_holder, TMEM_COLS); tmem_relinquish(); }
-
-    // steering of this (sequence, KV head): which of its key tiles hold highlighted tokens
-    const bool steer = p.steer && p.gain[b] != 0.f && (p.head_enable == nullptr || p.head_enable[hkv] != 0);
-    const uint8_t* hot_g = p.tile_hot + (size_t)b * p.n_qt;
-    if (steer)
-        for (int i = tid; i < min(n_kv, MAX_HOT_SMEM); i += NTHREADS) hot[i] = hot_g[i];
-    auto tile_is_hot = [&](int j) -> bool { return steer && (j < MAX_HOT_SMEM ? hot[j] : hot_g[j]) != 0; };
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_holder;
 
+    // Running counts shared by all roles (each keeps its own copy; they advance identically):
+    //   ev   kv_free events so far (n_kv + 1 per item: after the first score products, then after every step)
+    //   pr   V/K pairs so far (n_kv per item); pair t of an item uses V stage (pr + t) % NK and K stage (pr + t + 1) % NK
+    //   cA/cB  steps of tile A / B so far (phases of s_full, p_full, p_last)
+    Item it;
+    int round = 0;
+
     if (warp < 4) {
         reg_dec<REGS_CTRL>();
-        // Both control warps run their loops with all 32 lanes and elect one lane only around the issuing
+        // The control warps run their loops with all 32 lanes and elect one lane only around the issuing
         // instructions: addresses, descriptors and barrier phases then stay warp-uniform values.
         const bool leader = elect_one();
         if (warp == 0) {
             // ------------------------------------------------------------ TMA producer
-            if (leader) {
-                mbar_expect_tx(q_full + 0, SL::TILE);
-#pragma unroll
-                for (int c = 0; c < NBLK; ++c)
-                    tma_load_3d(smem + SL::Q + c * BLK_BYTES, &tmQ, q_full + 0, c * 64, tw[0].hq, seq0 + tw[0].qt * BM);
-                if (nB > 0) {
-                    mbar_expect_tx(q_full + 1, SL::TILE);
-#pragma unroll
-                    for (int c = 0; c < NBLK; ++c)
-                        tma_load_3d(smem + SL::Q + SL::TILE + c * BLK_BYTES, &tmQ, q_full + 1, c * 64, tw[1].hq, seq0 + tw[1].qt * BM);
+            uint32_t ev = 0, pr = 0, n_it = 0, n_qb = 0;
+            int prev_n = 0;
+            bool ok = true;
+            while (ok && next_item(round, it)) {
+                // Q, W and the first K of an item may land once the last score product of the previous item is
+                // done (event n_kv - 1 of that item), its V/K pairs once its last step is done (event n_kv)
+                if (n_it > 0) {
+                    const uint32_t e = ev - 2;
+                    ok = warp_wait(kv_free + e % NK, (e / NK) & 1, abort_flag, p.status, 12);
+                    if (!ok) break;
                 }
-                mbar_expect_tx(k0_full, SL::TILE);
-#pragma unroll
-                for (int c = 0; c < NBLK; ++c)
-                    tma_load_3d(smem + SL::K + c * BLK_BYTES, &tmK, k0_full, c * 64, hkv, seq0);
-                if (steer) {
-                    mbar_expect_tx(w_full, NBLK * SL::WBLK);
-#pragma unroll
-                    for (int c = 0; c < NBLK; ++c)
-                        tma_load_3d(smem + SL::W + c * SL::WBLK, &tmW, w_full, c * 64, 0, (b * p.Hkv + hkv) * D);
-                }
-            }
-            __syncwarp();
-            // V(t) and K(t+1) travel as a pair: both of their stages are released by the same event, the end of
-            // step t - NK of the MMA issuer (kv_free slot (t - NK + 1) % NK).
-#pragma unroll 1
-            for (int t = 0; t < n_kv; ++t) {
-                const int i = t - NK + 1;
-                if (i >= 0 && !warp_wait(kv_free + i % NK, (uint32_t)((i / NK) & 1), abort_flag, p.status, 10)) break;
                 if (leader) {
-                    const bool more = t + 1 < n_kv;
-                    mbar_expect_tx(kv_full + t % NK, more ? 2 * SL::TILE : SL::TILE);
+                    mbar_expect_tx(q_full + 0, SL::TILE);
 #pragma unroll
                     for (int c = 0; c < NBLK; ++c)
-                        tma_load_3d(smem + SL::V + (t % NK) * SL::TILE + c * BLK_BYTES, &tmV, kv_full + t % NK, c * 64, hkv, seq0 + t * BN);
-                    if (more) {
+                        tma_load_3d(smem + SL::Q + c * BLK_BYTES, &tmQ, q_full + 0, c * 64, it.hqA, it.seq0 + it.qtA * BM);
+                    if (it.nB > 0) {
+                        mbar_expect_tx(q_full + 1, SL::TILE);
 #pragma unroll
                         for (int c = 0; c < NBLK; ++c)
-                            tma_load_3d(smem + SL::K + ((t + 1) % NK) * SL::TILE + c * BLK_BYTES, &tmK, kv_full + t % NK, c * 64, hkv,
-                                        seq0 + (t + 1) * BN);
+                            tma_load_3d(smem + SL::Q + SL::TILE + c * BLK_BYTES, &tmQ, q_full + 1, c * 64, it.hqB, it.seq0 + it.qtB * BM);
+                    }
+                    mbar_expect_tx(k0_full, SL::TILE);
+#pragma unroll
+                    for (int c = 0; c < NBLK; ++c)
+                        tma_load_3d(smem + SL::K + (pr % NK) * SL::TILE + c * BLK_BYTES, &tmK, k0_full, c * 64, it.hkv, it.seq0);
+                    if (it.steer) {
+                        mbar_expect_tx(w_full, NBLK * SL::WBLK);
+#pragma unroll
+                        for (int c = 0; c < NBLK; ++c)
+                            tma_load_3d(smem + SL::W + c * SL::WBLK, &tmW, w_full, c * 64, 0, (it.b * p.Hkv + it.hkv) * D);
                     }
                 }
                 __syncwarp();
+                if (n_it > 0) {
+                    const uint32_t e = ev - 1;
+                    ok = warp_wait(kv_free + e % NK, (e / NK) & 1, abort_flag, p.status, 13);
+                    if (!ok) break;
+                }
+                // V(t) and K(t+1) travel as a pair: both of their stages are released by the same event, the end
+                // of step t - NK of the MMA issuer (event t - NK + 1 of this item)
+#pragma unroll 1
+                for (int t = 0; t < it.n_kv; ++t) {
+                    if (t >= NK - 1) {
+                        const uint32_t e = ev + (uint32_t)(t - NK + 1);
+                        ok = warp_wait(kv_free + e % NK, (e / NK) & 1, abort_flag, p.status, 10);
+                        if (!ok) break;
+                    }
+                    if (leader) {
+                        const bool more = t + 1 < it.n_kv;
+                        uint64_t* bar = kv_full + (pr + t) % NK;
+                        mbar_expect_tx(bar, more ? 2 * SL::TILE : SL::TILE);
+#pragma unroll
+                        for (int c = 0; c < NBLK; ++c)
+                            tma_load_3d(smem + SL::V + ((pr + t) % NK) * SL::TILE + c * BLK_BYTES, &tmV, bar, c * 64, it.hkv, it.seq0 + t * BN);
+                        if (more) {
+#pragma unroll
+                            for (int c = 0; c < NBLK; ++c)
+                                tma_load_3d(smem + SL::K + ((pr + t + 1) % NK) * SL::TILE + c * BLK_BYTES, &tmK, bar, c * 64, it.hkv,
+                                            it.seq0 + (t + 1) * BN);
+                        }
+                    }
+                    __syncwarp();
+                }
+                ev += it.n_kv + 1; pr += it.n_kv; ++n_it; prev_n = it.n_kv;
+                if (it.nB > 0) ++n_qb;
             }
+            (void)prev_n; (void)n_qb;
         } else if (warp == 1) {
             // ------------------------------------------------------------ MMA issuer
             constexpr uint32_t IDESC_S = umma_idesc_bf16(BN, false);
@@ -281,269 +319,315 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             const uint32_t dQ = umma_desc_lo(smem_u32(smem + SL::Q), 16), dK = umma_desc_lo(smem_u32(smem + SL::K), 16);
             const uint32_t dV = umma_desc_lo(smem_u32(smem + SL::V), BLK_BYTES);
             const uint32_t dW = umma_desc_lo(smem_u32(smem + SL::W), 16);
-            int n_hot = 0;          // highlighted tiles edited so far (phase of e_full / k_edited)
+            uint32_t ev = 0, pr = 0, n_it = 0, n_qb = 0, n_w = 0, n_ob[2] = {0, 0};
+            uint32_t cx[2] = {0, 0};      // steps of tile A / B so far
+            uint32_t n_hot = 0;           // highlighted tiles edited so far (phase of e_full / k_edited)
             bool ok = true;
             auto commit = [&](uint64_t* bar) {
                 if (leader) umma_commit(bar);
                 __syncwarp();
             };
-            // Before the first score product of key tile j (by tile x): if the tile holds highlighted tokens,
-            // dK = K W goes into the score columns of tile x (idle between P_x V and the next S_x), the editors
-            // add it to the staged tile, and only then may the tile be multiplied.
-            auto edit_K = [&](int x, int j) {
-                if (!tile_is_hot(j)) return;
-                if (n_hot == 0) ok = warp_wait(w_full, 0, abort_flag, p.status, 31);
-                if (!ok) return;
-                const uint32_t kd = dK + (uint32_t)(j % NK) * (SL::TILE >> 4);
-                const uint32_t dst = tmem_base + COL_S + 128 * x;
-                tc_fence_after();
-                if (leader) {
+            while (ok && next_item(round, it)) {
+                const uint8_t* hot_g = p.tile_hot + (size_t)it.b * p.n_qt;
+                bool w_seen = false;
+                // Before the first score product of key tile j (by tile x): if the tile holds highlighted tokens,
+                // dK = K W goes into the score columns of tile x (idle between P_x V and the next S_x), the editors
+                // add it to the staged tile, and only then may the tile be multiplied.
+                auto edit_K = [&](int x, int j, bool is_hot) {
+                    if (!is_hot) return;
+                    if (!w_seen) { ok = warp_wait(w_full, n_w & 1, abort_flag, p.status, 31); w_seen = true; }
+                    if (!ok) return;
+                    const uint32_t kd = dK + ((pr + (uint32_t)j) % NK) * (SL::TILE >> 4);
+                    const uint32_t dst = tmem_base + COL_S + 128 * x;
+                    tc_fence_after();
+                    if (leader) {
 #pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks) {
-                        const uint32_t offk = ((uint32_t)(ks >> 2) * BLK_BYTES + (uint32_t)(ks & 3) * 32) >> 4;
-                        const uint32_t offw = ((uint32_t)(ks >> 2) * SL::WBLK + (uint32_t)(ks & 3) * 32) >> 4;
-                        umma_ss(dst, kd + offk, DESC_HI, dW + offw, DESC_HI, IDESC_E, ks > 0 ? 1u : 0u);
+                        for (int ks = 0; ks < D / 16; ++ks) {
+                            const uint32_t offk = ((uint32_t)(ks >> 2) * BLK_BYTES + (uint32_t)(ks & 3) * 32) >> 4;
+                            const uint32_t offw = ((uint32_t)(ks >> 2) * SL::WBLK + (uint32_t)(ks & 3) * 32) >> 4;
+                            umma_ss(dst, kd + offk, DESC_HI, dW + offw, DESC_HI, IDESC_E, ks > 0 ? 1u : 0u);
+                        }
+                        umma_commit(e_full);
                     }
-                    umma_commit(e_full);
-                }
-                __syncwarp();
-                ok = warp_wait(k_edited, (uint32_t)(n_hot & 1), abort_flag, p.status, 32);
-                ++n_hot;
-            };
-            auto issue_S = [&](int x, int j) {
-                const uint32_t kd = dK + (uint32_t)(j % NK) * (SL::TILE >> 4), qd = dQ + (uint32_t)x * (SL::TILE >> 4);
-                const uint32_t dst = tmem_base + COL_S + 128 * x;
-                tc_fence_after();
-                if (leader) {
+                    __syncwarp();
+                    ok = warp_wait(k_edited, n_hot & 1, abort_flag, p.status, 32);
+                    ++n_hot;
+                };
+                auto issue_S = [&](int x, int j) {
+                    const uint32_t kd = dK + ((pr + (uint32_t)j) % NK) * (SL::TILE >> 4), qd = dQ + (uint32_t)x * (SL::TILE >> 4);
+                    const uint32_t dst = tmem_base + COL_S + 128 * x;
+                    tc_fence_after();
+                    if (leader) {
 #pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks) {
-                        // 16 elements along the contraction = 32 bytes inside a 64-element block
-                        const uint32_t off = ((uint32_t)(ks >> 2) * BLK_BYTES + (uint32_t)(ks & 3) * 32) >> 4;
-                        umma_ss(dst, qd + off, DESC_HI, kd + off, DESC_HI, IDESC_S, ks > 0 ? 1u : 0u);
+                        for (int ks = 0; ks < D / 16; ++ks) {
+                            // 16 elements along the contraction = 32 bytes inside a 64-element block
+                            const uint32_t off = ((uint32_t)(ks >> 2) * BLK_BYTES + (uint32_t)(ks & 3) * 32) >> 4;
+                            umma_ss(dst, qd + off, DESC_HI, kd + off, DESC_HI, IDESC_S, ks > 0 ? 1u : 0u);
+                        }
+                        umma_commit(s_full + x);
                     }
-                    umma_commit(s_full + x);
-                }
-                __syncwarp();
-            };
-            // P V of tile x and key tile j, key blocks [ks0, ks1) of 16 keys (2048 bytes of the V tile, 8 columns of P)
-            auto issue_PV = [&](int x, int j, int ks0, int ks1, bool last) {
-                const uint32_t vd = dV + (uint32_t)(j % NK) * (SL::TILE >> 4);
-                const uint32_t dst = tmem_base + COL_O + D * x, src = tmem_base + COL_S + 128 * x;
-                tc_fence_after();
-                if (leader) {
+                    __syncwarp();
+                };
+                // P V of tile x and key tile j, key blocks [ks0, ks1) of 16 keys (2048 bytes of the V tile, 8 columns of P)
+                auto issue_PV = [&](int x, int j, int ks0, int ks1, bool last) {
+                    const uint32_t vd = dV + ((pr + (uint32_t)j) % NK) * (SL::TILE >> 4);
+                    const uint32_t dst = tmem_base + COL_O + D * x, src = tmem_base + COL_S + 128 * x;
+                    tc_fence_after();
+                    if (leader) {
 #pragma unroll
-                    for (int ks = 0; ks < BN / 16; ++ks)
-                        if (ks >= ks0 && ks < ks1)
-                            umma_ts(dst, src + (uint32_t)ks * 8, vd + (uint32_t)ks * (2048 >> 4), DESC_HI, IDESC_PV,
-                                    (j > 0 || ks > 0) ? 1u : 0u);
-                    if (last) umma_commit(o_full + x);
+                        for (int ks = 0; ks < BN / 16; ++ks)
+                            if (ks >= ks0 && ks < ks1)
+                                umma_ts(dst, src + (uint32_t)ks * 8, vd + (uint32_t)ks * (2048 >> 4), DESC_HI, IDESC_PV,
+                                        (j > 0 || ks > 0) ? 1u : 0u);
+                        if (last) umma_commit(o_full + x);
+                    }
+                    __syncwarp();
+                };
+                const int nA = it.nA, nB = it.nB, n_kv = it.n_kv;
+                // highlight flags of key tiles 0 and 1 (later ones are fetched one step ahead of their use)
+                bool hot_cur = it.steer && hot_g[0] != 0;
+                bool hot_nxt = it.steer && n_kv > 1 && hot_g[1] != 0;
+                // One thread issues for both tiles, in a fixed order (A then B in every step): the in-order tensor
+                // pipe then keeps the two tiles half a period apart (softmax of one tile under the MMAs of the other).
+                ok = warp_wait(q_full + 0, n_it & 1, abort_flag, p.status, 20);
+                if (ok && nB > 0) ok = warp_wait(q_full + 1, n_qb & 1, abort_flag, p.status, 21);
+                if (ok) ok = warp_wait(k0_full, n_it & 1, abort_flag, p.status, 22);
+                if (ok) edit_K(0, 0, hot_cur);
+                if (ok) {
+                    issue_S(0, 0);
+                    if (nB > 0) issue_S(1, 0);
+                    // The edit operator of this item is seen here at the latest, before the event that lets the
+                    // producer load the next item's: a barrier that ran two phases ahead of its waiter would
+                    // never look complete to it.
+                    if (it.steer && !w_seen) { ok = warp_wait(w_full, n_w & 1, abort_flag, p.status, 35); w_seen = true; }
+                    commit(kv_free + ev % NK);
+                    ++ev;
                 }
-                __syncwarp();
-            };
-            // One thread issues for both tiles, in a fixed order: the in-order tensor pipe then keeps the two
-            // tiles half a period apart (softmax of one tile under the MMAs of the other).
-            ok = warp_wait(q_full + 0, 0, abort_flag, p.status, 20);
-            if (ok && nB > 0) ok = warp_wait(q_full + 1, 0, abort_flag, p.status, 21);
-            if (ok) ok = warp_wait(k0_full, 0, abort_flag, p.status, 22);
-            if (ok) edit_K(0, 0);
-            if (ok) {
-                issue_S(0, 0);
-                if (nB > 0) issue_S(1, 0);
-                commit(kv_free + 0);
-            }
 #pragma unroll 1
-            for (int j = 0; j < n_kv && ok; ++j) {
-                const int j1 = j + 1;
-                // V of this step and K of the next have landed once p_full completes: the relay warp vouches for
-                // them there, so this warp has no waits of its own for operands (every wait here is a bubble in
-                // the tensor pipe: its queue is only a couple of MMAs deep)
-                if (j < nA) {
-                    ok = warp_wait(p_full + 0, (uint32_t)(j & 1), abort_flag, p.status, 24);
-                    if (!ok) break;
-                    issue_PV(0, j, 0, 6, false);
-                    ok = warp_wait(p_last + 0, (uint32_t)(j & 1), abort_flag, p.status, 28);
-                    if (!ok) break;
-                    issue_PV(0, j, 6, 8, j == nA - 1);
-                    if (j1 < nA) {
-                        edit_K(0, j1);
+                for (int j = 0; j < n_kv && ok; ++j) {
+                    const int j1 = j + 1;
+                    const bool hot_j1 = hot_nxt;
+                    hot_nxt = it.steer && j + 2 < n_kv && hot_g[j + 2] != 0;
+                    // V of this step and K of the next have landed once p_full completes: the relay warp vouches
+                    // for them there, so this warp has no waits of its own for operands (every wait here is a
+                    // bubble in the tensor pipe: its queue is only a couple of MMAs deep)
+                    if (j < nA) {
+                        ok = warp_wait(p_full + 0, (cx[0] + j) & 1, abort_flag, p.status, 24);
                         if (!ok) break;
-                        issue_S(0, j1);
+                        issue_PV(0, j, 0, 6, false);
+                        ok = warp_wait(p_last + 0, (cx[0] + j) & 1, abort_flag, p.status, 28);
+                        if (!ok) break;
+                        issue_PV(0, j, 6, 8, j == nA - 1);
+                        if (j1 < nA) {
+                            edit_K(0, j1, hot_j1);
+                            if (!ok) break;
+                            issue_S(0, j1);
+                        }
                     }
+                    if (j < nB) {
+                        ok = warp_wait(p_full + 1, (cx[1] + j) & 1, abort_flag, p.status, 26);
+                        if (!ok) break;
+                        issue_PV(1, j, 0, 6, false);
+                        ok = warp_wait(p_last + 1, (cx[1] + j) & 1, abort_flag, p.status, 29);
+                        if (!ok) break;
+                        issue_PV(1, j, 6, 8, j == nB - 1);
+                    }
+                    if (j1 < nB) {
+                        if (j1 >= nA) edit_K(1, j1, hot_j1);      // tile A does not use this key tile: B is its first user
+                        if (!ok) break;
+                        issue_S(1, j1);
+                    }
+                    commit(kv_free + ev % NK);      // K(j+1) and V(j) may be overwritten
+                    ++ev;
                 }
-                if (j < nB) {
-                    ok = warp_wait(p_full + 1, (uint32_t)(j & 1), abort_flag, p.status, 26);
-                    if (!ok) break;
-                    issue_PV(1, j, 0, 6, false);
-                    ok = warp_wait(p_last + 1, (uint32_t)(j & 1), abort_flag, p.status, 29);
-                    if (!ok) break;
-                    issue_PV(1, j, 6, 8, j == nB - 1);
-                }
-                if (j1 < nB) {
-                    if (j1 >= nA) edit_K(1, j1);      // tile A does not use this key tile: B is its first user
-                    if (!ok) break;
-                    issue_S(1, j1);
-                }
-                commit(kv_free + j1 % NK);      // K(j+1) and V(j) may be overwritten
+                pr += n_kv; cx[0] += nA; cx[1] += nB; ++n_it;
+                if (nB > 0) ++n_qb;
+                if (it.steer) ++n_w;
             }
+            (void)n_ob;
         } else if (warp == 2) {
             // ------------------------------------------------------------ operand relay: "V(j) and K(j+1) have landed" as a
             // fifth arrival on p_full of step j, so that the MMA issuer waits on one barrier per hand-off
+            uint32_t pr = 0, cx[2] = {0, 0};
+            bool ok = true;
+            while (ok && next_item(round, it)) {
 #pragma unroll 1
-            for (int j = 0; j < n_kv; ++j) {
-                if (!warp_wait(kv_full + j % NK, (uint32_t)((j / NK) & 1), abort_flag, p.status, 23)) break;
-                if (lane == 0) {
-                    if (j < nA) mbar_arrive(p_full + 0);
-                    if (j < nB) mbar_arrive(p_full + 1);
+                for (int j = 0; j < it.n_kv; ++j) {
+                    const uint32_t g = pr + j;
+                    ok = warp_wait(kv_full + g % NK, (g / NK) & 1, abort_flag, p.status, 23);
+                    if (!ok) break;
+                    if (lane == 0) {
+                        if (j < it.nA) mbar_arrive(p_full + 0);
+                        if (j < it.nB) mbar_arrive(p_full + 1);
+                    }
+                    __syncwarp();
+                    // stay within the phase: the next arrival may only come after this phase has completed
+                    if (j < it.nA) ok = warp_wait(p_full + 0, (cx[0] + j) & 1, abort_flag, p.status, 33);
+                    if (ok && j < it.nB) ok = warp_wait(p_full + 1, (cx[1] + j) & 1, abort_flag, p.status, 34);
+                    if (!ok) break;
                 }
-                __syncwarp();
-                // stay within the phase: the next arrival may only come after this phase has completed
-                if (j < nA && !warp_wait(p_full + 0, (uint32_t)(j & 1), abort_flag, p.status, 33)) break;
-                if (j < nB && !warp_wait(p_full + 1, (uint32_t)(j & 1), abort_flag, p.status, 34)) break;
+                pr += it.n_kv; cx[0] += it.nA; cx[1] += it.nB;
             }
         }
     } else if (warp >= 12) {
         // ------------------------------------------------------------ key editors: one key row of the staged tile per thread
         reg_dec<REGS_EDIT>();
-        if (steer) {
-            const int row = (warp - 12) * 32 + lane;
-            const uint32_t t_lane = tmem_base + ((uint32_t)((warp - 12) * 32) << 16);
-            int n_hot = 0;
+        const int row = (warp - 12) * 32 + lane;
+        const uint32_t t_lane = tmem_base + ((uint32_t)((warp - 12) * 32) << 16);
+        uint32_t pr = 0, n_hot = 0;
+        bool ok = true;
+        while (ok && next_item(round, it)) {
+            if (it.steer) {
+                const uint8_t* hot_g = p.tile_hot + (size_t)it.b * p.n_qt;
 #pragma unroll 1
-            for (int j = 0; j < n_kv; ++j) {
-                if (!tile_is_hot(j)) continue;
-                const int kpos = j * BN + row;
-                const bool hl = kpos < Lb && p.mask[seq0 + kpos] != 0;
-                if (!warp_wait(e_full, (uint32_t)(n_hot & 1), abort_flag, p.status, 30)) break;
-                ++n_hot;
-                tc_fence_after();
-                const uint32_t tE = t_lane + COL_S + 128 * (j < nA ? 0 : 1);
-                uint8_t* sK = smem + SL::K + (j % NK) * SL::TILE;
+                for (int j = 0; j < it.n_kv; ++j) {
+                    if (hot_g[j] == 0) continue;
+                    const int kpos = j * BN + row;
+                    const bool hl = kpos < it.Lb && p.mask[it.seq0 + kpos] != 0;
+                    ok = warp_wait(e_full, n_hot & 1, abort_flag, p.status, 30);
+                    if (!ok) break;
+                    ++n_hot;
+                    tc_fence_after();
+                    const uint32_t tE = t_lane + COL_S + 128 * (j < it.nA ? 0 : 1);
+                    uint8_t* sK = smem + SL::K + ((pr + (uint32_t)j) % NK) * SL::TILE;
 #pragma unroll 1
-                for (int c = 0; c < D / 32; ++c) {
-                    uint32_t dk[32];
-                    tmem_ld32(tE + c * 32, dk);
-                    tmem_wait_ld_on(dk);
-                    if (hl) {
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t dk[32];
+                        tmem_ld32(tE + c * 32, dk);
+                        tmem_wait_ld_on(dk);
+                        if (hl) {
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {      // 8 elements = one 16-byte unit of the swizzled row
-                            const int col = c * 32 + q * 8;
-                            uint4* ptr = reinterpret_cast<uint4*>(sK + (col >> 6) * BLK_BYTES + sw128_offset(row, col & 63));
-                            uint4 kv = *ptr;
-                            uint32_t* w = reinterpret_cast<uint32_t*>(&kv);
+                            for (int q = 0; q < 4; ++q) {      // 8 elements = one 16-byte unit of the swizzled row
+                                const int col = c * 32 + q * 8;
+                                uint4* ptr = reinterpret_cast<uint4*>(sK + (col >> 6) * BLK_BYTES + sw128_offset(row, col & 63));
+                                uint4 kv = *ptr;
+                                uint32_t* w = reinterpret_cast<uint32_t*>(&kv);
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const float2 k2 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&w[e]));
-                                w[e] = pack_bf16(k2.x + __uint_as_float(dk[q * 8 + 2 * e]), k2.y + __uint_as_float(dk[q * 8 + 2 * e + 1]));
+                                for (int e = 0; e < 4; ++e) {
+                                    const float2 k2 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&w[e]));
+                                    w[e] = pack_bf16(k2.x + __uint_as_float(dk[q * 8 + 2 * e]), k2.y + __uint_as_float(dk[q * 8 + 2 * e + 1]));
+                                }
+                                *ptr = kv;
                             }
-                            *ptr = kv;
                         }
                     }
+                    fence_proxy_async();       // the rewritten rows are read next by the tensor core
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(k_edited);
                 }
-                fence_proxy_async();       // the rewritten rows are read next by the tensor core
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(k_edited);
             }
+            pr += it.n_kv;
         }
     } else {
         // ------------------------------------------------------------ softmax of tile x, one query row per thread
         reg_inc<REGS_SOFTMAX>();
         const int x = (warp - 4) >> 2;
-        const int nX = x ? nB : nA;
-        const int hqX = x ? tw[1].hq : tw[0].hq, qtX = x ? tw[1].qt : tw[0].qt;
         const int row = (warp & 3) * 32 + lane;
         const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
         const uint32_t tS = t_lane + COL_S + 128 * x, tO = t_lane + COL_O + D * x;
         const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
-        float m_run = -INFINITY, l_run = 0.f;
+        uint32_t cX = 0, n_o = 0;       // steps and items of this tile so far
         bool ok = true;
-        for (int j = 0; j < nX; ++j) {
-            ok = warp_wait(s_full + x, (uint32_t)(j & 1), abort_flag, p.status, 40 + x);
-            if (!ok) break;
-            tc_fence_after();
-            // the whole score row of this thread: 128 fp32 values in registers
-            uint32_t v[128];
+        while (ok && next_item(round, it)) {
+            const int nX = x ? it.nB : it.nA;
+            const int hqX = x ? it.hqB : it.hqA, qtX = x ? it.qtB : it.qtA;
+            if (nX == 0) continue;
+            float m_run = -INFINITY, l_run = 0.f;
+#pragma unroll 1
+            for (int j = 0; j < nX; ++j) {
+                ok = warp_wait(s_full + x, (cX + j) & 1, abort_flag, p.status, 40 + x);
+                if (!ok) break;
+                tc_fence_after();
+                // the whole score row of this thread: 128 fp32 values in registers
+                uint32_t v[128];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, reinterpret_cast<uint32_t(&)[32]>(v[32 * c]));
-            tmem_wait_ld();
-            if (j == nX - 1) {       // diagonal tile: keys after the query are masked
+                for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, reinterpret_cast<uint32_t(&)[32]>(v[32 * c]));
+                tmem_wait_ld();
+                if (j == nX - 1) {       // diagonal tile: keys after the query are masked
 #pragma unroll
-                for (int e = 0; e < 128; ++e)
-                    if (e > row) v[e] = 0xff800000u;
+                    for (int e = 0; e < 128; ++e)
+                        if (e > row) v[e] = 0xff800000u;
+                }
+                float mx[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    mx[q] = fmaxf(__uint_as_float(v[16 * q]), __uint_as_float(v[16 * q + 1]));
+#pragma unroll
+                    for (int e = 2; e < 16; e += 2) mx[q] = max3(mx[q], __uint_as_float(v[16 * q + e]), __uint_as_float(v[16 * q + e + 1]));
+                }
+                const float mx_all = fmaxf(max3(mx[0], mx[1], mx[2]), max3(mx[3], mx[4], max3(mx[5], mx[6], mx[7])));
+                const float m_new = fmaxf(m_run, mx_all * p.scale_log2);
+                // raise the running maximum only when it moved a lot; p may then exceed 1 (up to 2^8), which is harmless
+                const bool raise = (m_new - m_run) > LAZY_RESCALE_LOG2;      // true on the first tile (m_run = -inf)
+                const float factor = raise ? fast_exp2(m_run - m_new) : 1.f;
+                if (raise) m_run = m_new;
+                if (j > 0 && __any_sync(0xffffffffu, raise)) {
+                    uint32_t o[32];
+#pragma unroll 1
+                    for (int c = 0; c < D / 32; ++c) {
+                        tmem_ld32(tO + c * 32, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * factor);
+                        tmem_st32(tO + c * 32, o);
+                    }
+                }
+                const float2 nm2 = make_float2(-m_run, -m_run);
+                float2 sum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t pk16[16];
+#pragma unroll
+                    for (int e2 = 0; e2 < 16; ++e2) {
+                        const int e = 32 * c + 2 * e2;
+                        const float2 arg = __ffma2_rn(make_float2(__uint_as_float(v[e]), __uint_as_float(v[e + 1])), sc2, nm2);
+                        float2 pe;
+                        if ((POLY_PAIR_MASK >> e2) & 1u) {
+                            pe = exp2_poly2(arg);
+                        } else {
+                            pe.x = fast_exp2(arg.x);
+                            pe.y = fast_exp2(arg.y);
+                        }
+                        sum[e2 & 1] = __fadd2_rn(sum[e2 & 1], pe);
+                        pk16[e2] = pack_bf16(pe.x, pe.y);
+                    }
+                    tmem_st16(tS + c * 16, pk16);     // P (bf16 pairs) over score columns that are already in registers
+                    if (c == 2) {                     // keys 0-95 are in place: the tensor core may start on them
+                        tmem_wait_st();
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(p_full + x);
+                    }
+                }
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(p_last + x);
+                const float2 s2 = __fadd2_rn(sum[0], sum[1]);
+                l_run = l_run * factor + (s2.x + s2.y);
             }
-            float mx[8];
-#pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                mx[q] = fmaxf(__uint_as_float(v[16 * q]), __uint_as_float(v[16 * q + 1]));
-#pragma unroll
-                for (int e = 2; e < 16; e += 2) mx[q] = max3(mx[q], __uint_as_float(v[16 * q + e]), __uint_as_float(v[16 * q + e + 1]));
-            }
-            const float mx_all = fmaxf(max3(mx[0], mx[1], mx[2]), max3(mx[3], mx[4], max3(mx[5], mx[6], mx[7])));
-            const float m_new = fmaxf(m_run, mx_all * p.scale_log2);
-            // raise the running maximum only when it moved a lot; p may then exceed 1 (up to 2^8), which is harmless
-            const bool raise = (m_new - m_run) > LAZY_RESCALE_LOG2;      // true on the first tile (m_run = -inf)
-            const float factor = raise ? fast_exp2(m_run - m_new) : 1.f;
-            if (raise) m_run = m_new;
-            if (j > 0 && __any_sync(0xffffffffu, raise)) {
+            cX += nX;
+            if (ok) ok = warp_wait(o_full + x, n_o & 1, abort_flag, p.status, 44 + x);
+            ++n_o;
+            if (ok) {
+                // final normalisation and store; the next item's first P_x (hence its first P_x V into these
+                // columns) comes from these same threads, after they are done reading here
+                tc_fence_after();
+                const int qpos = qtX * BM + row;
+                const bool valid = qpos < it.Lb;
+                const size_t orow = (size_t)(it.seq0 + (valid ? qpos : 0)) * p.Hq + hqX;
+                const float inv = 1.f / l_run;
                 uint32_t o[32];
 #pragma unroll 1
                 for (int c = 0; c < D / 32; ++c) {
                     tmem_ld32(tO + c * 32, o);
                     tmem_wait_ld();
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * factor);
-                    tmem_st32(tO + c * 32, o);
+                    if (valid) store_chunk32<OutT>(static_cast<OutT*>(p.O) + orow * D + c * 32, o, inv);
                 }
+                if (valid && p.lse != nullptr) p.lse[orow] = (m_run + log2f(l_run)) * 0.6931471805599453f;
+                tc_fence_before();
             }
-            const float2 nm2 = make_float2(-m_run, -m_run);
-            float2 sum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t pk16[16];
-#pragma unroll
-                for (int e2 = 0; e2 < 16; ++e2) {
-                    const int e = 32 * c + 2 * e2;
-                    const float2 arg = __ffma2_rn(make_float2(__uint_as_float(v[e]), __uint_as_float(v[e + 1])), sc2, nm2);
-                    float2 pe;
-                    if ((POLY_PAIR_MASK >> e2) & 1u) {
-                        pe = exp2_poly2(arg);
-                    } else {
-                        pe.x = fast_exp2(arg.x);
-                        pe.y = fast_exp2(arg.y);
-                    }
-                    sum[e2 & 1] = __fadd2_rn(sum[e2 & 1], pe);
-                    pk16[e2] = pack_bf16(pe.x, pe.y);
-                }
-                tmem_st16(tS + c * 16, pk16);     // P (bf16 pairs) over score columns that are already in registers
-                if (c == 2) {                     // keys 0-95 are in place: the tensor core may start on them
-                    tmem_wait_st();
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(p_full + x);
-                }
-            }
-            tmem_wait_st();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(p_last + x);
-            const float2 s2 = __fadd2_rn(sum[0], sum[1]);
-            l_run = l_run * factor + (s2.x + s2.y);
-        }
-        if (ok && nX > 0) ok = warp_wait(o_full + x, 0, abort_flag, p.status, 44 + x);
-        if (ok && nX > 0) {
-            tc_fence_after();
-            const int qpos = qtX * BM + row;
-            const bool valid = qpos < Lb;
-            const size_t orow = (size_t)(seq0 + (valid ? qpos : 0)) * p.Hq + hqX;
-            const float inv = 1.f / l_run;
-            uint32_t o[32];
-#pragma unroll 1
-            for (int c = 0; c < D / 32; ++c) {
-                tmem_ld32(tO + c * 32, o);
-                tmem_wait_ld();
-                if (valid) store_chunk32<OutT>(static_cast<OutT*>(p.O) + orow * D + c * 32, o, inv);
-            }
-            if (valid && p.lse != nullptr) p.lse[orow] = (m_run + log2f(l_run)) * 0.6931471805599453f;
         }
     }
 
@@ -600,7 +684,14 @@ static seka_status launch_attn(const CUtensorMap& tq, const CUtensorMap& tk, con
                                  (int)SL::DYN_BYTES) != cudaSuccess) return SEKA_ERR_CUDA;
         configured = true;
     }
-    const unsigned grid = p.pair_heads ? (unsigned)p.n_qt * p.B * (p.Hq / 2) : (unsigned)((p.n_qt + 1) / 2) * p.B * p.Hq;
+    static int n_sm = 0;
+    if (n_sm == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm <= 0) { n_sm = 0; return SEKA_ERR_CUDA; }
+    }
+    // persistent CTAs, one per SM (the kernel needs the whole SM: all of tensor memory and most of shared memory)
+    const unsigned grid = (unsigned)(p.n_items < (long long)n_sm ? p.n_items : (long long)n_sm);
     seka_attn_fwd_kernel<D, OutT><<<grid, NTHREADS, SL::DYN_BYTES, st>>>(tq, tk, tv, tw, p);
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? SEKA_OK : SEKA_ERR_CUDA;
@@ -653,6 +744,7 @@ extern "C" seka_status seka_attention_fwd(const seka_shape* shape, const void* Q
     p.B = shape->batch; p.L = shape->max_seqlen; p.Hq = Hq; p.Hkv = Hkv;
     p.n_qt = w.n_tiles; p.steer = steer ? 1 : 0;
     p.pair_heads = ((Hq / Hkv) % 2 == 0) ? 1 : 0;
+    p.n_items = p.pair_heads ? (long long)p.n_qt * p.B * (Hq / 2) : (long long)((p.n_qt + 1) / 2) * p.B * Hq;
     const float scale = shape->softmax_scale > 0.f ? shape->softmax_scale : 1.f / sqrtf((float)D);
     p.scale_log2 = scale * 1.4426950408889634f;
 
