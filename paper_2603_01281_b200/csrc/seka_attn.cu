@@ -42,9 +42,10 @@ struct AttnParams {
     const uint8_t* tile_hot;      // [B, n_qt]: key tile holds a highlighted token
     int* status;
     int B, L, Hq, Hkv, n_qt;
-    long long n_items;    // work items (pairs of query tiles) of the launch
+    const ItemRecord* items;   // item table (built by the preparation kernel), heaviest first
+    const int* n_items;        // its length (device word)
+    long long n_items_max;
     int steer;
-    int pair_heads;       // 1: the two tiles of a CTA are two query heads of one KV group; 0: two consecutive query tiles
     float scale_log2;
 };
 
@@ -176,40 +177,40 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     // an earlier launch (or CTA) gave up on this workspace: all threads agree on leaving
     if (__syncthreads_or(*reinterpret_cast<volatile int*>(p.status) != 0)) return;
 
-    // The CTA is persistent: it walks its share of the items (heaviest first; odd rounds run the CTAs in
-    // reverse so that the shares come out even).  Every role decodes the same sequence of items by itself.
-    auto next_item = [&](int& round, Item& it) -> bool {
-        while (true) {
-            const long long G = gridDim.x;
-            const long long idx = (long long)round * G + ((round & 1) ? (G - 1 - blockIdx.x) : blockIdx.x);
-            ++round;
-            if (idx >= p.n_items) return false;
-            if (p.pair_heads) {
-                const int per_qt = p.B * (p.Hq >> 1);
-                const int qt = p.n_qt - 1 - (int)(idx / per_qt);
-                const int rem = (int)(idx % per_qt);
-                it.b = rem / (p.Hq >> 1);
-                const int hp = rem % (p.Hq >> 1);
-                it.hqA = 2 * hp; it.hqB = 2 * hp + 1;
-                it.qtA = it.qtB = qt;
-            } else {
-                const int per_qt = p.B * p.Hq;
-                const int qt2 = ((p.n_qt + 1) >> 1) - 1 - (int)(idx / per_qt);
-                const int rem = (int)(idx % per_qt);
-                it.b = rem / p.Hq;
-                it.hqA = it.hqB = rem % p.Hq;
-                it.qtA = 2 * qt2; it.qtB = 2 * qt2 + 1;
-            }
-            it.hkv = it.hqA / (p.Hq / p.Hkv);
-            it.seq0 = p.cu_seqlens ? p.cu_seqlens[it.b] : it.b * p.L;
-            it.Lb = p.cu_seqlens ? (p.cu_seqlens[it.b + 1] - it.seq0) : p.L;
-            it.nA = it.qtA * BM < it.Lb ? it.qtA + 1 : 0;
-            it.nB = it.qtB * BM < it.Lb ? it.qtB + 1 : 0;
-            if (it.nA == 0) continue;                       // beyond the sequence (tile B starts no earlier)
-            it.n_kv = max(it.nA, it.nB);
-            it.steer = p.steer && p.gain[it.b] != 0.f && (p.head_enable == nullptr || p.head_enable[it.hkv] != 0);
-            return true;
+    // The CTA is persistent: it walks its share of the item table (heaviest first; odd rounds run the CTAs in
+    // reverse so that the shares come out even).  Every role reads the same sequence of records by itself,
+    // one item ahead of its use (the load is issued when the previous item starts).
+    const int n_items = *p.n_items;
+    auto item_index = [&](int round) -> int {
+        const int G = (int)gridDim.x;
+        const long long idx = (long long)round * G + ((round & 1) ? (G - 1 - (int)blockIdx.x) : (int)blockIdx.x);
+        return idx < n_items ? (int)idx : -1;
+    };
+    int4 raw0 = make_int4(0, 0, 0, 0), raw1 = make_int4(0, 0, 0, 0);
+    int round = 0, idx_next = item_index(0);
+    auto fetch = [&]() {
+        if (idx_next >= 0) {
+            // volatile on purpose: the record is wanted one whole item later, and a plain load may be moved
+            // down to its first use, where it would cost a trip to memory on the path between two items
+            const int4* rec = reinterpret_cast<const int4*>(p.items + idx_next);
+            asm volatile("ld.global.nc.v4.s32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(raw0.x), "=r"(raw0.y), "=r"(raw0.z), "=r"(raw0.w) : "l"(rec));
+            asm volatile("ld.global.nc.v4.s32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(raw1.x), "=r"(raw1.y), "=r"(raw1.z), "=r"(raw1.w) : "l"(rec + 1));
         }
+    };
+    fetch();
+    auto next_item = [&](Item& it) -> bool {
+        if (idx_next < 0) return false;
+        it.seq0 = raw0.x; it.Lb = raw0.y; it.b = raw0.z; it.hkv = raw0.w;
+        it.hqA = raw1.x & 0xffff; it.hqB = raw1.x >> 16;
+        it.qtA = raw1.y & 0xffff; it.qtB = raw1.y >> 16;
+        it.nA = raw1.z & 0xffff; it.nB = raw1.z >> 16;
+        it.steer = raw1.w != 0;
+        it.n_kv = max(it.nA, it.nB);
+        idx_next = item_index(++round);
+        fetch();
+        return true;
     };
 
     if (tid == 0) {
@@ -233,7 +234,6 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     //   pr   V/K pairs so far (n_kv per item); pair t of an item uses V stage (pr + t) % NK and K stage (pr + t + 1) % NK
     //   cA/cB  steps of tile A / B so far (phases of s_full, p_full, p_last)
     Item it;
-    int round = 0;
 
     if (warp < 4) {
         reg_dec<REGS_CTRL>();
@@ -245,7 +245,7 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             uint32_t ev = 0, pr = 0, n_it = 0, n_qb = 0;
             int prev_n = 0;
             bool ok = true;
-            while (ok && next_item(round, it)) {
+            while (ok && next_item(it)) {
                 // Q, W and the first K of an item may land once the last score product of the previous item is
                 // done (event n_kv - 1 of that item), its V/K pairs once its last step is done (event n_kv)
                 if (n_it > 0) {
@@ -327,7 +327,7 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                 if (leader) umma_commit(bar);
                 __syncwarp();
             };
-            while (ok && next_item(round, it)) {
+            while (ok && next_item(it)) {
                 const uint8_t* hot_g = p.tile_hot + (size_t)it.b * p.n_qt;
                 bool w_seen = false;
                 // Before the first score product of key tile j (by tile x): if the tile holds highlighted tokens,
@@ -450,7 +450,7 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             // fifth arrival on p_full of step j, so that the MMA issuer waits on one barrier per hand-off
             uint32_t pr = 0, cx[2] = {0, 0};
             bool ok = true;
-            while (ok && next_item(round, it)) {
+            while (ok && next_item(it)) {
 #pragma unroll 1
                 for (int j = 0; j < it.n_kv; ++j) {
                     const uint32_t g = pr + j;
@@ -476,7 +476,7 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         const uint32_t t_lane = tmem_base + ((uint32_t)((warp - 12) * 32) << 16);
         uint32_t pr = 0, n_hot = 0;
         bool ok = true;
-        while (ok && next_item(round, it)) {
+        while (ok && next_item(it)) {
             if (it.steer) {
                 const uint8_t* hot_g = p.tile_hot + (size_t)it.b * p.n_qt;
 #pragma unroll 1
@@ -529,7 +529,7 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
         uint32_t cX = 0, n_o = 0;       // steps and items of this tile so far
         bool ok = true;
-        while (ok && next_item(round, it)) {
+        while (ok && next_item(it)) {
             const int nX = x ? it.nB : it.nA;
             const int hqX = x ? it.hqB : it.hqA, qtX = x ? it.qtB : it.qtA;
             if (nX == 0) continue;
@@ -691,7 +691,7 @@ static seka_status launch_attn(const CUtensorMap& tq, const CUtensorMap& tk, con
             cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm <= 0) { n_sm = 0; return SEKA_ERR_CUDA; }
     }
     // persistent CTAs, one per SM (the kernel needs the whole SM: all of tensor memory and most of shared memory)
-    const unsigned grid = (unsigned)(p.n_items < (long long)n_sm ? p.n_items : (long long)n_sm);
+    const unsigned grid = (unsigned)(p.n_items_max < (long long)n_sm ? p.n_items_max : (long long)n_sm);
     seka_attn_fwd_kernel<D, OutT><<<grid, NTHREADS, SL::DYN_BYTES, st>>>(tq, tk, tv, tw, p);
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? SEKA_OK : SEKA_ERR_CUDA;
@@ -713,6 +713,7 @@ extern "C" seka_status seka_attention_fwd(const seka_shape* shape, const void* Q
     const bool steer = mask != nullptr && U != nullptr;
     if (steer && !gain) return SEKA_ERR_INVALID_ARG;
     const WorkspaceLayout w = workspace_layout(shape);
+    if (w.n_tiles > 32767 || shape->n_q_heads > 32767 || w.n_items_max > 0x7fffffffLL) return SEKA_ERR_UNSUPPORTED;   // item records pack 15-bit fields
     if (!workspace || workspace_bytes < w.total || ((uintptr_t)workspace & 255)) return SEKA_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     char* ws = static_cast<char*>(workspace);
@@ -743,8 +744,9 @@ extern "C" seka_status seka_attention_fwd(const seka_shape* shape, const void* Q
     p.cu_seqlens = shape->cu_seqlens; p.tile_hot = tile_hot; p.status = reinterpret_cast<int*>(ws);
     p.B = shape->batch; p.L = shape->max_seqlen; p.Hq = Hq; p.Hkv = Hkv;
     p.n_qt = w.n_tiles; p.steer = steer ? 1 : 0;
-    p.pair_heads = ((Hq / Hkv) % 2 == 0) ? 1 : 0;
-    p.n_items = p.pair_heads ? (long long)p.n_qt * p.B * (Hq / 2) : (long long)((p.n_qt + 1) / 2) * p.B * Hq;
+    ItemRecord* items = reinterpret_cast<ItemRecord*>(ws + w.item_off);
+    launch_build_items(shape, w, steer, gain, head_enable, items, reinterpret_cast<int*>(ws) + 3, st);
+    p.items = items; p.n_items = reinterpret_cast<int*>(ws) + 3; p.n_items_max = w.n_items_max;
     const float scale = shape->softmax_scale > 0.f ? shape->softmax_scale : 1.f / sqrtf((float)D);
     p.scale_log2 = scale * 1.4426950408889634f;
 

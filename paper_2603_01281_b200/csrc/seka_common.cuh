@@ -13,9 +13,11 @@ namespace seka {
 
 // ---------------------------------------------------------------- workspace layout
 // [0, 256)            status block: word 0 = seka_status, word 1 = where the wait gave up,
-//                     word 2 = number of highlighted tokens found by the compaction pass
+//                     word 2 = number of highlighted tokens found by the compaction pass,
+//                     word 3 = number of work items in the item table of the fused kernel
 // [256, ...)          dense edit operators W[b][h] = gain_b * sum_m alpha_{b,h,m} U_m U_m^T as bf16 [D x D]
 // then                one byte per (sequence, 128-key tile): the tile contains a highlighted token
+// then                item table of the fused kernel (32 bytes per pair of query tiles, heaviest first)
 // then                compacted highlighted-token list (int32 per token)
 // then (fp32 inputs)  bf16 copies of Q, K, V
 constexpr size_t kStatusBytes = 256;
@@ -23,10 +25,13 @@ constexpr size_t kStatusBytes = 256;
 struct WorkspaceLayout {
     size_t w_off, w_bytes;            // bf16 [B, Hkv, D, D]
     size_t hot_off, hot_bytes;        // uint8 [B, ceil(max_seqlen / 128)]
+    size_t item_off, item_bytes;      // ItemRecord [n_items_max]
     size_t list_off, list_bytes;      // int32 [total_tokens]
     size_t cvt_off, cvt_bytes;        // bf16 copies of Q, K, V (fp32 inputs only)
     size_t total;
     int n_tiles;                      // key tiles per sequence = ceil(max_seqlen / 128)
+    int pair_heads;                   // items pair two query heads of a KV group (even group size) or two row tiles
+    long long n_items_max;            // item slots before empty ones (tiles beyond a short sequence) are dropped
 };
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -43,7 +48,13 @@ static inline WorkspaceLayout workspace_layout(const seka_shape* s) {
     w.w_bytes = align_up((size_t)s->batch * s->n_kv_heads * s->head_dim * s->head_dim * 2, 1024);
     w.hot_off = w.w_off + w.w_bytes;
     w.hot_bytes = align_up((size_t)s->batch * w.n_tiles + 1, 256);
-    w.list_off = w.hot_off + w.hot_bytes;
+    const int G = s->n_q_heads / s->n_kv_heads;
+    w.pair_heads = (G % 2 == 0) ? 1 : 0;
+    w.n_items_max = w.pair_heads ? (long long)w.n_tiles * s->batch * (s->n_q_heads / 2)
+                                 : (long long)((w.n_tiles + 1) / 2) * s->batch * s->n_q_heads;
+    w.item_off = w.hot_off + w.hot_bytes;
+    w.item_bytes = align_up((size_t)w.n_items_max * 32 + 32, 256);
+    w.list_off = w.item_off + w.item_bytes;
     w.list_bytes = align_up(T * 4 + 4, 256);
     w.cvt_off = w.list_off + w.list_bytes;
     w.cvt_bytes = 0;
@@ -53,6 +64,16 @@ static inline WorkspaceLayout workspace_layout(const seka_shape* s) {
     w.total = w.cvt_off + w.cvt_bytes;
     return w;
 }
+
+// One work item of the fused kernel: two 128-row query tiles that share a KV head of one sequence.
+struct __align__(16) ItemRecord {
+    int seq0, Lb;           // first token and length of the sequence
+    int b, hkv;
+    int hq;                 // query head of tile A | query head of tile B << 16
+    int qt;                 // row-tile index of tile A | of tile B << 16
+    int n;                  // key tiles of tile A | of tile B << 16 (0: the tile lies beyond the sequence)
+    int steer;              // the keys of this (sequence, KV head) are edited
+};
 
 extern unsigned long long g_launches;   // kernels launched by this library in this process
 
@@ -88,11 +109,21 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-// One poll: returns at once if the phase has completed, otherwise the hardware parks the thread until the
-// phase completes or about kPollNs have passed, whichever comes first (a parked thread takes no issue slots
-// from the warps that share its scheduler; a spinning one does).
+// One poll of an mbarrier phase.  The plain form returns at once either way (about 40 cycles when the phase
+// has completed).  The parked form, if the phase has not completed, lets the hardware park the thread until it
+// completes or about kPollNs have passed: a parked thread takes no issue slots from the warps that share its
+// scheduler, but the form costs about twice as much when the phase has already completed.
 constexpr uint32_t kPollNs = 20000;
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_try_wait_parked(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
@@ -105,15 +136,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // Bounded wait: gives up after kWaitLimitNs or as soon as another thread has raised the
 // CTA's abort flag, records where, raises the flag and returns false.  The caller must
 // then leave through its teardown path (no further waits succeed once the flag is up).
+// A few plain polls first (most waits on the tensor pipe's critical path find their phase
+// complete or nearly so), then parked ones.
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s; a whole launch takes milliseconds
+constexpr int kPlainPolls = 8;
 
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
                                           int* status, int where) {
+#pragma unroll 1
+    for (int i = 0; i < kPlainPolls; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
     uint64_t t0 = 0;
     while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
-        // a poll came back empty-handed: that is rare (tens of microseconds have passed), so the flag and
-        // the clock can be looked at every time
+        if (mbar_try_wait_parked(bar, parity)) return true;
+        // a parked poll came back empty-handed: that is rare (tens of microseconds have passed), so the flag
+        // and the clock can be looked at every time
         if (*abort_flag) return false;
         const uint64_t now = global_timer_ns();
         if (t0 == 0) {

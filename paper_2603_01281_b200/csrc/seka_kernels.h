@@ -11,6 +11,8 @@ namespace seka {
 void launch_prep_steering(const seka_shape* s, const float* U, const float* alpha, const float* gain,
                           const uint8_t* head_enable, const uint8_t* mask, void* W, uint8_t* tile_hot, int n_tiles,
                           cudaStream_t st);
+void launch_build_items(const seka_shape* s, const WorkspaceLayout& w, bool steer, const float* gain,
+                        const uint8_t* head_enable, ItemRecord* items, int* count, cudaStream_t st);
 void launch_compact_mask(const uint8_t* mask, int T, int* list, int* count, cudaStream_t st);
 void launch_convert_bf16(const float* in, void* out, size_t n, cudaStream_t st);
 

@@ -64,6 +64,79 @@ __global__ void prep_steering_kernel(const float* __restrict__ U, const float* _
     }
 }
 
+// Item table of the fused kernel: slot idx (heaviest row tiles first; the items of one (sequence, KV head)
+// next to each other) decoded into an ItemRecord.  Returns false for a slot whose tiles lie beyond the
+// sequence.
+__device__ __forceinline__ bool decode_item(long long idx, int B, int L, int Hq, int Hkv, int n_qt, int pair_heads,
+                                            const int* __restrict__ cu, int steer_call, const float* __restrict__ gain,
+                                            const uint8_t* __restrict__ head_enable, ItemRecord& r) {
+    int hqA, hqB, qtA, qtB;
+    if (pair_heads) {
+        const int per_qt = B * (Hq >> 1);
+        const int qt = n_qt - 1 - (int)(idx / per_qt);
+        const int rem = (int)(idx % per_qt);
+        r.b = rem / (Hq >> 1);
+        const int hp = rem % (Hq >> 1);
+        hqA = 2 * hp; hqB = 2 * hp + 1; qtA = qtB = qt;
+    } else {
+        const int per_qt = B * Hq;
+        const int qt2 = ((n_qt + 1) >> 1) - 1 - (int)(idx / per_qt);
+        const int rem = (int)(idx % per_qt);
+        r.b = rem / Hq;
+        hqA = hqB = rem % Hq; qtA = 2 * qt2; qtB = 2 * qt2 + 1;
+    }
+    r.hkv = hqA / (Hq / Hkv);
+    r.seq0 = cu ? cu[r.b] : r.b * L;
+    r.Lb = (cu ? cu[r.b + 1] : (r.b + 1) * L) - r.seq0;
+    const int nA = qtA * 128 < r.Lb ? qtA + 1 : 0, nB = qtB * 128 < r.Lb ? qtB + 1 : 0;
+    r.hq = hqA | (hqB << 16); r.qt = qtA | (qtB << 16); r.n = nA | (nB << 16);
+    r.steer = (steer_call && gain[r.b] != 0.f && (head_enable == nullptr || head_enable[r.hkv] != 0)) ? 1 : 0;
+    return nA > 0;
+}
+
+// Fixed-length batches have no empty slots: one thread per item.
+__global__ void build_items_kernel(long long n, int B, int L, int Hq, int Hkv, int n_qt, int pair_heads, int steer_call,
+                                   const float* __restrict__ gain, const uint8_t* __restrict__ head_enable,
+                                   ItemRecord* __restrict__ items, int* __restrict__ count) {
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx == 0) *count = (int)n;
+    if (idx >= n) return;
+    ItemRecord r;
+    decode_item(idx, B, L, Hq, Hkv, n_qt, pair_heads, nullptr, steer_call, gain, head_enable, r);
+    items[idx] = r;
+}
+
+// Packed variable-length batches: slots beyond a short sequence are dropped, order kept (one CTA scans).
+__global__ void build_items_varlen_kernel(long long n, int B, int L, int Hq, int Hkv, int n_qt, int pair_heads,
+                                          const int* __restrict__ cu, int steer_call, const float* __restrict__ gain,
+                                          const uint8_t* __restrict__ head_enable, ItemRecord* __restrict__ items,
+                                          int* __restrict__ count) {
+    __shared__ int warp_tot[32];
+    __shared__ int base_s;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nw = blockDim.x >> 5;
+    if (tid == 0) base_s = 0;
+    __syncthreads();
+    for (long long start = 0; start < n; start += blockDim.x) {
+        const long long idx = start + tid;
+        ItemRecord r;
+        const bool keep = idx < n && decode_item(idx, B, L, Hq, Hkv, n_qt, pair_heads, cu, steer_call, gain, head_enable, r);
+        const unsigned bal = __ballot_sync(0xffffffffu, keep);
+        if (lane == 0) warp_tot[wid] = __popc(bal);
+        __syncthreads();
+        int off = base_s;
+        for (int q = 0; q < wid; ++q) off += warp_tot[q];
+        if (keep) items[off + __popc(bal & ((1u << lane) - 1))] = r;
+        __syncthreads();
+        if (tid == 0) {
+            int tot = 0;
+            for (int q = 0; q < nw; ++q) tot += warp_tot[q];
+            base_s += tot;
+        }
+        __syncthreads();
+    }
+    if (tid == 0) *count = base_s;
+}
+
 // Appends the indices of highlighted tokens to `list` (order within a warp preserved).
 __global__ void compact_mask_kernel(const uint8_t* __restrict__ mask, int T, int* __restrict__ list,
                                     int* __restrict__ count) {
@@ -95,6 +168,19 @@ void launch_prep_steering(const seka_shape* sh, const float* U, const float* alp
                                                       static_cast<__nv_bfloat16*>(W), tile_hot, sh->batch,
                                                       sh->max_seqlen, sh->n_kv_heads, D, sh->rank, sh->n_experts,
                                                       n_tiles, n_w);
+    ++g_launches;
+}
+
+void launch_build_items(const seka_shape* sh, const WorkspaceLayout& w, bool steer, const float* gain,
+                        const uint8_t* head_enable, ItemRecord* items, int* count, cudaStream_t st) {
+    const long long n = w.n_items_max;
+    if (sh->cu_seqlens == nullptr)
+        build_items_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(n, sh->batch, sh->max_seqlen, sh->n_q_heads,
+                                                                       sh->n_kv_heads, w.n_tiles, w.pair_heads, steer ? 1 : 0,
+                                                                       gain, head_enable, items, count);
+    else
+        build_items_varlen_kernel<<<1, 1024, 0, st>>>(n, sh->batch, sh->max_seqlen, sh->n_q_heads, sh->n_kv_heads, w.n_tiles,
+                                                      w.pair_heads, sh->cu_seqlens, steer ? 1 : 0, gain, head_enable, items, count);
     ++g_launches;
 }
 
