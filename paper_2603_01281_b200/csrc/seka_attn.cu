@@ -46,6 +46,7 @@ struct AttnParams {
     const int* n_items;        // its length (device word)
     long long n_items_max;
     int steer;
+    int pair_heads;       // 1: the two tiles of an item are two query heads of one KV group; 0: two consecutive row tiles
     float scale_log2;
 };
 
@@ -53,8 +54,8 @@ constexpr int BM = 128, BN = 128;
 constexpr int NTHREADS = 512;
 constexpr uint32_t BLK_BYTES = 128 * 128;   // one [128 x 64] bf16 block
 constexpr float LAZY_RESCALE_LOG2 = 8.0f;   // the running maximum is only raised when it moved by more than this
-// registers per thread after the roles split (the CTA owns the whole register file: 4 x 128 x (56+184+184+88) = 64 Ki)
-constexpr int REGS_CTRL = 56, REGS_SOFTMAX = 184, REGS_EDIT = 88;
+// registers per thread after the roles split (the CTA owns the whole register file: 4 x 128 x (80+184+184+64) = 64 Ki)
+constexpr int REGS_CTRL = 80, REGS_SOFTMAX = 184, REGS_EDIT = 64;
 // which of the 16 element pairs of every 32-key chunk take the polynomial exp2 instead of the special-function unit
 constexpr uint32_t POLY_PAIR_MASK = SEKA_POLY_PAIR_MASK;
 
@@ -71,7 +72,8 @@ struct SmemLayout {
     static constexpr uint32_t BARS = W + (D / 64) * WBLK;  // mbarriers
     static constexpr uint32_t NBARS = 3 + 2 * NK + 8 + 3;
     static constexpr uint32_t MISC = BARS + NBARS * 8;     // tmem holder, abort flag
-    static constexpr uint32_t TOTAL = MISC + 16;
+    static constexpr uint32_t ITEMS = MISC + 16;           // one 32-byte item record per warp
+    static constexpr uint32_t TOTAL = ITEMS + 16 * 32;
     static constexpr uint32_t DYN_BYTES = TOTAL + 1024;    // slack for the 1024-byte alignment
 };
 
@@ -146,7 +148,7 @@ struct Item {
     bool steer;
 };
 
-template <int D, typename OutT>
+template <int D, typename OutT, bool TABLE>
 __global__ void __launch_bounds__(NTHREADS, 1)
 seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                      const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmW,
@@ -177,39 +179,71 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     // an earlier launch (or CTA) gave up on this workspace: all threads agree on leaving
     if (__syncthreads_or(*reinterpret_cast<volatile int*>(p.status) != 0)) return;
 
-    // The CTA is persistent: it walks its share of the item table (heaviest first; odd rounds run the CTAs in
-    // reverse so that the shares come out even).  Every role reads the same sequence of records by itself,
-    // one item ahead of its use (the load is issued when the previous item starts).
-    const int n_items = *p.n_items;
+    // The CTA is persistent: it walks its share of the items (heaviest first; odd rounds run the CTAs in
+    // reverse so that the shares come out even).  Every role goes through the same sequence of items by itself.
+    // Fixed-length batches decode the item from its index; packed variable-length batches, where many index
+    // slots are empty (row tiles beyond a short sequence), read a table from which those were dropped.
+    const int n_items = TABLE ? *p.n_items : (int)p.n_items_max;
     auto item_index = [&](int round) -> int {
         const int G = (int)gridDim.x;
         const long long idx = (long long)round * G + ((round & 1) ? (G - 1 - (int)blockIdx.x) : (int)blockIdx.x);
         return idx < n_items ? (int)idx : -1;
     };
-    int4 raw0 = make_int4(0, 0, 0, 0), raw1 = make_int4(0, 0, 0, 0);
-    int round = 0, idx_next = item_index(0);
-    auto fetch = [&]() {
-        if (idx_next >= 0) {
-            // volatile on purpose: the record is wanted one whole item later, and a plain load may be moved
-            // down to its first use, where it would cost a trip to memory on the path between two items
-            const int4* rec = reinterpret_cast<const int4*>(p.items + idx_next);
-            asm volatile("ld.global.nc.v4.s32 {%0, %1, %2, %3}, [%4];"
-                         : "=r"(raw0.x), "=r"(raw0.y), "=r"(raw0.z), "=r"(raw0.w) : "l"(rec));
-            asm volatile("ld.global.nc.v4.s32 {%0, %1, %2, %3}, [%4];"
-                         : "=r"(raw1.x), "=r"(raw1.y), "=r"(raw1.z), "=r"(raw1.w) : "l"(rec + 1));
+    // (table) the record of the next item is copied into a per-warp slot of shared memory while the current item
+    // runs, so that no registers are held for it; lane 0 issues the copy and waits for it
+    int round = 0, idx_next = TABLE ? item_index(0) : 0;
+    auto prefetch = [&]() {
+        if (TABLE && idx_next >= 0 && lane == 0) {
+            const uint32_t dst = smem_u32(smem + SL::ITEMS + warp * 32);
+            const ItemRecord* rec = p.items + idx_next;
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(rec) : "memory");
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(dst + 16), "l"(reinterpret_cast<const char*>(rec) + 16) : "memory");
+            asm volatile("cp.async.commit_group;" ::: "memory");
         }
     };
-    fetch();
+    prefetch();
     auto next_item = [&](Item& it) -> bool {
-        if (idx_next < 0) return false;
-        it.seq0 = raw0.x; it.Lb = raw0.y; it.b = raw0.z; it.hkv = raw0.w;
-        it.hqA = raw1.x & 0xffff; it.hqB = raw1.x >> 16;
-        it.qtA = raw1.y & 0xffff; it.qtB = raw1.y >> 16;
-        it.nA = raw1.z & 0xffff; it.nB = raw1.z >> 16;
-        it.steer = raw1.w != 0;
+        if (TABLE) {
+            if (idx_next < 0) return false;
+            const uint8_t* slot = smem + SL::ITEMS + warp * 32;
+            if (lane == 0) asm volatile("cp.async.wait_group 0;" ::: "memory");
+            __syncwarp();
+            const int4 raw0 = *reinterpret_cast<const int4*>(slot), raw1 = *reinterpret_cast<const int4*>(slot + 16);
+            it.seq0 = raw0.x; it.Lb = raw0.y; it.b = raw0.z; it.hkv = raw0.w;
+            it.hqA = raw1.x & 0xffff; it.hqB = raw1.x >> 16;
+            it.qtA = raw1.y & 0xffff; it.qtB = raw1.y >> 16;
+            it.nA = raw1.z & 0xffff; it.nB = raw1.z >> 16;
+            it.steer = raw1.w != 0;
+            __syncwarp();            // every lane has read the slot before it is refilled
+            idx_next = item_index(++round);
+            prefetch();
+        } else {
+            const int idx = item_index(round++);
+            if (idx < 0) return false;
+            if (p.pair_heads) {
+                const int per_qt = p.B * (p.Hq >> 1);
+                const int qt = p.n_qt - 1 - (int)((unsigned)idx / (unsigned)per_qt);
+                const int rem = (int)((unsigned)idx % (unsigned)per_qt);
+                it.b = rem / (p.Hq >> 1);
+                const int hp = rem % (p.Hq >> 1);
+                it.hqA = 2 * hp; it.hqB = 2 * hp + 1;
+                it.qtA = it.qtB = qt;
+            } else {
+                const int per_qt = p.B * p.Hq;
+                const int qt2 = ((p.n_qt + 1) >> 1) - 1 - (int)((unsigned)idx / (unsigned)per_qt);
+                const int rem = (int)((unsigned)idx % (unsigned)per_qt);
+                it.b = rem / p.Hq;
+                it.hqA = it.hqB = rem % p.Hq;
+                it.qtA = 2 * qt2; it.qtB = 2 * qt2 + 1;
+            }
+            it.hkv = it.hqA / (p.Hq / p.Hkv);
+            it.seq0 = it.b * p.L;       // fixed length: every slot holds work (tile B of the last odd pair may not)
+            it.Lb = p.L;
+            it.nA = it.qtA * BM < it.Lb ? it.qtA + 1 : 0;
+            it.nB = it.qtB * BM < it.Lb ? it.qtB + 1 : 0;
+            it.steer = p.steer && p.gain[it.b] != 0.f && (p.head_enable == nullptr || p.head_enable[it.hkv] != 0);
+        }
         it.n_kv = max(it.nA, it.nB);
-        idx_next = item_index(++round);
-        fetch();
         return true;
     };
 
@@ -674,13 +708,13 @@ static bool make_tile_map(CUtensorMap* m, const void* base, int d, int H, long l
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int D, typename OutT>
-static seka_status launch_attn(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                               const CUtensorMap& tw, const AttnParams& p, cudaStream_t st) {
+template <int D, typename OutT, bool TABLE>
+static seka_status launch_attn_t(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                                 const CUtensorMap& tw, const AttnParams& p, cudaStream_t st) {
     using SL = SmemLayout<D>;
     static bool configured = false;
     if (!configured) {
-        if (cudaFuncSetAttribute(seka_attn_fwd_kernel<D, OutT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(seka_attn_fwd_kernel<D, OutT, TABLE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)SL::DYN_BYTES) != cudaSuccess) return SEKA_ERR_CUDA;
         configured = true;
     }
@@ -692,9 +726,16 @@ static seka_status launch_attn(const CUtensorMap& tq, const CUtensorMap& tk, con
     }
     // persistent CTAs, one per SM (the kernel needs the whole SM: all of tensor memory and most of shared memory)
     const unsigned grid = (unsigned)(p.n_items_max < (long long)n_sm ? p.n_items_max : (long long)n_sm);
-    seka_attn_fwd_kernel<D, OutT><<<grid, NTHREADS, SL::DYN_BYTES, st>>>(tq, tk, tv, tw, p);
+    seka_attn_fwd_kernel<D, OutT, TABLE><<<grid, NTHREADS, SL::DYN_BYTES, st>>>(tq, tk, tv, tw, p);
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? SEKA_OK : SEKA_ERR_CUDA;
+}
+
+template <int D, typename OutT>
+static seka_status launch_attn(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
+                               const CUtensorMap& tw, const AttnParams& p, cudaStream_t st) {
+    return p.cu_seqlens != nullptr ? launch_attn_t<D, OutT, true>(tq, tk, tv, tw, p, st)
+                                   : launch_attn_t<D, OutT, false>(tq, tk, tv, tw, p, st);
 }
 
 }  // namespace seka
@@ -745,7 +786,9 @@ extern "C" seka_status seka_attention_fwd(const seka_shape* shape, const void* Q
     p.B = shape->batch; p.L = shape->max_seqlen; p.Hq = Hq; p.Hkv = Hkv;
     p.n_qt = w.n_tiles; p.steer = steer ? 1 : 0;
     ItemRecord* items = reinterpret_cast<ItemRecord*>(ws + w.item_off);
-    launch_build_items(shape, w, steer, gain, head_enable, items, reinterpret_cast<int*>(ws) + 3, st);
+    if (shape->cu_seqlens != nullptr)
+        launch_build_items(shape, w, steer, gain, head_enable, items, reinterpret_cast<int*>(ws) + 3, st);
+    p.pair_heads = w.pair_heads;
     p.items = items; p.n_items = reinterpret_cast<int*>(ws) + 3; p.n_items_max = w.n_items_max;
     const float scale = shape->softmax_scale > 0.f ? shape->softmax_scale : 1.f / sqrtf((float)D);
     p.scale_log2 = scale * 1.4426950408889634f;
