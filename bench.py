@@ -33,7 +33,7 @@ METRIC = "SEKA fused attention TFLOP/s (% BF16 peak); overhead vs g=0, 8B shape"
 WORKLOAD = "C2: 8B-shaped prefill layer B=4 Hq=32 Hkv=8 d=128 L=4096 bf16, rank 32, ~10% highlighted spans, g=1"
 # DRAM bytes of one fused-kernel launch on this workload from the ncu capture summarised in
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture exists.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None  # the kernel has changed since the last capture
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 418624512  # profiles/seka_attn_fwd_kernel_d128_C2.md (322.62 MB read + 96.00 MB written)
 
 
 def measured_peaks():
@@ -218,11 +218,16 @@ def main():
     if st != binding.SEKA_OK:
         raise SystemExit("device status: " + binding.status_string(st))
 
-    # the same kernel with steering off (g = 0 path), interleaved afterwards for the overhead figure
+    # the same kernel with steering off (g = 0 path): blocks of 20 steps of either kind alternate, so that clock
+    # and temperature drift under the power cap falls on both alike
     for _ in range(3):
         step(False)
-    ms0, _, _ = timed(args.steps, False)
-    ms1, _, _ = timed(args.steps, True)
+    ms0 = ms1 = 0.0
+    n_blocks = max(2, args.steps // 20)
+    for _ in range(n_blocks):
+        t, _, _ = timed(20, False); ms0 += t
+        t, _, _ = timed(20, True); ms1 += t
+    ms0 *= args.steps / (20.0 * n_blocks); ms1 *= args.steps / (20.0 * n_blocks)
 
     # end to end through the host-buffer entry point: H2D of Q, K, V, mask and D2H of O every step
     staging = torch.empty(binding.seka_host_staging_bytes(shp), dtype=torch.uint8, device="cuda")
