@@ -544,6 +544,7 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                                 *ptr = kv;
                             }
                         }
+                        __syncwarp();      // all lanes together again before the next warp-wide load
                     }
                     fence_proxy_async();       // the rewritten rows are read next by the tensor core
                     tc_fence_before();
@@ -696,7 +697,7 @@ static EncodeTiledFn encode_tiled_fn() {
 }
 
 // bf16 tensor [T, H, d] viewed as (d, H, T); tiles of 64 x 1 x box_rows with the 128-byte swizzle.
-static bool make_tile_map(CUtensorMap* m, const void* base, int d, int H, long long T, int box_rows = 128) {
+bool make_tile_map(CUtensorMap* m, const void* base, int d, int H, long long T, int box_rows) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (fn == nullptr) return false;
     cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)H, (cuuint64_t)T};

@@ -45,7 +45,8 @@ static inline WorkspaceLayout workspace_layout(const seka_shape* s) {
     const size_t T = (size_t)shape_total_tokens(s);
     w.n_tiles = (s->max_seqlen + 127) / 128;
     w.w_off = kStatusBytes;
-    w.w_bytes = align_up((size_t)s->batch * s->n_kv_heads * s->head_dim * s->head_dim * 2, 1024);
+    // W[b][h] of the fused kernel, or the projectors P[m][h] = U_m U_m^T of the stand-alone edit (two bf16 parts each)
+    w.w_bytes = align_up((size_t)(s->batch > 2 * s->n_experts ? s->batch : 2 * s->n_experts) * s->n_kv_heads * s->head_dim * s->head_dim * 2, 1024);
     w.hot_off = w.w_off + w.w_bytes;
     w.hot_bytes = align_up((size_t)s->batch * w.n_tiles + 1, 256);
     const int G = s->n_q_heads / s->n_kv_heads;

@@ -91,6 +91,204 @@ static void launch_edit_rows(const seka_shape* s, const void* K_in, void* K_out,
     ++g_launches;
 }
 
+// ---------------------------------------------------------------- bf16 tensors: one 128-token tile per step, on tcgen05
+//
+// A CTA (4 warps, one key row per thread) takes the (highlighted tile, KV head) pairs of the hot-tile list in turn:
+// TMA stages the [128 x D] key tile and the projector P[m][h] = U_m U_m^T (two bf16 parts), the tensor core forms
+// K P_m in tensor memory (two products per expert), every thread adds  g_b sum_m alpha_{b,h,m} (K P_m)[row]  to its row in shared
+// memory if the row is highlighted, and the warps then write the highlighted rows out, 16 bytes per lane with the
+// lanes of a row next to each other.  Unhighlighted rows are never written.  Several CTAs share an SM (64 KB of
+// shared memory and M * D tensor-memory columns each), so loads, products and stores of different tiles overlap.
+constexpr uint32_t EBLK = 128 * 128;        // one [128 x 64] bf16 block
+
+template <int D>
+struct EditSmem {
+    static constexpr uint32_t TILE = (D / 64) * EBLK;
+    static constexpr uint32_t PBLK = D * 128;
+    static constexpr uint32_t K = 0;
+    static constexpr uint32_t P = K + TILE;
+    static constexpr uint32_t FLAGS = P + (D / 64) * PBLK;
+    static constexpr uint32_t BARS = FLAGS + 128;
+    static constexpr uint32_t MISC = BARS + 16;
+    static constexpr uint32_t DYN_BYTES = MISC + 16 + 1024;
+};
+
+template <int D>
+__global__ void __launch_bounds__(128)
+edit_tiles_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmP,
+                  __nv_bfloat16* __restrict__ K_out, const uint8_t* __restrict__ mask, const float* __restrict__ alpha,
+                  const float* __restrict__ gain, const uint8_t* __restrict__ head_enable,
+                  const int* __restrict__ cu_seqlens, const int* __restrict__ hot_list, const int* __restrict__ hot_count,
+                  int* status, int L, int Hkv, int M, int n_tiles, uint32_t tmem_cols) {
+    using SL = EditSmem<D>;
+    constexpr int NBLK = D / 64;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* sK = smem + SL::K;
+    uint8_t* flags = smem + SL::FLAGS;
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + SL::BARS);
+    uint64_t* done = full + 1;
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + SL::MISC);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + SL::MISC + 4);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (__syncthreads_or(*reinterpret_cast<volatile int*>(status) != 0)) return;
+
+    if (tid == 0) {
+        mbar_init(full, 1); mbar_init(done, 1);
+        *abort_flag = 0;
+        mbar_fence_init();
+        tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmP);
+    }
+    __syncwarp();
+    if (warp == 0) { tmem_alloc(tmem_holder, tmem_cols); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_holder;
+    const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
+    constexpr uint32_t IDESC = umma_idesc_bf16(D, false);
+    constexpr uint32_t DESC_HI = umma_desc_hi_sw128(1024);
+    const uint32_t dK = umma_desc_lo(smem_u32(sK), 16), dP = umma_desc_lo(smem_u32(smem + SL::P), 16);
+
+    const long long n_work = (long long)(*hot_count) * Hkv;
+    uint32_t n_full = 0, n_done = 0;
+    bool ok = true;
+    for (long long idx = blockIdx.x; idx < n_work && ok; idx += gridDim.x) {
+        const int tile = hot_list[idx / Hkv], h = (int)(idx % Hkv);
+        const int b = tile / n_tiles, t = tile % n_tiles;
+        const float g = gain[b];
+        if (g == 0.f || (head_enable != nullptr && head_enable[h] == 0)) continue;      // same for the whole CTA
+        const int seq0 = cu_seqlens ? cu_seqlens[b] : b * L;
+        const int Lb = (cu_seqlens ? cu_seqlens[b + 1] : (b + 1) * L) - seq0;
+        const int kpos = t * 128 + tid;
+        const bool hl = kpos < Lb && mask[seq0 + kpos] != 0;
+        flags[tid] = hl ? 1 : 0;
+        // 2 M products: the high and the low part of every projector accumulate into the same columns
+        for (int mm = 0; mm < 2 * M && ok; ++mm) {
+            const int m = mm >> 1, part = mm & 1;
+            if (tid == 0) {
+                mbar_expect_tx(full, (mm == 0 ? SL::TILE : 0u) + NBLK * SL::PBLK);
+                if (mm == 0) {
+#pragma unroll
+                    for (int c = 0; c < NBLK; ++c) tma_load_3d(sK + c * EBLK, &tmK, full, c * 64, h, seq0 + t * 128);
+                }
+#pragma unroll
+                for (int c = 0; c < NBLK; ++c)
+                    tma_load_3d(smem + SL::P + c * SL::PBLK, &tmP, full, c * 64, 0, ((part * M + m) * Hkv + h) * D);
+            }
+            ok = mbar_wait(full, n_full & 1, abort_flag, status, 60);
+            ++n_full;
+            ok = __syncthreads_and(ok);
+            if (!ok) break;
+            if (tid == 0) {
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const uint32_t offk = ((uint32_t)(ks >> 2) * EBLK + (uint32_t)(ks & 3) * 32) >> 4;
+                    const uint32_t offp = ((uint32_t)(ks >> 2) * SL::PBLK + (uint32_t)(ks & 3) * 32) >> 4;
+                    umma_ss(tmem_base + (uint32_t)m * D, dK + offk, DESC_HI, dP + offp, DESC_HI, IDESC, (ks > 0 || part) ? 1u : 0u);
+                }
+                umma_commit(done);
+            }
+            ok = mbar_wait(done, n_done & 1, abort_flag, status, 61);       // P may be overwritten, K P_m may be read
+            ++n_done;
+            ok = __syncthreads_and(ok);
+        }
+        if (!ok) break;
+        tc_fence_after();
+        // this thread's row: k' = k + g sum_m alpha_m (K P_m)[row]
+        // (the tensor-memory loads are warp-wide instructions: every lane of a warp that has a highlighted row
+        // takes part in them, only the update of the row itself depends on the lane's own flag)
+        if (__any_sync(0xffffffffu, hl)) {
+#pragma unroll 1
+            for (int c = 0; c < D / 32; ++c) {
+                float dk[32];
+#pragma unroll
+                for (int e = 0; e < 32; ++e) dk[e] = 0.f;
+                for (int m = 0; m < M; ++m) {
+                    const float cm = g * (alpha != nullptr ? alpha[((size_t)b * Hkv + h) * M + m] : 1.f);
+                    uint32_t v[32];
+                    tmem_ld32(t_lane + (uint32_t)m * D + c * 32, v);
+                    tmem_wait_ld_on(v);
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) dk[e] = fmaf(cm, __uint_as_float(v[e]), dk[e]);
+                }
+                if (hl) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {      // 8 elements = one 16-byte unit of the swizzled row
+                        const int col = c * 32 + q * 8;
+                        uint4* ptr = reinterpret_cast<uint4*>(sK + (col >> 6) * EBLK + sw128_offset(tid, col & 63));
+                        uint4 kv = *ptr;
+                        uint32_t* w = reinterpret_cast<uint32_t*>(&kv);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float2 k2 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&w[e]));
+                            w[e] = pack_bf16(k2.x + dk[q * 8 + 2 * e], k2.y + dk[q * 8 + 2 * e + 1]);
+                        }
+                        *ptr = kv;
+                    }
+                }
+                __syncwarp();      // all lanes together again before the next warp-wide load
+            }
+        }
+        tc_fence_before();
+        __syncthreads();
+        // write the highlighted rows out: D / 8 lanes per row, 16 bytes each
+        constexpr int LPR = D / 8, RPI = 32 / LPR;
+#pragma unroll 1
+        for (int i = 0; i < 32 / RPI; ++i) {
+            const int row = warp * 32 + i * RPI + lane / LPR, col = (lane % LPR) * 8;
+            if (flags[row]) {
+                const uint4 v = *reinterpret_cast<const uint4*>(sK + (col >> 6) * EBLK + sw128_offset(row, col & 63));
+                *reinterpret_cast<uint4*>(K_out + ((size_t)(seq0 + t * 128 + row) * Hkv + h) * D + col) = v;
+            }
+        }
+        __syncthreads();        // the tile and the flags are reused by the next step
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        __syncwarp();
+        tmem_dealloc(tmem_base, tmem_cols);
+    }
+}
+
+template <int D>
+static seka_status launch_edit_tiles(const seka_shape* s, const WorkspaceLayout& w, const void* K_in, void* K_out,
+                                     const uint8_t* mask, const float* U, const float* alpha, const float* gain,
+                                     const uint8_t* he, char* ws, cudaStream_t st) {
+    using SL = EditSmem<D>;
+    static bool configured = false;
+    static int n_sm = 0;
+    if (!configured) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm <= 0) return SEKA_ERR_CUDA;
+        if (cudaFuncSetAttribute(edit_tiles_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SL::DYN_BYTES) != cudaSuccess)
+            return SEKA_ERR_CUDA;
+        configured = true;
+    }
+    int* status = reinterpret_cast<int*>(ws);
+    void* P = ws + w.w_off;
+    uint8_t* tile_hot = reinterpret_cast<uint8_t*>(ws + w.hot_off);
+    int* hot_list = reinterpret_cast<int*>(ws + w.list_off);
+    launch_prep_edit(s, U, mask, P, tile_hot, w.n_tiles, hot_list, status + 2, st);
+    const int T = shape_total_tokens(s), Hkv = s->n_kv_heads, M = s->n_experts;
+    CUtensorMap tk, tp;
+    if (!make_tile_map(&tk, K_in, D, Hkv, T) || !make_tile_map(&tp, P, D, 1, (long long)2 * M * Hkv * D, D)) return SEKA_ERR_CUDA;
+    uint32_t cols = 32;
+    while (cols < (uint32_t)(M * D)) cols *= 2;
+    const int per_sm = (int)(512 / cols) < 3 ? (int)(512 / cols) : 3;          // tensor memory and shared memory per SM
+    const long long work_max = (long long)s->batch * w.n_tiles * Hkv;
+    const long long want = (long long)n_sm * per_sm;
+    const unsigned grid = (unsigned)(work_max < want ? work_max : want);
+    edit_tiles_kernel<D><<<grid, 128, SL::DYN_BYTES, st>>>(tk, tp, static_cast<__nv_bfloat16*>(K_out), mask, alpha, gain, he,
+                                                         s->cu_seqlens, hot_list, status + 2, status, s->max_seqlen, Hkv, M,
+                                                         w.n_tiles, cols);
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? SEKA_OK : SEKA_ERR_CUDA;
+}
+
 }  // namespace seka
 
 extern "C" seka_status seka_edit_keys(const seka_shape* shape, const void* K_in, void* K_out, const uint8_t* mask,
@@ -114,6 +312,13 @@ extern "C" seka_status seka_edit_keys(const seka_shape* shape, const void* K_in,
     if (K_out != K_in) {
         const size_t bytes = (size_t)T * shape->n_kv_heads * shape->head_dim * esz;
         if (cudaMemcpyAsync(K_out, K_in, bytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return SEKA_ERR_CUDA;
+    }
+    // bf16 tensors go through the tensor-core tile kernel (the projector products of all experts have to fit
+    // into tensor memory); fp32 tensors, and banks too large for that, take the fp32 row kernel
+    if (shape->dtype == SEKA_BF16 && (long long)shape->n_experts * shape->head_dim <= 512 && ((uintptr_t)workspace & 255) == 0) {
+        if (shape->head_dim == 128)
+            return launch_edit_tiles<128>(shape, w, K_in, K_out, mask, U, alpha, gain, head_enable, ws, st);
+        return launch_edit_tiles<64>(shape, w, K_in, K_out, mask, U, alpha, gain, head_enable, ws, st);
     }
     launch_compact_mask(mask, T, list, status + 2, st);
     if (shape->dtype == SEKA_F32)

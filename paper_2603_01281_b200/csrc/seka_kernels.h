@@ -16,6 +16,12 @@ void launch_build_items(const seka_shape* s, const WorkspaceLayout& w, bool stee
 void launch_compact_mask(const uint8_t* mask, int T, int* list, int* count, cudaStream_t st);
 void launch_convert_bf16(const float* in, void* out, size_t n, cudaStream_t st);
 
+void launch_prep_edit(const seka_shape* s, const float* U, const uint8_t* mask, void* P, uint8_t* tile_hot, int n_tiles,
+                      int* hot_list, int* hot_count, cudaStream_t st);
+
+// bf16 tensor [T, H, d] viewed as (d, H, T) for TMA: tiles of 64 x 1 x box_rows with the 128-byte swizzle.
+bool make_tile_map(CUtensorMap* m, const void* base, int d, int H, long long T, int box_rows = 128);
+
 seka_status validate_shape(const seka_shape* s);
 
 }  // namespace seka

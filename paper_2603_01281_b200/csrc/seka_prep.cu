@@ -64,6 +64,68 @@ __global__ void prep_steering_kernel(const float* __restrict__ U, const float* _
     }
 }
 
+// Operand preparation of the stand-alone edit, one launch:
+//   blocks [0, n_p):   a 32 x 32 tile of the projector P[m][h] = U_m[h] U_m[h]^T (bf16 [D x D], as a high and a low
+//                      part: [M, Hkv] matrices of high parts, then as many of low parts); gain and routing
+//                      coefficients are applied per row when dK is added, so this does not depend on the batch;
+//   blocks [n_p, ...): one warp per (sequence, 128-key tile): flag, and the tiles that hold a highlighted token
+//                      appended to `hot_list` (any order).
+__global__ void prep_edit_kernel(const float* __restrict__ U, const uint8_t* __restrict__ mask,
+                                 const int* __restrict__ cu_seqlens, __nv_bfloat16* __restrict__ P,
+                                 uint8_t* __restrict__ tile_hot, int* __restrict__ hot_list, int* __restrict__ hot_count,
+                                 int B, int L, int Hkv, int D, int r, int M, int n_tiles, int n_p) {
+    const int tid = threadIdx.x;
+    if ((int)blockIdx.x < n_p) {
+        const int tiles = D / 32;
+        const int mh = blockIdx.x / (tiles * tiles), t = blockIdx.x % (tiles * tiles);
+        const int i0 = (t / tiles) * 32, j0 = (t % tiles) * 32;
+        __shared__ float ui[32][33], uj[32][33];
+        const int tx = tid & 31, ty = tid >> 5;
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        const float* Um = U + (size_t)mh * D * r;          // U is [M, Hkv, D, r]: (m, h) pairs are consecutive
+        for (int k0 = 0; k0 < r; k0 += 32) {
+            __syncthreads();
+            for (int q = ty; q < 32; q += 8) {
+                const bool in = k0 + tx < r;
+                ui[q][tx] = in ? Um[(size_t)(i0 + q) * r + k0 + tx] : 0.f;
+                uj[q][tx] = in ? Um[(size_t)(j0 + q) * r + k0 + tx] : 0.f;
+            }
+            __syncthreads();
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int i = ty + 8 * q;
+#pragma unroll 8
+                for (int k = 0; k < 32; ++k) acc[q] = fmaf(ui[i][k], uj[tx][k], acc[q]);
+            }
+        }
+        // two bf16 parts, P = hi + lo to about 2^-17: the edit keeps fp32-like accuracy on bf16 tensor cores
+        __nv_bfloat16* Phi = P + (size_t)mh * D * D;
+        __nv_bfloat16* Plo = P + ((size_t)M * Hkv + mh) * D * D;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const __nv_bfloat16 hi = __float2bfloat16_rn(acc[q]);
+            Phi[(size_t)(i0 + ty + 8 * q) * D + j0 + tx] = hi;
+            Plo[(size_t)(i0 + ty + 8 * q) * D + j0 + tx] = __float2bfloat16_rn(acc[q] - __bfloat162float(hi));
+        }
+    } else {
+        const int item = ((int)blockIdx.x - n_p) * 8 + (tid >> 5), lane = tid & 31;
+        if (item >= B * n_tiles) return;
+        const int b = item / n_tiles, t = item % n_tiles;
+        const int seq0 = cu_seqlens ? cu_seqlens[b] : b * L;
+        const int Lb = (cu_seqlens ? cu_seqlens[b + 1] : (b + 1) * L) - seq0;
+        bool any = false;
+        for (int q = 0; q < 4; ++q) {
+            const int pos = t * 128 + q * 32 + lane;
+            any = any || (pos < Lb && mask[seq0 + pos] != 0);
+        }
+        any = __any_sync(0xffffffffu, any);
+        if (lane == 0) {
+            tile_hot[item] = any ? 1 : 0;
+            if (any) hot_list[atomicAdd(hot_count, 1)] = item;
+        }
+    }
+}
+
 // Item table of the fused kernel: slot idx (heaviest row tiles first; the items of one (sequence, KV head)
 // next to each other) decoded into an ItemRecord.  Returns false for a slot whose tiles lie beyond the
 // sequence.
@@ -168,6 +230,18 @@ void launch_prep_steering(const seka_shape* sh, const float* U, const float* alp
                                                       static_cast<__nv_bfloat16*>(W), tile_hot, sh->batch,
                                                       sh->max_seqlen, sh->n_kv_heads, D, sh->rank, sh->n_experts,
                                                       n_tiles, n_w);
+    ++g_launches;
+}
+
+void launch_prep_edit(const seka_shape* sh, const float* U, const uint8_t* mask, void* P, uint8_t* tile_hot, int n_tiles,
+                      int* hot_list, int* hot_count, cudaStream_t st) {
+    const int D = sh->head_dim, tiles = D / 32;
+    const int n_p = sh->n_experts * sh->n_kv_heads * tiles * tiles;
+    const int n_flag = (sh->batch * n_tiles + 7) / 8;
+    cudaMemsetAsync(hot_count, 0, sizeof(int), st);
+    prep_edit_kernel<<<n_p + n_flag, 256, 0, st>>>(U, mask, sh->cu_seqlens, static_cast<__nv_bfloat16*>(P), tile_hot, hot_list,
+                                                  hot_count, sh->batch, sh->max_seqlen, sh->n_kv_heads, D, sh->rank,
+                                                  sh->n_experts, n_tiles, n_p);
     ++g_launches;
 }
 

@@ -13,6 +13,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2603_01281_b200 import binding, inputs
 
 import helpers as H
@@ -43,7 +44,14 @@ def test_static_scratch_edit_matches_workspace_edit_twice():
         got, ref = _both(w)
         assert np.isfinite(got).all()
         rowmax = np.abs(ref).max(axis=-1, keepdims=True)
-        assert (np.abs(got - ref) / rowmax).max() <= 2.0 ** -8          # the edit tolerance of the other tests
+        # The other tests hold an edited bf16 key to 2^-8 of its row maximum against the exact edit.  The two
+        # entry points no longer share their arithmetic (row kernel in fp32 here, tensor-core tiles there), so
+        # each is held to that bound against the fp64 oracle, and to twice it against the other.
+        exact = oracle.edit_keys(w.K, w.mask, w.cu_seqlens, w.U, gain=w.gain)
+        emax = np.abs(exact).max(axis=-1, keepdims=True)
+        assert (np.abs(got - exact) / emax).max() <= 2.0 ** -8
+        assert (np.abs(ref - exact) / emax).max() <= 2.0 ** -8
+        assert (np.abs(got - ref) / rowmax).max() <= 2.0 ** -7
         hl = w.mask != 0
         assert np.array_equal(got[~hl], w.K[~hl].astype(np.float64))    # untouched rows stay bit-identical
 
