@@ -114,6 +114,44 @@ def cpu_oracle_sample(w, budget_s: float, seed: int = 0):
     return flops, secs, nrows
 
 
+def edit_keys_bench(w, peaks, layers: int = 36, steps: int = 20):
+    """Stand-alone key edit on a layer-stacked key cache [layers * B, L, Hkv, d] (bf16, in place): the hook of
+    Algorithm 1 applied to the cached keys of every layer of an 8B-shaped model in one launch.  Returns achieved
+    GB/s on the algorithmic bytes (highlighted rows read and written once, the mask read once) at two densities."""
+    import torch
+    from paper_2603_01281_b200 import binding
+    out = {}
+    B, L, Hkv, d = layers * w.batch, w.max_seqlen, w.n_kv_heads, w.head_dim
+    gen = torch.Generator(device="cuda"); gen.manual_seed(260301281)
+    K = torch.randn((B * L, Hkv, d), device="cuda", dtype=torch.float32, generator=gen).to(torch.bfloat16)
+    U = torch.from_numpy(w.U).cuda(); gain = torch.ones(B, device="cuda")
+    shp = binding.make_shape(batch=B, max_seqlen=L, n_q_heads=w.n_q_heads, n_kv_heads=Hkv, head_dim=d, rank=w.rank,
+                             n_experts=1, dtype=torch.bfloat16)
+    ws = binding.new_workspace(shp)
+    masks = {"10pct_spans": torch.from_numpy(np.tile(w.mask, layers)).cuda(),
+             "100pct": torch.ones(B * L, dtype=torch.uint8, device="cuda")}
+    for name, mask in masks.items():
+        n_h = int(mask.sum().item())
+        alg_bytes = 2.0 * n_h * Hkv * d * 2 + B * L + U.numel() * 4
+        for _ in range(3):
+            binding.seka_edit_keys(shp, K, K, mask, U, None, gain, None, ws)
+        torch.cuda.synchronize()
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            binding.seka_edit_keys(shp, K, K, mask, U, None, gain, None, ws)
+        e1.record(); torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / steps
+        gbs = alg_bytes / (ms * 1e-3) / 1e9
+        out[name] = {"ms": ms, "GB/s": gbs, "frac_of_hbm_peak": gbs / peaks["hbm_gbs"], "algorithmic_MB": alg_bytes / 1e6,
+                     "highlighted_tokens": n_h}
+        K.normal_(generator=gen)      # the edit multiplies the steered component every call: start from fresh keys
+    st = binding.seka_poll_status(ws)
+    out["status"] = binding.status_string(st)
+    out["cache"] = "bf16 [%d layers x %d, %d, %d, %d] = %.2f GB, in place" % (layers, w.batch, L, Hkv, d, K.numel() * 2 / 1e9)
+    return out
+
+
 def run_reference(args, rank: int):
     """The reference arm: the CPU oracle on a bounded sample of the same workload, K timed steps."""
     if rank != 0:
@@ -148,6 +186,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle work for cpu_baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-edit-bench", action="store_true", help="skip the stand-alone key-edit measurement")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -218,16 +257,20 @@ def main():
     if st != binding.SEKA_OK:
         raise SystemExit("device status: " + binding.status_string(st))
 
-    # the same kernel with steering off (g = 0 path): blocks of 20 steps of either kind alternate, so that clock
-    # and temperature drift under the power cap falls on both alike
+    # the same kernel with steering off (g = 0 path): single steps of either kind alternate, each between its own
+    # pair of events, so that clock and temperature drift under the power cap falls on both alike
     for _ in range(3):
         step(False)
-    ms0 = ms1 = 0.0
-    n_blocks = max(2, args.steps // 20)
-    for _ in range(n_blocks):
-        t, _, _ = timed(20, False); ms0 += t
-        t, _, _ = timed(20, True); ms1 += t
-    ms0 *= args.steps / (20.0 * n_blocks); ms1 *= args.steps / (20.0 * n_blocks)
+    n_alt = max(10, min(args.steps, 100))
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(2 * n_alt + 1)]
+    barrier()
+    evs[0].record()
+    for i in range(n_alt):
+        step(False); evs[2 * i + 1].record()
+        step(True); evs[2 * i + 2].record()
+    barrier()
+    ms0 = sum(evs[2 * i].elapsed_time(evs[2 * i + 1]) for i in range(n_alt)) / n_alt * args.steps
+    ms1 = sum(evs[2 * i + 1].elapsed_time(evs[2 * i + 2]) for i in range(n_alt)) / n_alt * args.steps
 
     # end to end through the host-buffer entry point: H2D of Q, K, V, mask and D2H of O every step
     staging = torch.empty(binding.seka_host_staging_bytes(shp), dtype=torch.uint8, device="cuda")
@@ -248,6 +291,10 @@ def main():
     if world > 1:
         t = torch.tensor([e2e_ms], device="cuda"); dist.all_reduce(t, op=dist.ReduceOp.MAX); e2e_ms = float(t.item())
     h2d = sum(t.numel() * t.element_size() for t in (hQ, hK, hV, hmask)); d2h = hO.numel() * hO.element_size()
+
+    edit_res = None
+    if rank == 0 and world == 1 and not args.no_edit_bench:
+        edit_res = edit_keys_bench(w, measured_peaks())
 
     if rank == 0:
         peaks = measured_peaks()
@@ -273,6 +320,8 @@ def main():
                       "ms_per_step_g0": ms0 / args.steps, "ms_per_step_steered": ms1 / args.steps,
                       "overhead_vs_g0": ms1 / ms0 - 1.0, "flops_per_step": flops_step},
         }
+        if edit_res is not None:
+            line["extra"]["edit_keys"] = edit_res
         if world == 1 and not args.no_cpu_baseline:
             import oracle
             f, s, r = cpu_oracle_sample(w, args.cpu_budget)

@@ -140,6 +140,42 @@ template <> __device__ __forceinline__ void store_chunk32<float>(float* dst, con
                             __uint_as_float(v[4 * c + 2]) * inv, __uint_as_float(v[4 * c + 3]) * inv);
 }
 
+// Adds dK (fp32, tensor memory, one key row per lane) to this thread's row of a staged K tile for the 32-column
+// chunks [c0, c1); rows whose flag is clear are left alone.  The tensor-memory loads are warp-wide: every lane
+// takes part in them whatever its flag.  The four 16-byte units of a chunk are read before any is written back
+// (a store followed by a load of the same array would keep the updates strictly in sequence).
+__device__ __forceinline__ void drain_edit(uint32_t tE, uint8_t* sK, int row, bool hl, int c0, int c1) {
+#pragma unroll 1
+    for (int c = c0; c < c1; ++c) {
+        uint32_t dk[32];
+        tmem_ld32(tE + c * 32, dk);
+        tmem_wait_ld_on(dk);
+        if (hl) {
+            uint4* ptr[4];
+            uint4 kv[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {      // 8 elements = one 16-byte unit of the swizzled row
+                const int col = c * 32 + q * 8;
+                ptr[q] = reinterpret_cast<uint4*>(sK + (col >> 6) * (128 * 128) + sw128_offset(row, col & 63));
+                kv[q] = *ptr[q];
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                uint32_t* w = reinterpret_cast<uint32_t*>(&kv[q]);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float2 k2 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&w[e]));
+                    const float2 s2 = __fadd2_rn(k2, make_float2(__uint_as_float(dk[q * 8 + 2 * e]), __uint_as_float(dk[q * 8 + 2 * e + 1])));
+                    w[e] = pack_bf16(s2.x, s2.y);
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) *ptr[q] = kv[q];
+        }
+        __syncwarp();      // all lanes together again before the next warp-wide load
+    }
+}
+
 // One unit of work of a CTA: two 128-row query tiles that share a KV head of one sequence.
 struct Item {
     int b, hkv, seq0, Lb;
@@ -171,7 +207,7 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     uint64_t* o_full = p_last + 2;           // [2]   last P V of tile x finished
     uint64_t* w_full = o_full + 2;           // [1]   edit operator landed
     uint64_t* e_full = w_full + 1;           // [1]   dK = K W of the current highlighted tile is in tensor memory
-    uint64_t* k_edited = e_full + 1;         // [1]   4 editor-warp arrivals: the staged tile now holds K'
+    uint64_t* k_edited = e_full + 1;         // [1]   4 editor-warp + 4 softmax-warp arrivals: the staged tile now holds K'
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + SL::MISC);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + SL::MISC + 4);
 
@@ -251,7 +287,7 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         mbar_init(q_full + 0, 1); mbar_init(q_full + 1, 1); mbar_init(k0_full, 1);
         for (int i = 0; i < NK; ++i) { mbar_init(kv_full + i, 1); mbar_init(kv_free + i, 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(s_full + i, 1); mbar_init(p_full + i, 5); mbar_init(p_last + i, 4); mbar_init(o_full + i, 1); }
-        mbar_init(w_full, 1); mbar_init(e_full, 1); mbar_init(k_edited, 4);
+        mbar_init(w_full, 1); mbar_init(e_full, 1); mbar_init(k_edited, 8);
         *abort_flag = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
@@ -524,28 +560,7 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     tc_fence_after();
                     const uint32_t tE = t_lane + COL_S + 128 * (j < it.nA ? 0 : 1);
                     uint8_t* sK = smem + SL::K + ((pr + (uint32_t)j) % NK) * SL::TILE;
-#pragma unroll 1
-                    for (int c = 0; c < D / 32; ++c) {
-                        uint32_t dk[32];
-                        tmem_ld32(tE + c * 32, dk);
-                        tmem_wait_ld_on(dk);
-                        if (hl) {
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) {      // 8 elements = one 16-byte unit of the swizzled row
-                                const int col = c * 32 + q * 8;
-                                uint4* ptr = reinterpret_cast<uint4*>(sK + (col >> 6) * BLK_BYTES + sw128_offset(row, col & 63));
-                                uint4 kv = *ptr;
-                                uint32_t* w = reinterpret_cast<uint32_t*>(&kv);
-#pragma unroll
-                                for (int e = 0; e < 4; ++e) {
-                                    const float2 k2 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&w[e]));
-                                    w[e] = pack_bf16(k2.x + __uint_as_float(dk[q * 8 + 2 * e]), k2.y + __uint_as_float(dk[q * 8 + 2 * e + 1]));
-                                }
-                                *ptr = kv;
-                            }
-                        }
-                        __syncwarp();      // all lanes together again before the next warp-wide load
-                    }
+                    drain_edit(tE, sK, row, hl, 0, D / 64);      // the other half of the columns is taken by the idle softmax warps
                     fence_proxy_async();       // the rewritten rows are read next by the tensor core
                     tc_fence_before();
                     __syncwarp();
@@ -563,14 +578,39 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         const uint32_t tS = t_lane + COL_S + 128 * x, tO = t_lane + COL_O + D * x;
         const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
         uint32_t cX = 0, n_o = 0;       // steps and items of this tile so far
+        uint32_t pr = 0, n_hot = 0;     // V/K pairs and highlighted key tiles so far (all items)
         bool ok = true;
         while (ok && next_item(it)) {
             const int nX = x ? it.nB : it.nA;
             const int hqX = x ? it.hqB : it.hqA, qtX = x ? it.qtB : it.qtA;
-            if (nX == 0) continue;
+            const uint8_t* hot_g = p.tile_hot + (size_t)it.b * p.n_qt;
+            if (nX == 0) {      // tile B lies beyond the sequence: only the counts move
+                if (it.steer)
+                    for (int j = 0; j < it.n_kv; ++j) n_hot += hot_g[j] != 0 ? 1u : 0u;
+                pr += it.n_kv;
+                continue;
+            }
             float m_run = -INFINITY, l_run = 0.f;
 #pragma unroll 1
             for (int j = 0; j < nX; ++j) {
+                // Key tile j holds highlighted tokens and this tile is the first to use it: while waiting for its
+                // scores anyway, these warps add the upper half of the columns of dK to the staged K tile (the
+                // key editors take the lower half).  Every softmax warp counts the highlighted tiles.
+                if (it.steer && hot_g[j] != 0) {
+                    if ((j < it.nA ? 0 : 1) == x) {
+                        const int kpos = j * BN + row;
+                        const bool hl = kpos < it.Lb && p.mask[it.seq0 + kpos] != 0;
+                        ok = warp_wait(e_full, n_hot & 1, abort_flag, p.status, 36 + x);
+                        if (!ok) break;
+                        tc_fence_after();
+                        drain_edit(tS, smem + SL::K + ((pr + (uint32_t)j) % NK) * SL::TILE, row, hl, D / 64, D / 32);
+                        fence_proxy_async();
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(k_edited);
+                    }
+                    ++n_hot;
+                }
                 ok = warp_wait(s_full + x, (cX + j) & 1, abort_flag, p.status, 40 + x);
                 if (!ok) break;
                 tc_fence_after();
@@ -642,7 +682,10 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                 const float2 s2 = __fadd2_rn(sum[0], sum[1]);
                 l_run = l_run * factor + (s2.x + s2.y);
             }
-            cX += nX;
+            // highlighted tiles that only the other tile uses are counted too
+            if (it.steer)
+                for (int j = nX; j < it.n_kv; ++j) n_hot += hot_g[j] != 0 ? 1u : 0u;
+            cX += nX; pr += it.n_kv;
             if (ok) ok = warp_wait(o_full + x, n_o & 1, abort_flag, p.status, 44 + x);
             ++n_o;
             if (ok) {
