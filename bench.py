@@ -200,7 +200,7 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2603_01281_b200 import binding, inputs
+    from paper_2603_01281_b200 import binding, inputs, sharding
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
@@ -211,7 +211,7 @@ def main():
 
     sampler = ClockSampler(local_rank) if rank == 0 else None    # started early: nvidia-smi takes a while to come up
     # every rank: its own batch of the same shape (sequences are independent units)
-    w = inputs.make_workload("C2", seed_offset=rank)
+    w = inputs.make_workload("C2", seed_offset=sharding.rank_seed_offset(rank))
     dt = torch.bfloat16
     dev = {k: torch.from_numpy(getattr(w, k)).cuda().to(dt) for k in ("Q", "K", "V")}
     mask = torch.from_numpy(w.mask).cuda(); U = torch.from_numpy(w.U).cuda(); gain = torch.from_numpy(w.gain).cuda()
@@ -227,9 +227,7 @@ def main():
                                    U if steer else None, None, gain, None, ws)
 
     def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+        sharding.barrier(torch.cuda.synchronize)
 
     def timed(nsteps, steer=True):
         ev0 = torch.cuda.Event(enable_timing=True); ev1 = torch.cuda.Event(enable_timing=True)
@@ -241,9 +239,7 @@ def main():
         ev1.record()
         barrier()
         t1 = time.time()
-        ms = ev0.elapsed_time(ev1)
-        if world > 1:
-            t = torch.tensor([ms], device="cuda"); dist.all_reduce(t, op=dist.ReduceOp.MAX); ms = float(t.item())
+        ms = sharding.max_over_ranks(ev0.elapsed_time(ev1), "cuda")
         return ms, t0, t1
 
     for _ in range(args.warmup):
@@ -287,9 +283,7 @@ def main():
     for _ in range(e2e_steps):
         e2e_step()
     ev1.record(); barrier()
-    e2e_ms = ev0.elapsed_time(ev1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], device="cuda"); dist.all_reduce(t, op=dist.ReduceOp.MAX); e2e_ms = float(t.item())
+    e2e_ms = sharding.max_over_ranks(ev0.elapsed_time(ev1), "cuda")
     h2d = sum(t.numel() * t.element_size() for t in (hQ, hK, hV, hmask)); d2h = hO.numel() * hO.element_size()
 
     edit_res = None
@@ -299,7 +293,7 @@ def main():
     if rank == 0:
         peaks = measured_peaks()
         ms_step = ms / args.steps
-        value = world * flops_step * args.steps / (ms * 1e-3) / 1e12
+        value = sharding.whole_job_rate(flops_step, args.steps, ms, world) / 1e12
         per_gpu = value / world
         line = {
             "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
