@@ -93,28 +93,31 @@ static void launch_edit_rows(const seka_shape* s, const void* K_in, void* K_out,
 
 // ---------------------------------------------------------------- bf16 tensors: one 128-token tile per step, on tcgen05
 //
-// A CTA (4 warps, one key row per thread) takes the (highlighted tile, KV head) pairs of the hot-tile list in turn:
-// TMA stages the [128 x D] key tile and the projector P[m][h] = U_m U_m^T (two bf16 parts), the tensor core forms
-// K P_m in tensor memory (two products per expert), every thread adds  g_b sum_m alpha_{b,h,m} (K P_m)[row]  to its row in shared
-// memory if the row is highlighted, and the warps then write the highlighted rows out, 16 bytes per lane with the
-// lanes of a row next to each other.  Unhighlighted rows are never written.  Several CTAs share an SM (64 KB of
-// shared memory and M * D tensor-memory columns each), so loads, products and stores of different tiles overlap.
+// A CTA (8 warps) takes a contiguous run of the (KV head, highlighted tile) pairs, head-major, so that the projector
+// P[m][h] = U_m U_m^T (two bf16 parts, resident in shared memory) changes rarely: TMA stages the [128 x D] key tile,
+// the tensor core forms K P_m in tensor memory (two products per expert), every thread adds
+// g_b sum_m alpha_{b,h,m} (K P_m)[row] to half of its row in shared memory if the row is highlighted, and the warps
+// then write the highlighted rows out, 16 bytes per lane with the lanes of a row next to each other.
+// Unhighlighted rows are never written.  Two CTAs share an SM (96 KB of shared memory and M * D tensor-memory
+// columns each), so the loads, products and stores of different tiles overlap.
 constexpr uint32_t EBLK = 128 * 128;        // one [128 x 64] bf16 block
+constexpr int EDIT_THREADS = 256;
 
 template <int D>
 struct EditSmem {
     static constexpr uint32_t TILE = (D / 64) * EBLK;
     static constexpr uint32_t PBLK = D * 128;
+    static constexpr uint32_t PMAT = (D / 64) * PBLK;       // one D x D bf16 matrix
     static constexpr uint32_t K = 0;
-    static constexpr uint32_t P = K + TILE;
-    static constexpr uint32_t FLAGS = P + (D / 64) * PBLK;
+    static constexpr uint32_t P = K + TILE;                 // high part, then low part
+    static constexpr uint32_t FLAGS = P + 2 * PMAT;
     static constexpr uint32_t BARS = FLAGS + 128;
     static constexpr uint32_t MISC = BARS + 16;
     static constexpr uint32_t DYN_BYTES = MISC + 16 + 1024;
 };
 
 template <int D>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(EDIT_THREADS)
 edit_tiles_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmP,
                   __nv_bfloat16* __restrict__ K_out, const uint8_t* __restrict__ mask, const float* __restrict__ alpha,
                   const float* __restrict__ gain, const uint8_t* __restrict__ head_enable,
@@ -131,6 +134,7 @@ edit_tiles_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + SL::MISC);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + SL::MISC + 4);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int row = tid & 127, half = tid >> 7;      // key row of the tile, and which half of its columns this thread updates
     if (__syncthreads_or(*reinterpret_cast<volatile int*>(status) != 0)) return;
 
     if (tid == 0) {
@@ -145,63 +149,77 @@ edit_tiles_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_holder;
-    const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
+    const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
     constexpr uint32_t IDESC = umma_idesc_bf16(D, false);
     constexpr uint32_t DESC_HI = umma_desc_hi_sw128(1024);
     const uint32_t dK = umma_desc_lo(smem_u32(sK), 16), dP = umma_desc_lo(smem_u32(smem + SL::P), 16);
 
-    const long long n_work = (long long)(*hot_count) * Hkv;
+    const int n_hot = *hot_count;
+    const long long n_work = (long long)n_hot * Hkv;
+    const long long per = (n_work + gridDim.x - 1) / gridDim.x;
+    const long long w0 = (long long)blockIdx.x * per, w1 = w0 + per < n_work ? w0 + per : n_work;
     uint32_t n_full = 0, n_done = 0;
+    int resident = -1;          // (m, h) pair whose projector is in shared memory: m * Hkv + h
     bool ok = true;
-    for (long long idx = blockIdx.x; idx < n_work && ok; idx += gridDim.x) {
-        const int tile = hot_list[idx / Hkv], h = (int)(idx % Hkv);
+    for (long long idx = w0; idx < w1 && ok; ++idx) {
+        const int h = (int)(idx / n_hot), tile = hot_list[idx % n_hot];
         const int b = tile / n_tiles, t = tile % n_tiles;
         const float g = gain[b];
         if (g == 0.f || (head_enable != nullptr && head_enable[h] == 0)) continue;      // same for the whole CTA
         const int seq0 = cu_seqlens ? cu_seqlens[b] : b * L;
         const int Lb = (cu_seqlens ? cu_seqlens[b + 1] : (b + 1) * L) - seq0;
-        const int kpos = t * 128 + tid;
+        const int kpos = t * 128 + row;
         const bool hl = kpos < Lb && mask[seq0 + kpos] != 0;
-        flags[tid] = hl ? 1 : 0;
-        // 2 M products: the high and the low part of every projector accumulate into the same columns
-        for (int mm = 0; mm < 2 * M && ok; ++mm) {
-            const int m = mm >> 1, part = mm & 1;
-            if (tid == 0) {
-                mbar_expect_tx(full, (mm == 0 ? SL::TILE : 0u) + NBLK * SL::PBLK);
-                if (mm == 0) {
+        if (half == 0) flags[row] = hl ? 1 : 0;
+        for (int m = 0; m < M && ok; ++m) {
+            const bool load_p = resident != m * Hkv + h;
+            if (m == 0 || load_p) {
+                if (tid == 0) {
+                    mbar_expect_tx(full, (m == 0 ? SL::TILE : 0u) + (load_p ? 2 * SL::PMAT : 0u));
+                    if (m == 0) {
 #pragma unroll
-                    for (int c = 0; c < NBLK; ++c) tma_load_3d(sK + c * EBLK, &tmK, full, c * 64, h, seq0 + t * 128);
+                        for (int c = 0; c < NBLK; ++c) tma_load_3d(sK + c * EBLK, &tmK, full, c * 64, h, seq0 + t * 128);
+                    }
+                    if (load_p) {
+#pragma unroll
+                        for (int part = 0; part < 2; ++part)
+#pragma unroll
+                            for (int c = 0; c < NBLK; ++c)
+                                tma_load_3d(smem + SL::P + part * SL::PMAT + c * SL::PBLK, &tmP, full, c * 64, 0,
+                                            ((part * M + m) * Hkv + h) * D);
+                    }
                 }
-#pragma unroll
-                for (int c = 0; c < NBLK; ++c)
-                    tma_load_3d(smem + SL::P + c * SL::PBLK, &tmP, full, c * 64, 0, ((part * M + m) * Hkv + h) * D);
+                resident = m * Hkv + h;
+                ok = mbar_wait(full, n_full & 1, abort_flag, status, 60);
+                ++n_full;
+                ok = __syncthreads_and(ok);
+                if (!ok) break;
             }
-            ok = mbar_wait(full, n_full & 1, abort_flag, status, 60);
-            ++n_full;
-            ok = __syncthreads_and(ok);
-            if (!ok) break;
             if (tid == 0) {
                 tc_fence_after();
+                // the high and the low part of the projector accumulate into the same columns
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint32_t offk = ((uint32_t)(ks >> 2) * EBLK + (uint32_t)(ks & 3) * 32) >> 4;
-                    const uint32_t offp = ((uint32_t)(ks >> 2) * SL::PBLK + (uint32_t)(ks & 3) * 32) >> 4;
-                    umma_ss(tmem_base + (uint32_t)m * D, dK + offk, DESC_HI, dP + offp, DESC_HI, IDESC, (ks > 0 || part) ? 1u : 0u);
-                }
+                for (int part = 0; part < 2; ++part)
+#pragma unroll
+                    for (int ks = 0; ks < D / 16; ++ks) {
+                        const uint32_t offk = ((uint32_t)(ks >> 2) * EBLK + (uint32_t)(ks & 3) * 32) >> 4;
+                        const uint32_t offp = ((uint32_t)part * SL::PMAT + (uint32_t)(ks >> 2) * SL::PBLK + (uint32_t)(ks & 3) * 32) >> 4;
+                        umma_ss(tmem_base + (uint32_t)m * D, dK + offk, DESC_HI, dP + offp, DESC_HI, IDESC, (ks > 0 || part) ? 1u : 0u);
+                    }
                 umma_commit(done);
             }
-            ok = mbar_wait(done, n_done & 1, abort_flag, status, 61);       // P may be overwritten, K P_m may be read
+            ok = mbar_wait(done, n_done & 1, abort_flag, status, 61);       // the projector may be replaced, K P_m may be read
             ++n_done;
             ok = __syncthreads_and(ok);
         }
         if (!ok) break;
         tc_fence_after();
-        // this thread's row: k' = k + g sum_m alpha_m (K P_m)[row]
+        // this thread's half row: k' = k + g sum_m alpha_m (K P_m)[row]
         // (the tensor-memory loads are warp-wide instructions: every lane of a warp that has a highlighted row
         // takes part in them, only the update of the row itself depends on the lane's own flag)
         if (__any_sync(0xffffffffu, hl)) {
 #pragma unroll 1
-            for (int c = 0; c < D / 32; ++c) {
+            for (int c = half * (D / 64); c < (half + 1) * (D / 64); ++c) {
                 float dk[32];
 #pragma unroll
                 for (int e = 0; e < 32; ++e) dk[e] = 0.f;
@@ -214,33 +232,39 @@ edit_tiles_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
                     for (int e = 0; e < 32; ++e) dk[e] = fmaf(cm, __uint_as_float(v[e]), dk[e]);
                 }
                 if (hl) {
+                    uint4* ptr[4];
+                    uint4 kv[4];
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {      // 8 elements = one 16-byte unit of the swizzled row
+                    for (int q = 0; q < 4; ++q) {      // 8 elements = one 16-byte unit of the swizzled row; reads before writes
                         const int col = c * 32 + q * 8;
-                        uint4* ptr = reinterpret_cast<uint4*>(sK + (col >> 6) * EBLK + sw128_offset(tid, col & 63));
-                        uint4 kv = *ptr;
-                        uint32_t* w = reinterpret_cast<uint32_t*>(&kv);
+                        ptr[q] = reinterpret_cast<uint4*>(sK + (col >> 6) * EBLK + sw128_offset(row, col & 63));
+                        kv[q] = *ptr[q];
+                    }
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        uint32_t* w = reinterpret_cast<uint32_t*>(&kv[q]);
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const float2 k2 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&w[e]));
                             w[e] = pack_bf16(k2.x + dk[q * 8 + 2 * e], k2.y + dk[q * 8 + 2 * e + 1]);
                         }
-                        *ptr = kv;
                     }
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) *ptr[q] = kv[q];
                 }
                 __syncwarp();      // all lanes together again before the next warp-wide load
             }
         }
         tc_fence_before();
         __syncthreads();
-        // write the highlighted rows out: D / 8 lanes per row, 16 bytes each
+        // write the highlighted rows out: D / 8 lanes per row, 16 bytes each; 16 rows per warp
         constexpr int LPR = D / 8, RPI = 32 / LPR;
 #pragma unroll 1
-        for (int i = 0; i < 32 / RPI; ++i) {
-            const int row = warp * 32 + i * RPI + lane / LPR, col = (lane % LPR) * 8;
-            if (flags[row]) {
-                const uint4 v = *reinterpret_cast<const uint4*>(sK + (col >> 6) * EBLK + sw128_offset(row, col & 63));
-                *reinterpret_cast<uint4*>(K_out + ((size_t)(seq0 + t * 128 + row) * Hkv + h) * D + col) = v;
+        for (int i = 0; i < 16 / RPI; ++i) {
+            const int r = warp * 16 + i * RPI + lane / LPR, col = (lane % LPR) * 8;
+            if (flags[r]) {
+                const uint4 v = *reinterpret_cast<const uint4*>(sK + (col >> 6) * EBLK + sw128_offset(r, col & 63));
+                *reinterpret_cast<uint4*>(K_out + ((size_t)(seq0 + t * 128 + r) * Hkv + h) * D + col) = v;
             }
         }
         __syncthreads();        // the tile and the flags are reused by the next step
@@ -278,11 +302,11 @@ static seka_status launch_edit_tiles(const seka_shape* s, const WorkspaceLayout&
     if (!make_tile_map(&tk, K_in, D, Hkv, T) || !make_tile_map(&tp, P, D, 1, (long long)2 * M * Hkv * D, D)) return SEKA_ERR_CUDA;
     uint32_t cols = 32;
     while (cols < (uint32_t)(M * D)) cols *= 2;
-    const int per_sm = (int)(512 / cols) < 3 ? (int)(512 / cols) : 3;          // tensor memory and shared memory per SM
+    const int per_sm = (int)(512 / cols) < 2 ? (int)(512 / cols) : 2;          // tensor memory and shared memory per SM
     const long long work_max = (long long)s->batch * w.n_tiles * Hkv;
     const long long want = (long long)n_sm * per_sm;
     const unsigned grid = (unsigned)(work_max < want ? work_max : want);
-    edit_tiles_kernel<D><<<grid, 128, SL::DYN_BYTES, st>>>(tk, tp, static_cast<__nv_bfloat16*>(K_out), mask, alpha, gain, he,
+    edit_tiles_kernel<D><<<grid, EDIT_THREADS, SL::DYN_BYTES, st>>>(tk, tp, static_cast<__nv_bfloat16*>(K_out), mask, alpha, gain, he,
                                                          s->cu_seqlens, hot_list, status + 2, status, s->max_seqlen, Hkv, M,
                                                          w.n_tiles, cols);
     ++g_launches;
