@@ -22,6 +22,9 @@
  *    kernels compute U (U^T k)).  alpha is fp32 [B, Hkv, M] or NULL (all ones).
  *    gain is fp32 [B] (any sign, zero allowed).  head_enable is uint8 [Hkv] or NULL
  *    (all heads steered).
+ *  - The two-projector edit of Eq. 4, k' = k + (g+ P+ k + g- P- k) / 2 with P+ from the leading k+ vectors and
+ *    P- from the vectors after the leading k- ones (Eq. 2), is the same blend with two "experts":
+ *    U_1 = U+[:, :k+], U_2 = U-[:, k-:] (zero-padded to a common r), alpha = (g+/2, g-/2), gain = 1.
  *  - Calls are asynchronous on `cuda_stream` (a cudaStream_t passed as void*).
  *    Argument errors are returned before anything is launched.  A device-side wait
  *    that runs out (every wait in the kernels is bounded) records SEKA_ERR_TIMEOUT in

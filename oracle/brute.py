@@ -79,3 +79,36 @@ def attention_logit_bias(Q, K, V, mask, U, alpha=None, g=1.0, head_enable=None, 
         O[:, hq, :] = P @ V[:, h, :]
         LSE[:, hq] = lse
     return O, LSE
+
+
+def two_projector_edit(K, mask, U_pos, k_pos, U_neg, k_neg, g_pos, g_neg, head_enable=None):
+    """The general SEKA key edit, Eq. 4 with the projectors of Eq. 2, on one sequence (K is [L, Hkv, d]):
+
+        P+ = U+[:, :k+] U+[:, :k+]^T          (leading k+ left-singular vectors of the positive cross-covariance)
+        P- = U-[:, k-:] U-[:, k-:]^T          (the vectors AFTER the leading k- ones of the negative cross-covariance)
+        k' = k + (g+ P+ k + g- P- k) / 2      at highlighted tokens, other tokens untouched.
+
+    U_pos and U_neg are [Hkv, d, d] (full orthogonal factors, one per KV head); k_pos and k_neg are the ranks chosen
+    by the variance criterion of Eq. 3.  Dense d x d projectors, fp64, no shortcuts.
+    """
+    K = np.asarray(K, dtype=np.float64)
+    out = K.copy()
+    hl = np.asarray(mask) != 0
+    for h in range(K.shape[1]):
+        if head_enable is not None and not head_enable[h]:
+            continue
+        Up = np.asarray(U_pos[h], dtype=np.float64)[:, :k_pos]
+        Un = np.asarray(U_neg[h], dtype=np.float64)[:, k_neg:]
+        P_pos = Up @ Up.T
+        P_neg = Un @ Un.T
+        for t in np.nonzero(hl)[0]:
+            k = K[t, h]
+            out[t, h] = k + (g_pos * (P_pos @ k) + g_neg * (P_neg @ k)) / 2.0
+    return out
+
+
+def rank_by_variance(S, gamma):
+    """Eq. 3: the smallest k whose leading singular values hold at least the fraction gamma of their sum."""
+    S = np.asarray(S, dtype=np.float64)
+    c = np.cumsum(S) / np.sum(S)
+    return int(np.searchsorted(c, gamma - 1e-15) + 1)

@@ -210,3 +210,46 @@ def test_fused_full_size_sampled_rows(name, nrows):
     mx, mean = H.check_attention(O[idx], Oref, name, kappa=kappa)
     np.testing.assert_allclose(LSE[idx], Lref, atol=2e-2)
     print("%s: rows %d max abs %.3e mean abs %.3e" % (name, len(idx), mx, mean))
+
+
+# ----------------------------------------------------------------- the two-projector edit of Eq. 4 through the bank interface
+
+def test_two_projector_edit_maps_onto_the_expert_bank():
+    """Eq. 4, k' = k + (g+ P+ k + g- P- k)/2 with P- built from the vectors after the leading k- ones (Eq. 2), is
+    the blend sum_m alpha_m U_m U_m^T of two "experts": U_1 = U+[:, :k+], U_2 = U-[:, k-:] (zero-padded to a
+    common width), alpha = (g+/2, g-/2), gain 1.  Edited keys and fused attention against the dense oracle."""
+    from oracle import brute
+    d, Hq, Hkv, L = 128, 4, 2, 300
+    w = inputs.make_custom(seed=21, dtype="bf16", lens=[L], n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, rank=8,
+                           gain=1.0, mask_kind="runs", highlight=0.25)
+    rng = np.random.default_rng(22)
+    Up = np.stack([np.linalg.qr(rng.standard_normal((d, d)))[0] for _ in range(Hkv)])
+    Un = np.stack([np.linalg.qr(rng.standard_normal((d, d)))[0] for _ in range(Hkv)])
+    k_pos, k_neg, g_pos, g_neg = 12, 100, 0.6, -0.4
+    r = max(k_pos, d - k_neg)
+    bank = np.zeros((2, Hkv, d, r), dtype=np.float32)
+    bank[0, :, :, :k_pos] = Up[:, :, :k_pos]
+    bank[1, :, :, :d - k_neg] = Un[:, :, k_neg:]
+    alpha = np.tile(np.array([g_pos / 2, g_neg / 2]), (1, Hkv, 1))
+    # the oracle consumes the bank as stored (fp32), like the kernels
+    K_ref = brute.two_projector_edit(w.K, w.mask, bank[0].astype(np.float64)[:, :, :], k_pos,
+                                     np.concatenate([np.zeros((Hkv, d, k_neg)), bank[1].astype(np.float64)[:, :, :d - k_neg]], axis=2),
+                                     k_neg, g_pos, g_neg)
+    dev = H.device_tensors(w)
+    dev["U"] = torch.from_numpy(bank).cuda()
+    shp = binding.make_shape(batch=1, max_seqlen=L, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=d, rank=r, n_experts=2,
+                             dtype=torch.bfloat16)
+    ws = binding.new_workspace(shp)
+    a = torch.from_numpy(alpha.astype(np.float32)).cuda()
+    Kout = torch.full_like(dev["K"], float("nan"))
+    binding.seka_edit_keys(shp, dev["K"], Kout, dev["mask"], dev["U"], a, dev["gain"], None, ws)
+    got = Kout.double().cpu().numpy()
+    rel = np.abs(got - K_ref) / np.abs(K_ref).max(axis=-1, keepdims=True)
+    assert rel.max() <= 2.0 ** -8, rel.max()
+    hl = w.mask != 0
+    assert np.array_equal(got[~hl], w.K[~hl].astype(np.float64))
+    O = torch.full_like(dev["Q"], float("nan"))
+    binding.seka_attention_fwd(shp, dev["Q"], dev["K"], dev["V"], O, None, dev["mask"], dev["U"], a, dev["gain"], None, ws)
+    assert binding.seka_poll_status(ws) == binding.SEKA_OK
+    Oref, _, idx = oracle.attention_rows(w.Q.astype(np.float64), K_ref, w.V.astype(np.float64), w.cu_seqlens, None)
+    H.check_attention(O.double().cpu().numpy()[idx], Oref, "two projectors")

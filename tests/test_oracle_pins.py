@@ -250,3 +250,51 @@ def test_blend_factor_form_equals_dense_projector():
     a = oracle.route(w.Q, w.cu_seqlens, w.U, w.sigma, 0)
     Kp = oracle.edit_keys(w.K, w.mask, w.cu_seqlens, w.U, alpha=a, gain=w.gain)
     np.testing.assert_allclose(Kp, brute.edited_keys(w.K, w.mask, w.U, a[0], float(w.gain[0])), atol=1e-12)
+
+
+# ----------------------------------------------------------------- two-projector edit (Eq. 2-4)
+
+def _two_bases(seed, Hkv, d):
+    rng = np.random.default_rng(seed)
+    Up = np.stack([np.linalg.qr(rng.standard_normal((d, d)))[0] for _ in range(Hkv)])
+    Un = np.stack([np.linalg.qr(rng.standard_normal((d, d)))[0] for _ in range(Hkv)])
+    return Up, Un
+
+
+def test_two_projector_edit_closed_forms():
+    from oracle import brute
+    d, Hkv, L = 16, 2, 12
+    Up, Un = _two_bases(5, Hkv, d)
+    rng = np.random.default_rng(6)
+    mask = np.zeros(L, dtype=np.uint8); mask[[1, 4, 5, 11]] = 1
+    k_pos, k_neg, gp, gn = 3, 10, 0.8, -0.6
+    # a key inside span(U+[:, :k+]) and orthogonal to span(U-[:, k-:]) is scaled by (1 + g+/2); build one by projecting
+    h = 0
+    Pn = Un[h][:, k_neg:] @ Un[h][:, k_neg:].T
+    Pp = Up[h][:, :k_pos] @ Up[h][:, :k_pos].T
+    K = rng.standard_normal((L, Hkv, d))
+    out = brute.two_projector_edit(K, mask, Up, k_pos, Un, k_neg, gp, gn)
+    hl = mask != 0
+    assert np.array_equal(out[~hl], K[~hl])                                   # untouched rows
+    for t in np.nonzero(hl)[0]:
+        k = K[t, h]
+        np.testing.assert_allclose(out[t, h], k + 0.5 * gp * Pp @ k + 0.5 * gn * Pn @ k, atol=1e-13)
+        # components: along a leading positive vector the edit adds g+/2 of it (plus what P- sees of it)
+        u = Up[h][:, 0]
+        np.testing.assert_allclose(u @ out[t, h], u @ k + 0.5 * gp * (u @ k) + 0.5 * gn * (u @ (Pn @ k)), atol=1e-13)
+    # g- = 0 reduces to the single-projector edit with gain g+/2 (checked against the C oracle)
+    out1 = brute.two_projector_edit(K, mask, Up, k_pos, Un, k_neg, gp, 0.0)
+    ref = oracle.edit_keys(K, mask, [0, L], Up[None, :, :, :k_pos], gain=gp / 2)
+    np.testing.assert_allclose(out1, ref, atol=1e-13)
+    # k- = 0 and g+ = 0: P- is the identity, every highlighted key is scaled by (1 + g-/2)
+    out2 = brute.two_projector_edit(K, mask, Up, k_pos, Un, 0, 0.0, gn)
+    np.testing.assert_allclose(out2[hl], (1 + gn / 2) * K[hl], atol=1e-13)
+    # the trailing vectors are used, not the leading ones: swapping them changes the result
+    out3 = brute.two_projector_edit(K, mask, Up, k_pos, Un[:, :, ::-1], k_neg, gp, gn)
+    assert np.abs(out3 - out).max() > 1e-3
+
+
+def test_rank_by_variance_rule():
+    from oracle import brute
+    S = np.array([4.0, 3.0, 2.0, 1.0])            # cumulative fractions 0.4, 0.7, 0.9, 1.0
+    assert [brute.rank_by_variance(S, g) for g in (0.3, 0.4, 0.41, 0.7, 0.9, 0.95, 1.0)] == [1, 1, 2, 2, 3, 4, 4]
