@@ -101,6 +101,12 @@ static void launch_edit_rows(const seka_shape* s, const void* K_in, void* K_out,
 // Unhighlighted rows are never written.  Two CTAs share an SM (96 KB of shared memory and M * D tensor-memory
 // columns each), so the loads, products and stores of different tiles overlap.
 constexpr uint32_t EBLK = 128 * 128;        // one [128 x 64] bf16 block
+
+// all lanes of a warp wait on the same barrier and then agree on the outcome
+__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status, int where) {
+    const bool ok = mbar_wait(bar, parity, abort_flag, status, where);
+    return __all_sync(0xffffffffu, ok);
+}
 constexpr int EDIT_THREADS = 256;
 
 template <int D>
@@ -277,6 +283,256 @@ edit_tiles_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     }
 }
 
+// ---------------------------------------------------------------- single projector (plain SEKA): the same work as a pipeline
+//
+// One persistent CTA per SM with three roles, so that several key tiles are in flight per SM and the tensor-core
+// product of one tile runs under the drain and write-out of the one before:
+//   warp 8   producer: walks this CTA's run of (KV head, highlighted tile) pairs, stages key tiles through a ring of
+//            NS shared-memory stages by TMA, writes the rows' highlight flags and the tile's coordinates beside them,
+//            and (re)loads the projector when the head changes (after the ring has drained);
+//   warp 9   MMA issuer: K P (two bf16 parts) into one of two sets of tensor-memory columns;
+//   warps 0-7  drain: half a key row per thread, k' = k + c (K P)[row] into the staged tile for highlighted rows,
+//            then the highlighted rows go out 16 bytes per lane; the stage and the columns are handed back.
+constexpr int EP_NS = 4;                      // key tiles in flight per SM
+constexpr int EP_THREADS = 320;
+
+struct EpMeta { int tok0, h, valid, p_gen; float c; int pad[3]; };     // per stage: first token, head, end marker, projector generation, g * alpha
+
+template <int D>
+struct EpSmem {
+    static constexpr uint32_t TILE = (D / 64) * EBLK;
+    static constexpr uint32_t PBLK = D * 128;
+    static constexpr uint32_t PMAT = (D / 64) * PBLK;
+    static constexpr uint32_t K = 0;                        // EP_NS stages
+    static constexpr uint32_t P = K + EP_NS * TILE;         // high part, then low part
+    static constexpr uint32_t FLAGS = P + 2 * PMAT;         // EP_NS x 128 bytes
+    static constexpr uint32_t META = FLAGS + EP_NS * 128;   // EP_NS x 32 bytes
+    static constexpr uint32_t BARS = META + EP_NS * 32;     // full[NS], free[NS], mma_done[2], cols_free[2], p_full, meet[2]
+    static constexpr uint32_t NBARS = 2 * EP_NS + 7;
+    static constexpr uint32_t MISC = BARS + NBARS * 8;
+    static constexpr uint32_t DYN_BYTES = MISC + 16 + 1024;
+};
+
+template <int D>
+__global__ void __launch_bounds__(EP_THREADS, 1)
+edit_tiles_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmP,
+                       __nv_bfloat16* __restrict__ K_out, const uint8_t* __restrict__ mask, const float* __restrict__ alpha,
+                       const float* __restrict__ gain, const uint8_t* __restrict__ head_enable,
+                       const int* __restrict__ cu_seqlens, const int* __restrict__ hot_list, const int* __restrict__ hot_count,
+                       int* status, int L, int Hkv, int n_tiles) {
+    using SL = EpSmem<D>;
+    constexpr int NBLK = D / 64;
+    constexpr uint32_t TMEM_COLS = 2 * D < 32 ? 32 : 2 * D;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SL::BARS);
+    uint64_t* full = bars;                     // [NS]  tile landed (TMA bytes) and flags / coordinates written (producer)
+    uint64_t* freeb = full + EP_NS;            // [NS]  8 drain-warp arrivals: the stage may be refilled
+    uint64_t* mma_done = freeb + EP_NS;        // [2]   K P of a tile is in column set c
+    uint64_t* cols_free = mma_done + 2;        // [2]   8 drain-warp arrivals: column set c has been read
+    uint64_t* p_full = cols_free + 2;          // [1]   projector landed
+    uint64_t* meetb = p_full + 1;              // [2]   8 drain-warp arrivals: all rows of the tile are updated
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + SL::MISC);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + SL::MISC + 4);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (__syncthreads_or(*reinterpret_cast<volatile int*>(status) != 0)) return;
+
+    if (tid == 0) {
+        for (int i = 0; i < EP_NS; ++i) { mbar_init(full + i, 2); mbar_init(freeb + i, 8); }
+        for (int i = 0; i < 2; ++i) { mbar_init(mma_done + i, 1); mbar_init(cols_free + i, 8); mbar_init(meetb + i, 8); }
+        mbar_init(p_full, 1);
+        *abort_flag = 0;
+        mbar_fence_init();
+        tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmP);
+    }
+    __syncwarp();
+    if (warp == 0) { tmem_alloc(tmem_holder, TMEM_COLS); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_holder;
+
+    if (warp == 8) {
+        // ------------------------------------------------------------ producer
+        const int n_hot = *hot_count;
+        const long long n_work = (long long)n_hot * Hkv;
+        const long long per = (n_work + gridDim.x - 1) / gridDim.x;
+        long long w0 = (long long)blockIdx.x * per;
+        if (w0 > n_work) w0 = n_work;                 // a CTA without work still pushes the end marker
+        const long long w1 = w0 + per < n_work ? w0 + per : n_work;
+        uint32_t n_push = 0;      // stages filled so far
+        int p_gen = 0, cur_h = -1;
+        bool ok = true;
+        for (long long idx = w0; idx <= w1 && ok; ++idx) {
+            const bool last = idx >= w1;                    // one more stage after the work: the end marker
+            int h = 0, tile = 0, b = 0, t = 0, seq0 = 0, Lb = 0;
+            float c = 0.f;
+            if (!last) {
+                h = (int)(idx / n_hot); tile = hot_list[idx % n_hot];
+                b = tile / n_tiles; t = tile % n_tiles;
+                const float g = gain[b];
+                if (g == 0.f || (head_enable != nullptr && head_enable[h] == 0)) continue;
+                c = g * (alpha != nullptr ? alpha[(size_t)b * Hkv + h] : 1.f);
+                seq0 = cu_seqlens ? cu_seqlens[b] : b * L;
+                Lb = (cu_seqlens ? cu_seqlens[b + 1] : (b + 1) * L) - seq0;
+                if (h != cur_h) {
+                    // the projector changes: every tile of the old head must be through the tensor core (here: the
+                    // whole ring handed back), then the new one is loaded
+                    for (uint32_t q = n_push >= EP_NS ? n_push - EP_NS : 0; q < n_push && ok; ++q)
+                        ok = warp_wait(freeb + q % EP_NS, (q / EP_NS) & 1, abort_flag, status, 62);
+                    if (!ok) break;
+                    if (lane == 0) {
+                        mbar_expect_tx(p_full, 2 * SL::PMAT);
+#pragma unroll
+                        for (int part = 0; part < 2; ++part)
+#pragma unroll
+                            for (int cb = 0; cb < NBLK; ++cb)
+                                tma_load_3d(smem + SL::P + part * SL::PMAT + cb * SL::PBLK, &tmP, p_full, cb * 64, 0, (part * Hkv + h) * D);
+                    }
+                    __syncwarp();
+                    cur_h = h; ++p_gen;
+                }
+            }
+            const uint32_t s = n_push % EP_NS;
+            if (n_push >= EP_NS) {
+                ok = warp_wait(freeb + s, ((n_push / EP_NS) - 1) & 1, abort_flag, status, 63);
+                if (!ok) break;
+            }
+            uint8_t* fl = smem + SL::FLAGS + s * 128;
+            if (!last) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int kpos = t * 128 + q * 32 + lane;
+                    fl[q * 32 + lane] = (kpos < Lb && mask[seq0 + kpos] != 0) ? 1 : 0;
+                }
+            }
+            if (lane == 0) {
+                EpMeta* m = reinterpret_cast<EpMeta*>(smem + SL::META + s * 32);
+                m->tok0 = seq0 + t * 128; m->h = h; m->valid = last ? 0 : 1; m->p_gen = p_gen; m->c = c;
+                if (!last) {
+                    mbar_expect_tx(full + s, SL::TILE);
+#pragma unroll
+                    for (int cb = 0; cb < NBLK; ++cb) tma_load_3d(smem + SL::K + s * SL::TILE + cb * EBLK, &tmK, full + s, cb * 64, h, seq0 + t * 128);
+                } else {
+                    mbar_arrive(full + s);
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(full + s);       // second arrival: flags and coordinates are in place
+            ++n_push;
+        }
+    } else if (warp == 9) {
+        // ------------------------------------------------------------ MMA issuer
+        constexpr uint32_t IDESC = umma_idesc_bf16(D, false);
+        constexpr uint32_t DESC_HI = umma_desc_hi_sw128(1024);
+        const uint32_t dK = umma_desc_lo(smem_u32(smem + SL::K), 16), dP = umma_desc_lo(smem_u32(smem + SL::P), 16);
+        int seen_gen = 0;
+        bool ok = true;
+        for (uint32_t n = 0; ok; ++n) {
+            const uint32_t s = n % EP_NS, cset = n & 1;
+            ok = warp_wait(full + s, (n / EP_NS) & 1, abort_flag, status, 64);
+            if (!ok) break;
+            const EpMeta m = *reinterpret_cast<const EpMeta*>(smem + SL::META + s * 32);
+            if (!m.valid) break;
+            if (m.p_gen != seen_gen) {
+                ok = warp_wait(p_full, (uint32_t)(m.p_gen - 1) & 1, abort_flag, status, 65);
+                if (!ok) break;
+                seen_gen = m.p_gen;
+            }
+            if (n >= 2) {
+                ok = warp_wait(cols_free + cset, ((n >> 1) - 1) & 1, abort_flag, status, 66);
+                if (!ok) break;
+            }
+            tc_fence_after();
+            if (lane == 0) {
+                const uint32_t kd = dK + s * (SL::TILE >> 4);
+#pragma unroll
+                for (int part = 0; part < 2; ++part)
+#pragma unroll
+                    for (int ks = 0; ks < D / 16; ++ks) {
+                        const uint32_t offk = ((uint32_t)(ks >> 2) * EBLK + (uint32_t)(ks & 3) * 32) >> 4;
+                        const uint32_t offp = ((uint32_t)part * SL::PMAT + (uint32_t)(ks >> 2) * SL::PBLK + (uint32_t)(ks & 3) * 32) >> 4;
+                        umma_ss(tmem_base + cset * D, kd + offk, DESC_HI, dP + offp, DESC_HI, IDESC, (ks > 0 || part) ? 1u : 0u);
+                    }
+                umma_commit(mma_done + cset);
+            }
+            __syncwarp();
+        }
+    } else if (warp < 8) {
+        // ------------------------------------------------------------ drain and write-out
+        const int row = tid & 127, half = tid >> 7;
+        const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+        bool ok = true;
+        for (uint32_t n = 0; ok; ++n) {
+            const uint32_t s = n % EP_NS, cset = n & 1;
+            ok = warp_wait(full + s, (n / EP_NS) & 1, abort_flag, status, 67);
+            if (!ok) break;
+            const EpMeta m = *reinterpret_cast<const EpMeta*>(smem + SL::META + s * 32);
+            if (!m.valid) break;
+            uint8_t* sK = smem + SL::K + s * SL::TILE;
+            const uint8_t* fl = smem + SL::FLAGS + s * 128;
+            const bool hl = fl[row] != 0;
+            ok = warp_wait(mma_done + cset, (n >> 1) & 1, abort_flag, status, 68);
+            if (!ok) break;
+            tc_fence_after();
+            // (the tensor-memory loads are warp-wide: every lane takes part, only the row update depends on the flag)
+            if (__any_sync(0xffffffffu, hl)) {
+#pragma unroll 1
+                for (int c = half * (D / 64); c < (half + 1) * (D / 64); ++c) {
+                    uint32_t v[32];
+                    tmem_ld32(t_lane + cset * D + c * 32, v);
+                    tmem_wait_ld_on(v);
+                    if (hl) {
+                        uint4* ptr[4];
+                        uint4 kv[4];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {      // 8 elements = one 16-byte unit of the swizzled row; reads before writes
+                            const int col = c * 32 + q * 8;
+                            ptr[q] = reinterpret_cast<uint4*>(sK + (col >> 6) * EBLK + sw128_offset(row, col & 63));
+                            kv[q] = *ptr[q];
+                        }
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            uint32_t* w = reinterpret_cast<uint32_t*>(&kv[q]);
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const float2 k2 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&w[e]));
+                                w[e] = pack_bf16(fmaf(m.c, __uint_as_float(v[q * 8 + 2 * e]), k2.x), fmaf(m.c, __uint_as_float(v[q * 8 + 2 * e + 1]), k2.y));
+                            }
+                        }
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) *ptr[q] = kv[q];
+                    }
+                    __syncwarp();      // all lanes together again before the next warp-wide load
+                }
+            }
+            // the columns are read: the next product may use them; all rows updated: the tile may be written out
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) { mbar_arrive(cols_free + cset); mbar_arrive(meetb + cset); }
+            ok = warp_wait(meetb + cset, (n >> 1) & 1, abort_flag, status, 69);
+            if (!ok) break;
+            constexpr int LPR = D / 8, RPI = 32 / LPR;
+#pragma unroll 1
+            for (int i = 0; i < 16 / RPI; ++i) {
+                const int r = warp * 16 + i * RPI + lane / LPR, col = (lane % LPR) * 8;
+                if (fl[r]) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(sK + (col >> 6) * EBLK + sw128_offset(r, col & 63));
+                    *reinterpret_cast<uint4*>(K_out + ((size_t)(m.tok0 + r) * Hkv + m.h) * D + col) = v;
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(freeb + s);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        __syncwarp();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
 template <int D>
 static seka_status launch_edit_tiles(const seka_shape* s, const WorkspaceLayout& w, const void* K_in, void* K_out,
                                      const uint8_t* mask, const float* U, const float* alpha, const float* gain,
@@ -300,6 +556,22 @@ static seka_status launch_edit_tiles(const seka_shape* s, const WorkspaceLayout&
     const int T = shape_total_tokens(s), Hkv = s->n_kv_heads, M = s->n_experts;
     CUtensorMap tk, tp;
     if (!make_tile_map(&tk, K_in, D, Hkv, T) || !make_tile_map(&tp, P, D, 1, (long long)2 * M * Hkv * D, D)) return SEKA_ERR_CUDA;
+    if (M == 1) {
+        using PL = EpSmem<D>;
+        static bool configured_p = false;
+        if (!configured_p) {
+            if (cudaFuncSetAttribute(edit_tiles_pipe_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PL::DYN_BYTES) != cudaSuccess)
+                return SEKA_ERR_CUDA;
+            configured_p = true;
+        }
+        const long long work = (long long)s->batch * w.n_tiles * Hkv;
+        const unsigned gridp = (unsigned)(work < (long long)n_sm ? work : (long long)n_sm);
+        edit_tiles_pipe_kernel<D><<<gridp, EP_THREADS, PL::DYN_BYTES, st>>>(tk, tp, static_cast<__nv_bfloat16*>(K_out), mask, alpha, gain, he,
+                                                                          s->cu_seqlens, hot_list, status + 2, status, s->max_seqlen,
+                                                                          Hkv, w.n_tiles);
+        ++g_launches;
+        return cudaGetLastError() == cudaSuccess ? SEKA_OK : SEKA_ERR_CUDA;
+    }
     uint32_t cols = 32;
     while (cols < (uint32_t)(M * D)) cols *= 2;
     const int per_sm = (int)(512 / cols) < 2 ? (int)(512 / cols) : 2;          // tensor memory and shared memory per SM
