@@ -194,6 +194,10 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     constexpr int NBLK = D / 64;
     constexpr uint32_t TMEM_COLS = 512;
     constexpr uint32_t COL_S = 0, COL_O = 256;     // S_x at COL_S + 128 x, O_x at COL_O + D x
+    // head_dim 64 leaves 128 columns unused: dK of a highlighted key tile gets columns of its own there and is
+    // formed while the previous step's P V runs; head_dim 128 has to borrow the idle score columns of a tile
+    constexpr bool EDIT_OWN_COLS = (D == 64);
+    constexpr uint32_t COL_E = 384;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SL::BARS);
@@ -408,7 +412,7 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     if (!w_seen) { ok = warp_wait(w_full, n_w & 1, abort_flag, p.status, 31); w_seen = true; }
                     if (!ok) return;
                     const uint32_t kd = dK + ((pr + (uint32_t)j) % NK) * (SL::TILE >> 4);
-                    const uint32_t dst = tmem_base + COL_S + 128 * x;
+                    const uint32_t dst = tmem_base + (EDIT_OWN_COLS ? COL_E : COL_S + 128 * x);
                     tc_fence_after();
                     if (leader) {
 #pragma unroll
@@ -420,6 +424,10 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                         umma_commit(e_full);
                     }
                     __syncwarp();
+                };
+                // ... and the wait for the rows to be updated, kept apart: with columns of its own the product can be
+                // issued a good while before the edited tile is needed
+                auto edit_done = [&]() {
                     ok = warp_wait(k_edited, n_hot & 1, abort_flag, p.status, 32);
                     ++n_hot;
                 };
@@ -462,7 +470,7 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                 ok = warp_wait(q_full + 0, n_it & 1, abort_flag, p.status, 20);
                 if (ok && nB > 0) ok = warp_wait(q_full + 1, n_qb & 1, abort_flag, p.status, 21);
                 if (ok) ok = warp_wait(k0_full, n_it & 1, abort_flag, p.status, 22);
-                if (ok) edit_K(0, 0, hot_cur);
+                if (ok && hot_cur) { edit_K(0, 0, true); if (ok) edit_done(); }
                 if (ok) {
                     issue_S(0, 0);
                     if (nB > 0) issue_S(1, 0);
@@ -484,12 +492,17 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     if (j < nA) {
                         ok = warp_wait(p_full + 0, (cx[0] + j) & 1, abort_flag, p.status, 24);
                         if (!ok) break;
+                        if (EDIT_OWN_COLS && hot_j1 && j1 < nA) edit_K(0, j1, true);      // K(j1) has landed (the relay vouches), P_A V hides the drain
+                        if (!ok) break;
                         issue_PV(0, j, 0, 6, false);
                         ok = warp_wait(p_last + 0, (cx[0] + j) & 1, abort_flag, p.status, 28);
                         if (!ok) break;
                         issue_PV(0, j, 6, 8, j == nA - 1);
                         if (j1 < nA) {
-                            edit_K(0, j1, hot_j1);
+                            if (hot_j1) {
+                                if (!EDIT_OWN_COLS) edit_K(0, j1, true);
+                                if (ok) edit_done();
+                            }
                             if (!ok) break;
                             issue_S(0, j1);
                         }
@@ -503,7 +516,10 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                         issue_PV(1, j, 6, 8, j == nB - 1);
                     }
                     if (j1 < nB) {
-                        if (j1 >= nA) edit_K(1, j1, hot_j1);      // tile A does not use this key tile: B is its first user
+                        if (j1 >= nA && hot_j1) {      // tile A does not use this key tile: B is its first user
+                            edit_K(1, j1, true);
+                            if (ok) edit_done();
+                        }
                         if (!ok) break;
                         issue_S(1, j1);
                     }
@@ -558,7 +574,7 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     if (!ok) break;
                     ++n_hot;
                     tc_fence_after();
-                    const uint32_t tE = t_lane + COL_S + 128 * (j < it.nA ? 0 : 1);
+                    const uint32_t tE = t_lane + (EDIT_OWN_COLS ? COL_E : COL_S + 128 * (j < it.nA ? 0 : 1));
                     uint8_t* sK = smem + SL::K + ((pr + (uint32_t)j) % NK) * SL::TILE;
                     drain_edit(tE, sK, row, hl, 0, D / 64);      // the other half of the columns is taken by the idle softmax warps
                     fence_proxy_async();       // the rewritten rows are read next by the tensor core
@@ -603,7 +619,7 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                         ok = warp_wait(e_full, n_hot & 1, abort_flag, p.status, 36 + x);
                         if (!ok) break;
                         tc_fence_after();
-                        drain_edit(tS, smem + SL::K + ((pr + (uint32_t)j) % NK) * SL::TILE, row, hl, D / 64, D / 32);
+                        drain_edit(EDIT_OWN_COLS ? t_lane + COL_E : tS, smem + SL::K + ((pr + (uint32_t)j) % NK) * SL::TILE, row, hl, D / 64, D / 32);
                         fence_proxy_async();
                         tc_fence_before();
                         __syncwarp();
