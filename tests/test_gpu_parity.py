@@ -253,3 +253,26 @@ def test_two_projector_edit_maps_onto_the_expert_bank():
     assert binding.seka_poll_status(ws) == binding.SEKA_OK
     Oref, _, idx = oracle.attention_rows(w.Q.astype(np.float64), K_ref, w.V.astype(np.float64), w.cu_seqlens, None)
     H.check_attention(O.double().cpu().numpy()[idx], Oref, "two projectors")
+
+
+# ----------------------------------------------------------------- wide banks and many items per CTA
+
+def test_wide_expert_banks():
+    """Stacked rank M*r above the head dimension (the dense operator does not care), and a bank too large for the
+    tensor-core edit kernel (M*d > 512), which takes the fp32 row kernel."""
+    for M, r in [(3, 64), (5, 16)]:
+        w = inputs.make_custom(seed=50 + M, dtype="bf16", lens=[260, 130], n_q_heads=4, n_kv_heads=2, head_dim=128, rank=r,
+                               n_experts=M, gain=[0.5, -0.5], highlight=0.3)
+        alpha = np.random.default_rng(M).uniform(-1, 1, size=(w.batch, w.n_kv_heads, M))
+        _check_edit(w, H.run_edit(w, alpha=alpha), alpha=alpha)
+        _fused_vs_oracle(w, alpha=alpha, label="M%d r%d" % (M, r), short_rows=True)
+
+
+def test_more_items_than_sms():
+    """Fixed-length batch with more (row-tile, head-pair) items than the GPU has SMs: every persistent CTA walks
+    several items (odd and even rounds), with steering on some sequences only and one KV head switched off."""
+    w = inputs.make_custom(seed=60, dtype="bf16", lens=[2432, 2432], n_q_heads=8, n_kv_heads=2, head_dim=128, rank=16,
+                           gain=[1.0, 0.0], highlight=0.2)
+    he = np.array([1, 0], dtype=np.uint8)
+    rows = H.sampled_rows(w, 40, seed=3)
+    _fused_vs_oracle(w, head_enable=he, rows=rows, label="152 items")
