@@ -9,7 +9,10 @@ input is upcast to float64 and nothing is rounded afterwards.
 
 Functions follow the paper: ``route`` is Eq. 6 (Section 3.3), ``edit_keys`` is
 the hook of Algorithm 1/2 with k' = k + g P k (Section 2, Eq. 7), and
-``attention_rows`` is causal softmax attention with the score of Section 2.
+``attention_rows`` is causal softmax attention with the score of Section 2;
+``decode_attention`` is the attention of one generated token over the whole
+(already edited) key cache, the situation after the hook of Algorithm 1 has run
+"before generation".
 The reading of the routing query under GQA (sum over the group's query heads)
 is PARITY UNPINNED: the paper does not fix it.
 """
@@ -153,3 +156,39 @@ def seka_attention(Q, K, V, mask, cu_seqlens, U, alpha=None, gain=None, head_ena
     """The whole steered path: edit the highlighted keys, then causal attention."""
     Kp = edit_keys(K, mask, cu_seqlens, U, alpha, gain, head_enable)
     return attention_rows(Q, Kp, V, cu_seqlens, rows, scale)
+
+
+def decode_attention(q, Kp, V, cu_seqlens: Sequence[int], scale: Optional[float] = None):
+    """Attention of one new query token per sequence over its whole cache of (already edited) keys.
+
+    Algorithm 1 edits the prompt's keys once, before generation; every generated token then attends to
+    all cached tokens with the score of Section 2: for sequence b and query head h (KV head h // G)
+        O[b, h] = sum_j softmax_j(q[b, h] . k'_j * scale) v_j,   j over the sequence's cached tokens.
+    q is [B, Hq, d]; Kp and V are packed [T, Hkv, d].  Returns O [B, Hq, d] and LSE [B, Hq] (natural log);
+    a sequence without cached tokens gives O = 0 and LSE = -inf.  Written as the definition, in fp64.
+    """
+    q = _f64(q); Kp = _f64(Kp); V = _f64(V)
+    B, Hq, d = q.shape
+    Hkv = Kp.shape[1]
+    assert Hq % Hkv == 0 and len(cu_seqlens) == B + 1
+    G = Hq // Hkv
+    scale = 1.0 / np.sqrt(d) if not scale else float(scale)
+    O = np.zeros((B, Hq, d)); LSE = np.full((B, Hq), -np.inf)
+    for b in range(B):
+        s, e = int(cu_seqlens[b]), int(cu_seqlens[b + 1])
+        if e == s:
+            continue
+        for h in range(Hq):
+            logits = (Kp[s:e, h // G, :] @ q[b, h]) * scale
+            top = logits.max()
+            w = np.exp(logits - top)
+            den = w.sum()
+            O[b, h] = (w / den) @ V[s:e, h // G, :]
+            LSE[b, h] = top + np.log(den)
+    return O, LSE
+
+
+def seka_decode(q, K, V, mask, cu_seqlens, U, alpha=None, gain=None, head_enable=None, scale: Optional[float] = None):
+    """The decode path: edit the highlighted cached keys once, then one decode step over the edited cache."""
+    Kp = edit_keys(K, mask, cu_seqlens, U, alpha, gain, head_enable)
+    return decode_attention(q, Kp, V, cu_seqlens, scale)

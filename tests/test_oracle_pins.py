@@ -298,3 +298,101 @@ def test_rank_by_variance_rule():
     from oracle import brute
     S = np.array([4.0, 3.0, 2.0, 1.0])            # cumulative fractions 0.4, 0.7, 0.9, 1.0
     assert [brute.rank_by_variance(S, g) for g in (0.3, 0.4, 0.41, 0.7, 0.9, 0.95, 1.0)] == [1, 1, 2, 2, 3, 4, 4]
+
+
+# ----------------------------------------------------------------- decode step over the edited cache
+
+def _decode_case(seed=5, lens=(37, 1, 64), Hq=6, Hkv=2, d=16):
+    rng = np.random.default_rng(seed)
+    T = int(sum(lens))
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    q = rng.standard_normal((len(lens), Hq, d))
+    K = rng.standard_normal((T, Hkv, d))
+    V = rng.standard_normal((T, Hkv, d))
+    return q, K, V, cu
+
+
+def test_decode_hand_case_and_pure_python_loops():
+    # two cached tokens, scores 0 and ln 3 (scale 1/sqrt(4) = 1/2, q.k = 2 ln 3): weights 1/4 and 3/4
+    q = np.zeros((1, 1, 4)); q[0, 0, 0] = 2.0
+    K = np.zeros((2, 1, 4)); K[1, 0, 0] = math.log(3.0)
+    V = np.zeros((2, 1, 4)); V[0, 0, :] = 4.0; V[1, 0, :] = 8.0
+    O, LSE = oracle.decode_attention(q, K, V, [0, 2])
+    np.testing.assert_allclose(O[0, 0], 7.0, atol=1e-14)
+    np.testing.assert_allclose(LSE[0, 0], math.log(4.0), atol=1e-14)
+    # scalar loops on a tiny random case, GQA group of 3
+    q, K, V, cu = _decode_case(lens=(5, 3), Hq=6, Hkv=2, d=4)
+    O, LSE = oracle.decode_attention(q, K, V, cu)
+    for b in range(2):
+        for h in range(6):
+            num = [0.0] * 4; den = 0.0
+            for t in range(int(cu[b]), int(cu[b + 1])):
+                s = sum(q[b, h, c] * K[t, h // 3, c] for c in range(4)) / 2.0
+                den += math.exp(s)
+                for c in range(4):
+                    num[c] += math.exp(s) * V[t, h // 3, c]
+            np.testing.assert_allclose(O[b, h], [x / den for x in num], rtol=1e-12)
+            np.testing.assert_allclose(LSE[b, h], math.log(den), rtol=1e-12)
+
+
+def test_decode_is_the_last_row_of_causal_attention():
+    # a generated token that attends to its whole cache is the last row of causal attention
+    # (the C routine is a separate implementation)
+    q, K, V, cu = _decode_case()
+    Q = np.zeros((K.shape[0], q.shape[1], q.shape[2]))
+    for b in range(q.shape[0]):
+        Q[cu[b + 1] - 1] = q[b]
+    rows = [np.array([cu[b + 1] - cu[b] - 1]) for b in range(q.shape[0])]
+    O_ref, L_ref, _ = oracle.attention_rows(Q, K, V, cu, rows)
+    O, LSE = oracle.decode_attention(q, K, V, cu)
+    np.testing.assert_allclose(O, O_ref, rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(LSE, L_ref, rtol=1e-12, atol=1e-13)
+
+
+def test_decode_closed_forms():
+    q, K, V, cu = _decode_case()
+    O, LSE = oracle.decode_attention(q, K, V, cu)
+    B, Hq, d = q.shape
+    G = Hq // K.shape[1]
+    # equal keys: uniform weights, the output is the mean value and LSE = score + ln L
+    Ke = np.broadcast_to(K[:1], K.shape).copy()
+    Oe, Le = oracle.decode_attention(q, Ke, V, cu)
+    for b in range(B):
+        s, e = int(cu[b]), int(cu[b + 1])
+        for h in range(Hq):
+            np.testing.assert_allclose(Oe[b, h], V[s:e, h // G].mean(axis=0), rtol=1e-12, atol=1e-13)
+            np.testing.assert_allclose(Le[b, h], q[b, h] @ Ke[0, h // G] / math.sqrt(d) + math.log(e - s), rtol=1e-12)
+    # adding one vector c to every key shifts all scores of a head alike: O unchanged, LSE + q.c * scale
+    c = np.random.default_rng(9).standard_normal((K.shape[1], d))
+    Os, Ls = oracle.decode_attention(q, K + c[None], V, cu)
+    np.testing.assert_allclose(Os, O, rtol=1e-10, atol=1e-12)
+    shift = np.einsum("bhd,hd->bh", q, np.repeat(c, G, axis=0)) / math.sqrt(d)
+    np.testing.assert_allclose(Ls, LSE + shift, rtol=1e-12, atol=1e-12)
+    # one key far along q dominates: the output is that token's value
+    Kd = K.copy(); t = int(cu[0]) + 3
+    Kd[t, 0] = 200.0 * q[0, 0] / np.linalg.norm(q[0, 0])
+    Od, _ = oracle.decode_attention(q, Kd, V, cu)
+    np.testing.assert_allclose(Od[0, 0], V[t, 0], atol=1e-9)
+    # values enter linearly; a sequence with one cached token returns that token's value
+    O2, _ = oracle.decode_attention(q, K, 2.0 * V + 1.0, cu)
+    np.testing.assert_allclose(O2, 2.0 * O + 1.0, rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(O[1], np.repeat(V[cu[1]], G, axis=0), atol=1e-14)
+    # softmax scale override and an empty cache
+    O3, _ = oracle.decode_attention(q, K, V, cu, scale=0.5)
+    O4, _ = oracle.decode_attention(q * 0.5 * math.sqrt(d), K, V, cu)
+    np.testing.assert_allclose(O3, O4, rtol=1e-12, atol=1e-13)
+    Oz, Lz = oracle.decode_attention(q[:1], K[:0], V[:0], [0, 0])
+    assert np.all(Oz == 0) and np.all(np.isneginf(Lz))
+
+
+def test_decode_over_edited_cache_uses_edited_keys():
+    # highlighted tokens with the identity projector (full rank) have their scores multiplied by 1 + g (Eq. 12)
+    w = tiny(seed=4, L=40, d=8, r=8, gain=1.5)
+    q = np.random.default_rng(2).standard_normal((1, w.n_q_heads, w.head_dim))
+    U = np.broadcast_to(np.eye(8), (1, w.n_kv_heads, 8, 8)).copy()
+    O, LSE = oracle.seka_decode(q, w.K, w.V, w.mask, w.cu_seqlens, U, gain=w.gain)
+    Kp = w.K.astype(np.float64).copy()
+    Kp[w.mask != 0] *= 1.0 + 1.5
+    O_ref, L_ref = oracle.decode_attention(q, Kp, w.V, w.cu_seqlens)
+    np.testing.assert_allclose(O, O_ref, rtol=1e-10, atol=1e-12)
+    np.testing.assert_allclose(LSE, L_ref, rtol=1e-10, atol=1e-12)
