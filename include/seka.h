@@ -154,6 +154,25 @@ seka_status seka_edit_keys_static(const seka_shape* shape, const void* K_in, voi
                                   const uint8_t* mask, const float* U, const float* alpha,
                                   const float* gain, const uint8_t* head_enable, void* cuda_stream);
 
+/*
+ * One decode step over a cached key tensor whose highlighted keys have already been edited (Algorithm 1 runs the
+ * hook once, "before generation": seka_edit_keys in place on the prompt's keys; every generated token then
+ * attends to the whole cache with the score of Section 2).  For sequence b and query head h
+ *     O[b, h, :] = sum_j softmax_j(Q[b, h, :] . K[t_j, h / (Hq/Hkv), :] * scale) V[t_j, h / (Hq/Hkv), :]
+ * over the cached tokens t_j of sequence b (all of them: the new token's own key and value are the last
+ * cached row).  Q and O are bf16 [B, Hq, d] (one query token per sequence); K and V are the packed caches
+ * [T, Hkv, d] described above; lse, if not NULL, receives fp32 [B, Hq] (natural log).  A sequence without
+ * cached tokens gets O = 0 and lse = -inf.  K and V are read once and never written.
+ * Only SEKA_BF16, at most 16 query heads per KV head and at most 65535 sequences (SEKA_ERR_UNSUPPORTED
+ * otherwise); rank and n_experts of the shape are not used.  `workspace` holds the per-chunk partial results:
+ * seka_decode_workspace_bytes(shape) bytes, 256-byte aligned, its first 256 bytes the status block that
+ * seka_reset_status / seka_poll_status read.
+ */
+size_t seka_decode_workspace_bytes(const seka_shape* shape);
+seka_status seka_decode_attention(const seka_shape* shape, const void* Q, const void* K, const void* V,
+                                  void* O, float* lse, void* workspace, size_t workspace_bytes,
+                                  void* cuda_stream);
+
 /* Clears the device status word (async on the stream); call once before first use of a workspace. */
 seka_status seka_reset_status(void* workspace, void* cuda_stream);
 /* Synchronises the stream and returns the device status word (SEKA_OK if no wait ran out). */

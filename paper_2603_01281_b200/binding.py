@@ -20,7 +20,8 @@ SEKA_F32, SEKA_BF16 = 0, 1
 
 EXPORTS = ["seka_workspace_bytes", "seka_edit_keys", "adaseka_route", "seka_attention_fwd",
            "seka_host_staging_bytes", "seka_attention_fwd_host", "seka_reset_status", "seka_poll_status",
-           "seka_status_string", "seka_launch_count", "seka_edit_keys_static"]
+           "seka_status_string", "seka_launch_count", "seka_edit_keys_static", "seka_decode_workspace_bytes",
+           "seka_decode_attention"]
 SEKA_STATIC_MAX_TOKENS = 262144
 
 
@@ -62,6 +63,9 @@ def load() -> ctypes.CDLL:
         lib.seka_attention_fwd_host.argtypes = [sp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t,
                                                 vp, ctypes.c_size_t, vp]
         lib.seka_attention_fwd_host.restype = ctypes.c_int
+        lib.seka_decode_workspace_bytes.argtypes = [sp]; lib.seka_decode_workspace_bytes.restype = ctypes.c_size_t
+        lib.seka_decode_attention.argtypes = [sp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        lib.seka_decode_attention.restype = ctypes.c_int
         lib.seka_reset_status.argtypes = [vp, vp]; lib.seka_reset_status.restype = ctypes.c_int
         lib.seka_poll_status.argtypes = [vp, vp]; lib.seka_poll_status.restype = ctypes.c_int
         lib.seka_status_string.argtypes = [ctypes.c_int]; lib.seka_status_string.restype = ctypes.c_char_p
@@ -155,6 +159,17 @@ def seka_attention_fwd_host(shape: SekaShape, h_Q, h_K, h_V, h_O, h_lse, h_mask,
                                           _ptr(h_lse), _ptr(h_mask), _ptr(U), _ptr(alpha), _ptr(gain),
                                           _ptr(head_enable), _ptr(staging), staging.numel(), _ptr(workspace),
                                           workspace.numel(), _stream()), "seka_attention_fwd_host")
+
+
+def seka_decode_workspace_bytes(shape: SekaShape) -> int:
+    return int(load().seka_decode_workspace_bytes(ctypes.byref(shape)))
+
+
+def seka_decode_attention(shape: SekaShape, Q, K, V, O, lse, workspace) -> None:
+    """One decode step over the (already edited) cache: Q and O are [B, Hq, d], K and V the packed caches."""
+    _check(load().seka_decode_attention(ctypes.byref(shape), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(lse),
+                                        _ptr(workspace), workspace.numel() if workspace is not None else 0,
+                                        _stream()), "seka_decode_attention")
 
 
 def seka_reset_status(workspace) -> None:
