@@ -109,6 +109,20 @@ seka_status seka_attention_fwd(const seka_shape* shape, const void* Q, const voi
                                void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * AdaSEKA in one call (Algorithm 2): seka_attention_fwd with the routing coefficients of Eq. 6 computed inside
+ * the library's operand-preparation launch instead of by a separate adaseka_route call, so the routed variant
+ * launches exactly what the plain one does.  sigma and k_route are those of adaseka_route; the result equals
+ * adaseka_route followed by seka_attention_fwd bit for bit.  alpha_out, if not NULL, receives the coefficients
+ * (fp32 [B, Hkv, M]).  mask, U and sigma are required.
+ */
+seka_status seka_attention_fwd_routed(const seka_shape* shape, const void* Q, const void* K,
+                                      const void* V, void* O, float* lse,
+                                      const uint8_t* mask, const float* U, const float* sigma,
+                                      int32_t k_route, float* alpha_out,
+                                      const float* gain, const uint8_t* head_enable,
+                                      void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Same computation as seka_attention_fwd for callers whose tensors live in HOST memory
  * (pinned memory makes the copies asynchronous): h_Q, h_K, h_V, h_mask are copied to
  * `staging` (device, seka_host_staging_bytes(shape) bytes, 256-byte aligned), the

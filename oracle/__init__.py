@@ -89,6 +89,8 @@ def route(Q, cu_seqlens: Sequence[int], U, sigma, k_route: int = 0) -> np.ndarra
     alpha = np.zeros((B, Hkv, M), dtype=np.float64)
     for b in range(B):
         last = int(cu_seqlens[b + 1]) - 1
+        if last < int(cu_seqlens[b]):
+            continue                      # a sequence without tokens has no last query: alpha = 0, nothing to steer
         q_last = np.ascontiguousarray(Q[last])
         out = np.zeros((Hkv, M), dtype=np.float64)
         lib.seka_oracle_route(Hq, Hkv, d, r, M, k_route, _dp(q_last), _dp(U), _dp(sigma), _dp(out))

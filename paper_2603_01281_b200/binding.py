@@ -21,7 +21,7 @@ SEKA_F32, SEKA_BF16 = 0, 1
 EXPORTS = ["seka_workspace_bytes", "seka_edit_keys", "adaseka_route", "seka_attention_fwd",
            "seka_host_staging_bytes", "seka_attention_fwd_host", "seka_reset_status", "seka_poll_status",
            "seka_status_string", "seka_launch_count", "seka_edit_keys_static", "seka_decode_workspace_bytes",
-           "seka_decode_attention"]
+           "seka_decode_attention", "seka_attention_fwd_routed"]
 SEKA_STATIC_MAX_TOKENS = 262144
 
 
@@ -60,6 +60,9 @@ def load() -> ctypes.CDLL:
         lib.adaseka_route.restype = ctypes.c_int
         lib.seka_attention_fwd.argtypes = [sp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
         lib.seka_attention_fwd.restype = ctypes.c_int
+        lib.seka_attention_fwd_routed.argtypes = [sp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_int32, vp, vp, vp, vp,
+                                                  ctypes.c_size_t, vp]
+        lib.seka_attention_fwd_routed.restype = ctypes.c_int
         lib.seka_attention_fwd_host.argtypes = [sp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t,
                                                 vp, ctypes.c_size_t, vp]
         lib.seka_attention_fwd_host.restype = ctypes.c_int
@@ -148,6 +151,16 @@ def seka_attention_fwd(shape: SekaShape, Q, K, V, O, lse, mask, U, alpha, gain, 
                                      _ptr(U), _ptr(alpha), _ptr(gain), _ptr(head_enable), _ptr(workspace),
                                      workspace.numel() if workspace is not None else 0, _stream()),
            "seka_attention_fwd")
+
+
+def seka_attention_fwd_routed(shape: SekaShape, Q, K, V, O, lse, mask, U, sigma, k_route: int, alpha_out, gain,
+                              head_enable, workspace) -> None:
+    """AdaSEKA in one call: the routing of Eq. 6 runs inside the operand-preparation launch."""
+    _check(load().seka_attention_fwd_routed(ctypes.byref(shape), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(lse),
+                                            _ptr(mask), _ptr(U), _ptr(sigma), int(k_route), _ptr(alpha_out), _ptr(gain),
+                                            _ptr(head_enable), _ptr(workspace),
+                                            workspace.numel() if workspace is not None else 0, _stream()),
+           "seka_attention_fwd_routed")
 
 
 def seka_attention_fwd_host(shape: SekaShape, h_Q, h_K, h_V, h_O, h_lse, h_mask, U, alpha, gain, head_enable,

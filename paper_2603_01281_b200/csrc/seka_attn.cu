@@ -798,13 +798,13 @@ static seka_status launch_attn(const CUtensorMap& tq, const CUtensorMap& tk, con
                                    : launch_attn_t<D, OutT, false>(tq, tk, tv, tw, p, st);
 }
 
-}  // namespace seka
-
-extern "C" seka_status seka_attention_fwd(const seka_shape* shape, const void* Q, const void* K, const void* V,
-                                          void* O, float* lse, const uint8_t* mask, const float* U,
-                                          const float* alpha, const float* gain, const uint8_t* head_enable,
-                                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
-    using namespace seka;
+// The fused forward behind both entry points: coefficients either given (`alpha`, may be null) or, with `sigma`
+// set, routed inside the preparation launch (Eq. 6) and reported through `alpha_out`.
+static seka_status attention_fwd_impl(const seka_shape* shape, const void* Q, const void* K, const void* V,
+                                      void* O, float* lse, const uint8_t* mask, const float* U,
+                                      const float* alpha, const float* sigma, int k_route, float* alpha_out,
+                                      const float* gain, const uint8_t* head_enable,
+                                      void* workspace, size_t workspace_bytes, void* cuda_stream) {
     seka_status stc = validate_shape(shape);
     if (stc != SEKA_OK) return stc;
     const int T = shape_total_tokens(shape);
@@ -833,7 +833,7 @@ extern "C" seka_status seka_attention_fwd(const seka_shape* shape, const void* Q
     }
     void* W = ws + w.w_off;
     uint8_t* tile_hot = reinterpret_cast<uint8_t*>(ws + w.hot_off);
-    if (steer) launch_prep_steering(shape, U, alpha, gain, head_enable, mask, W, tile_hot, w.n_tiles, st);
+    if (steer) launch_prep_steering(shape, U, alpha, gain, head_enable, mask, W, tile_hot, w.n_tiles, st, Q, sigma, k_route, alpha_out);
 
     CUtensorMap tq, tk, tv, tw;
     if (!make_tile_map(&tq, q16, D, Hq, T) || !make_tile_map(&tk, k16, D, Hkv, T) || !make_tile_map(&tv, v16, D, Hkv, T) ||
@@ -859,6 +859,28 @@ extern "C" seka_status seka_attention_fwd(const seka_shape* shape, const void* Q
     }
     return shape->dtype == SEKA_F32 ? launch_attn<64, float>(tq, tk, tv, tw, p, st)
                                     : launch_attn<64, __nv_bfloat16>(tq, tk, tv, tw, p, st);
+}
+
+}  // namespace seka
+
+extern "C" seka_status seka_attention_fwd(const seka_shape* shape, const void* Q, const void* K, const void* V,
+                                          void* O, float* lse, const uint8_t* mask, const float* U,
+                                          const float* alpha, const float* gain, const uint8_t* head_enable,
+                                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return seka::attention_fwd_impl(shape, Q, K, V, O, lse, mask, U, alpha, nullptr, 0, nullptr, gain, head_enable,
+                                    workspace, workspace_bytes, cuda_stream);
+}
+
+extern "C" seka_status seka_attention_fwd_routed(const seka_shape* shape, const void* Q, const void* K, const void* V,
+                                                 void* O, float* lse, const uint8_t* mask, const float* U,
+                                                 const float* sigma, int32_t k_route, float* alpha_out,
+                                                 const float* gain, const uint8_t* head_enable,
+                                                 void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (shape == nullptr || mask == nullptr || U == nullptr || sigma == nullptr) return SEKA_ERR_INVALID_ARG;
+    if (k_route < 0 || k_route > shape->rank) return SEKA_ERR_INVALID_ARG;
+    if (k_route == 0) k_route = shape->rank;
+    return seka::attention_fwd_impl(shape, Q, K, V, O, lse, mask, U, nullptr, sigma, k_route, alpha_out, gain,
+                                    head_enable, workspace, workspace_bytes, cuda_stream);
 }
 
 extern "C" size_t seka_host_staging_bytes(const seka_shape* shape) {

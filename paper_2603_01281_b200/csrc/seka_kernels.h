@@ -8,9 +8,12 @@
 
 namespace seka {
 
+// With `sigma` set, the routing coefficients of Eq. 6 are computed inside the launch from Q_route (the caller's Q
+// in its own dtype) instead of being read from `alpha`, and written to `alpha_out` if that is not null.
 void launch_prep_steering(const seka_shape* s, const float* U, const float* alpha, const float* gain,
                           const uint8_t* head_enable, const uint8_t* mask, void* W, uint8_t* tile_hot, int n_tiles,
-                          cudaStream_t st);
+                          cudaStream_t st, const void* Q_route = nullptr, const float* sigma = nullptr, int k_route = 0,
+                          float* alpha_out = nullptr);
 void launch_build_items(const seka_shape* s, const WorkspaceLayout& w, bool steer, const float* gain,
                         const uint8_t* head_enable, ItemRecord* items, int* count, cudaStream_t st);
 void launch_compact_mask(const uint8_t* mask, int T, int* list, int* count, cudaStream_t st);

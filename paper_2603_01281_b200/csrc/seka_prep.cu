@@ -1,6 +1,7 @@
 // Small preparation kernels: dense edit operators and per-tile highlight flags for the fused kernel,
 // highlight-mask compaction, fp32 -> bf16 input conversion.
 #include "seka_kernels.h"
+#include "seka_route.cuh"
 
 namespace seka {
 
@@ -10,24 +11,41 @@ namespace seka {
 //                      edit of a key tile is one product  K' = K + K W  (W is symmetric).  Pairs (b, h) that are
 //                      not steered (zero gain, head switched off) are skipped: the fused kernel never reads them.
 //   blocks [n_w, ...): one warp per (sequence, 128-key tile): does the tile hold a highlighted token?
+// With `route.sigma` set the routing coefficients of Eq. 6 are computed here as well (each block of a (b, h) pair
+// repeats the few thousand multiply-adds, from the last token's query), so that AdaSEKA needs no launch of its own
+// before the forward; the coefficients are also written to `route.alpha_out` if that is set.
+struct RouteArgs {
+    const void* Q; int q_is_f32; const float* sigma; int k_route; int Hq; float* alpha_out;
+};
+
 __global__ void prep_steering_kernel(const float* __restrict__ U, const float* __restrict__ alpha,
                                      const float* __restrict__ gain, const uint8_t* __restrict__ head_enable,
                                      const uint8_t* __restrict__ mask, const int* __restrict__ cu_seqlens,
                                      __nv_bfloat16* __restrict__ W, uint8_t* __restrict__ tile_hot,
-                                     int B, int L, int Hkv, int D, int r, int M, int n_tiles, int n_w) {
+                                     int B, int L, int Hkv, int D, int r, int M, int n_tiles, int n_w,
+                                     const RouteArgs route) {
     const int tid = threadIdx.x;
+    extern __shared__ double route_sm[];
     if ((int)blockIdx.x < n_w) {
         const int tiles = D / 32;
         const int bh = blockIdx.x / (tiles * tiles), t = blockIdx.x % (tiles * tiles);
         const int b = bh / Hkv, h = bh % Hkv;
         const float g = gain[b];
+        const double* routed = nullptr;
+        if (route.sigma != nullptr) {
+            routed = route_group(route.Q, route.q_is_f32, U, route.sigma, cu_seqlens, L, route.Hq, Hkv, D, r, M,
+                                 route.k_route, b, h, route_sm);
+            if (t == 0 && route.alpha_out != nullptr)
+                for (int m = tid; m < M; m += blockDim.x) route.alpha_out[(size_t)bh * M + m] = (float)routed[m];
+        }
         if (g == 0.f || (head_enable != nullptr && head_enable[h] == 0)) return;
         const int i0 = (t / tiles) * 32, j0 = (t % tiles) * 32;
         __shared__ float ui[32][33], uj[32][33];
         const int tx = tid & 31, ty = tid >> 5;          // 256 threads: 8 rows of 32
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
         for (int m = 0; m < M; ++m) {
-            const float a = g * (alpha != nullptr ? alpha[((size_t)b * Hkv + h) * M + m] : 1.f);
+            const float a = g * (routed != nullptr ? (float)routed[m]
+                                                   : (alpha != nullptr ? alpha[((size_t)b * Hkv + h) * M + m] : 1.f));
             const float* Um = U + ((size_t)m * Hkv + h) * D * r;
             for (int k0 = 0; k0 < r; k0 += 32) {
                 __syncthreads();
@@ -222,14 +240,17 @@ __global__ void convert_f32_bf16_kernel(const float4* __restrict__ in, uint2* __
 
 void launch_prep_steering(const seka_shape* sh, const float* U, const float* alpha, const float* gain,
                           const uint8_t* head_enable, const uint8_t* mask, void* W, uint8_t* tile_hot, int n_tiles,
-                          cudaStream_t st) {
+                          cudaStream_t st, const void* Q_route, const float* sigma, int k_route, float* alpha_out) {
     const int D = sh->head_dim, tiles = D / 32;
     const int n_w = sh->batch * sh->n_kv_heads * tiles * tiles;
     const int n_flag = (sh->batch * n_tiles + 7) / 8;
-    prep_steering_kernel<<<n_w + n_flag, 256, 0, st>>>(U, alpha, gain, head_enable, mask, sh->cu_seqlens,
-                                                      static_cast<__nv_bfloat16*>(W), tile_hot, sh->batch,
-                                                      sh->max_seqlen, sh->n_kv_heads, D, sh->rank, sh->n_experts,
-                                                      n_tiles, n_w);
+    RouteArgs route{Q_route, sh->dtype == SEKA_F32 ? 1 : 0, sigma, k_route, sh->n_q_heads, alpha_out};
+    const size_t smem = sigma != nullptr ? route_smem_bytes(D, sh->n_experts, k_route) : 0;
+    if (smem > 48 * 1024) cudaFuncSetAttribute(prep_steering_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    prep_steering_kernel<<<n_w + n_flag, 256, smem, st>>>(U, alpha, gain, head_enable, mask, sh->cu_seqlens,
+                                                         static_cast<__nv_bfloat16*>(W), tile_hot, sh->batch,
+                                                         sh->max_seqlen, sh->n_kv_heads, D, sh->rank, sh->n_experts,
+                                                         n_tiles, n_w, route);
     ++g_launches;
 }
 

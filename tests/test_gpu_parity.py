@@ -276,3 +276,46 @@ def test_more_items_than_sms():
     he = np.array([1, 0], dtype=np.uint8)
     rows = H.sampled_rows(w, 40, seed=3)
     _fused_vs_oracle(w, head_enable=he, rows=rows, label="152 items")
+
+
+# ----------------------------------------------------------------- AdaSEKA in one call (routing inside the preparation launch)
+
+@pytest.mark.parametrize("case", ["C3", "small_f32", "small_varlen"])
+def test_routed_forward_equals_route_then_forward(case):
+    if case == "C3":
+        w = inputs.make_workload("C3"); k_route = 0; he = None
+    elif case == "small_f32":
+        w = inputs.make_custom(seed=5, dtype="f32", lens=[200, 140], n_q_heads=8, n_kv_heads=2, head_dim=64, rank=16,
+                               n_experts=3, gain=[0.8, 0.0]); k_route = 5; he = None
+    else:
+        w = inputs.make_custom(seed=6, dtype="bf16", lens=[17, 300, 1, 0, 129], n_q_heads=14, n_kv_heads=2, head_dim=128,
+                               rank=8, n_experts=4, gain=1.0); k_route = 8; he = [1, 0]
+    dev = H.device_tensors(w)
+    shp = H.shape_of(w, dev)
+    hed = None if he is None else torch.tensor(he, dtype=torch.uint8, device="cuda")
+    launches0 = binding.seka_launch_count()
+    # two calls
+    alpha = torch.full((w.batch, w.n_kv_heads, w.n_experts), float("nan"), device="cuda")
+    ws = binding.new_workspace(shp)
+    O2 = torch.full_like(dev["Q"], float("nan")); lse2 = torch.empty((w.total_tokens, w.n_q_heads), device="cuda")
+    binding.adaseka_route(shp, dev["Q"], dev["U"], dev["sigma"], k_route, alpha)
+    binding.seka_attention_fwd(shp, dev["Q"], dev["K"], dev["V"], O2, lse2, dev["mask"], dev["U"], alpha, dev["gain"], hed, ws)
+    launches_two = binding.seka_launch_count() - launches0
+    # one call
+    alpha1 = torch.full_like(alpha, float("nan"))
+    ws1 = binding.new_workspace(shp)
+    O1 = torch.full_like(dev["Q"], float("nan")); lse1 = torch.empty_like(lse2)
+    binding.seka_attention_fwd_routed(shp, dev["Q"], dev["K"], dev["V"], O1, lse1, dev["mask"], dev["U"], dev["sigma"],
+                                      k_route, alpha1, dev["gain"], hed, ws1)
+    launches_one = binding.seka_launch_count() - launches0 - launches_two
+    assert binding.seka_poll_status(ws1) == binding.SEKA_OK
+    assert launches_one == launches_two - 1
+    assert torch.equal(alpha1, alpha)
+    assert torch.equal(O1.view(torch.int16 if O1.dtype == torch.bfloat16 else torch.int32),
+                       O2.view(torch.int16 if O2.dtype == torch.bfloat16 else torch.int32))
+    assert torch.equal(lse1, lse2)
+    a_ref = oracle.route(w.Q, w.cu_seqlens, w.U, w.sigma, k_route)
+    np.testing.assert_allclose(alpha1.cpu().numpy(), a_ref, atol=1e-5)
+    if case != "C3":
+        Oref, Lref, idx = H.oracle_rows(w, None, alpha=a_ref, head_enable=he)
+        H.check_attention(O1.double().cpu().numpy()[idx], Oref, case)

@@ -223,6 +223,15 @@ def test_single_expert_unit_alpha_is_seka():
     assert np.array_equal(a, b)
 
 
+def test_routing_of_an_empty_sequence_is_zero():
+    w = tiny(seed=8, lens=[5, 0, 7], M=3, r=4)
+    a = oracle.route(w.Q, w.cu_seqlens, w.U, w.sigma, 0)
+    assert np.all(a[1] == 0.0) and np.all(np.abs(a[[0, 2]]).max(-1) == 1.0)
+    # the neighbours are what they are without the empty sequence in between
+    w2_cu = np.array([0, 5, 12])
+    np.testing.assert_array_equal(a[[0, 2]], oracle.route(w.Q, w2_cu, w.U, w.sigma, 0))
+
+
 def test_routing_invariants():
     w = inputs.make_custom(seed=71, dtype="f32", lens=[9, 14], n_q_heads=8, n_kv_heads=2, head_dim=16, rank=6,
                            n_experts=4, gain=1.0)
