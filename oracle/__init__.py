@@ -12,7 +12,9 @@ the hook of Algorithm 1/2 with k' = k + g P k (Section 2, Eq. 7), and
 ``attention_rows`` is causal softmax attention with the score of Section 2;
 ``decode_attention`` is the attention of one generated token over the whole
 (already edited) key cache, the situation after the hook of Algorithm 1 has run
-"before generation".
+"before generation"; ``learn_projections`` is the offline spectral learning of
+Section 3.1 (cross-covariances, SVD, the rank rule of Eq. 3) with the
+head-selection statistic of Section 3.4.
 The reading of the routing query under GQA (sum over the group's query heads)
 is PARITY UNPINNED: the paper does not fix it.
 """
@@ -194,3 +196,45 @@ def seka_decode(q, K, V, mask, cu_seqlens, U, alpha=None, gain=None, head_enable
     """The decode path: edit the highlighted cached keys once, then one decode step over the edited cache."""
     Kp = edit_keys(K, mask, cu_seqlens, U, alpha, gain, head_enable)
     return decode_attention(q, Kp, V, cu_seqlens, scale)
+
+
+def learn_projections(h, h_pos, h_neg, gamma: float, answer_tokens=None):
+    """Offline spectral learning of the projections (Section 3.1, Eq. 2-3, first loop of Algorithm 1) and the
+    head-selection statistic of Section 3.4, for every (layer, head) slot at once.
+
+    h, h_pos, h_neg are the neutral / positive / negative key embeddings [n, H, d] (H runs over all (layer, KV head)
+    pairs).  Per slot:  Omega+ = h^T h+ / n,  Omega- = h^T h- / n  (d x d);  SVD of each (numpy / LAPACK, singular
+    values descending);  k+ / k- = the smallest k whose leading singular values hold at least the fraction gamma of
+    their sum;  D = mean over the answer tokens of ||h+_i - h-_i||_2  (answer_tokens: boolean [n], default all).
+    Returns a dict of fp64 arrays: omega_pos, omega_neg [H, d, d]; U_pos, U_neg [H, d, d] (columns = left singular
+    vectors); S_pos, S_neg [H, d]; k_pos, k_neg [H] (int); D [H].
+    """
+    h = _f64(h); h_pos = _f64(h_pos); h_neg = _f64(h_neg)
+    n, H, d = h.shape
+    assert h_pos.shape == h.shape and h_neg.shape == h.shape and n > 0 and 0.0 < gamma <= 1.0
+    sel = np.ones(n, dtype=bool) if answer_tokens is None else np.asarray(answer_tokens) != 0
+    out = {"omega_pos": np.zeros((H, d, d)), "omega_neg": np.zeros((H, d, d)),
+           "U_pos": np.zeros((H, d, d)), "U_neg": np.zeros((H, d, d)),
+           "S_pos": np.zeros((H, d)), "S_neg": np.zeros((H, d)),
+           "k_pos": np.zeros(H, dtype=np.int64), "k_neg": np.zeros(H, dtype=np.int64), "D": np.zeros(H)}
+
+    def smallest_rank(S):
+        total = S.sum()
+        run = 0.0
+        for k in range(1, d + 1):
+            run += S[k - 1]
+            if run >= gamma * total:
+                return k
+        return d
+
+    for s in range(H):
+        for tag, other in (("pos", h_pos), ("neg", h_neg)):
+            omega = h[:, s, :].T @ other[:, s, :] / n
+            U, S, _ = np.linalg.svd(omega)
+            out["omega_" + tag][s] = omega
+            out["U_" + tag][s] = U
+            out["S_" + tag][s] = S
+            out["k_" + tag][s] = smallest_rank(S)
+        diff = h_pos[sel, s, :] - h_neg[sel, s, :]
+        out["D"][s] = np.sqrt((diff * diff).sum(axis=1)).mean() if sel.any() else 0.0
+    return out

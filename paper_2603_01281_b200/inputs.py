@@ -274,3 +274,32 @@ def sample_rows(rng: np.random.Generator, L: int, mask: np.ndarray, n: int, tile
         pool = np.setdiff1d(np.arange(L), np.asarray(must))
         must = sorted(set(must) | set(rng.choice(pool, size=extra, replace=False).tolist()))
     return np.asarray(must, dtype=np.int32)
+
+
+def contrastive_embeddings(*, seed: int, n: int, slots: int, head_dim: int, rank: int = 8, dtype: str = "bf16"):
+    """Synthetic stand-in for the key embeddings of the paper's contrastive prompts (Section 3.1): for each of
+    `slots` (layer, KV head) pairs, n neutral keys with a decaying per-dimension spread (0.98**j), and positive /
+    negative keys in which a planted `rank`-dimensional relevance subspace is amplified by a_s / attenuated by
+    a_s / 2 (a_s uniform in [0.3, 1.5]; every fourth slot has a_s = 0, i.e. a head that does not react), plus
+    N(0, 0.1) noise.  Also a Bernoulli(0.3) set of "answer tokens".  Returns float32 arrays h, h_pos, h_neg
+    [n, slots, d] (rounded to the storage type), answer_tokens uint8 [n], the planted bases [slots, d, rank] and
+    the strengths a_s.  Draws only; none of the learning arithmetic lives here."""
+    rng = np.random.default_rng(BASE_SEED + 1000 + seed)
+    d = head_dim
+    decay = (0.98 ** np.arange(d)).astype(np.float64)
+    h = np.empty((n, slots, d), dtype=np.float32); hp = np.empty_like(h); hn = np.empty_like(h)
+    bases = np.empty((slots, d, rank), dtype=np.float64)
+    strength = rng.uniform(0.3, 1.5, size=slots)
+    strength[3::4] = 0.0
+    for s in range(slots):
+        q, _ = np.linalg.qr(rng.standard_normal((d, rank)))
+        bases[s] = q
+        z = rng.standard_normal((n, d)) * decay
+        lift = (z @ q) @ q.T
+        h[:, s] = z
+        hp[:, s] = z + strength[s] * lift + 0.1 * rng.standard_normal((n, d))
+        hn[:, s] = z - 0.5 * strength[s] * lift + 0.1 * rng.standard_normal((n, d))
+    if dtype == "bf16":
+        h, hp, hn = round_to_bf16(h), round_to_bf16(hp), round_to_bf16(hn)
+    answer = (rng.random(n) < 0.3).astype(np.uint8)
+    return h, hp, hn, answer, bases, strength

@@ -405,3 +405,77 @@ def test_decode_over_edited_cache_uses_edited_keys():
     O_ref, L_ref = oracle.decode_attention(q, Kp, w.V, w.cu_seqlens)
     np.testing.assert_allclose(O, O_ref, rtol=1e-10, atol=1e-12)
     np.testing.assert_allclose(LSE, L_ref, rtol=1e-10, atol=1e-12)
+
+
+# ----------------------------------------------------------------- offline spectral learning (Section 3.1, Eq. 2-3, Section 3.4)
+
+def test_learner_hand_case():
+    # Omega+ = h^T h+ / 2 = diag(1.5, 1); Omega- = diag(0.5, 2): singular values sorted descending
+    h = np.array([[1.0, 0.0], [0.0, 2.0]]).reshape(2, 1, 2)
+    hp = np.array([[3.0, 0.0], [0.0, 1.0]]).reshape(2, 1, 2)
+    hn = np.array([[1.0, 0.0], [0.0, 2.0]]).reshape(2, 1, 2)
+    r = oracle.learn_projections(h, hp, hn, gamma=0.6)
+    np.testing.assert_allclose(r["omega_pos"][0], np.diag([1.5, 1.0]), atol=1e-15)
+    np.testing.assert_allclose(r["S_pos"][0], [1.5, 1.0], atol=1e-15)
+    np.testing.assert_allclose(np.abs(r["U_pos"][0]), np.eye(2), atol=1e-15)
+    np.testing.assert_allclose(r["S_neg"][0], [2.0, 0.5], atol=1e-15)
+    np.testing.assert_allclose(np.abs(r["U_neg"][0]), [[0, 1], [1, 0]], atol=1e-15)      # the second axis leads
+    assert r["k_pos"][0] == 1 and r["k_neg"][0] == 1                  # 1.5 / 2.5 = 0.6 and 2 / 2.5 = 0.8 reach gamma
+    assert oracle.learn_projections(h, hp, hn, gamma=0.61)["k_pos"][0] == 2
+    # D: ||h+ - h-|| per token = 2 and 1; mean 1.5; only the second token an answer token -> 1
+    np.testing.assert_allclose(r["D"][0], 1.5, atol=1e-15)
+    np.testing.assert_allclose(oracle.learn_projections(h, hp, hn, 0.6, answer_tokens=[0, 1])["D"][0], 1.0, atol=1e-15)
+
+
+def test_learner_recovers_a_planted_subspace_exactly():
+    # neutral keys with h^T h / n = I exactly, positive keys h (I + a B B^T), negative keys h (I - b B B^T):
+    # Omega+ = I + a B B^T and Omega- = I - b B B^T, whose spectra and subspaces are known in closed form
+    rng = np.random.default_rng(3)
+    n, d, r, a, b = 200, 12, 3, 2.0, 0.75
+    qf, _ = np.linalg.qr(rng.standard_normal((n, d)))
+    h = math.sqrt(n) * qf
+    B, _ = np.linalg.qr(rng.standard_normal((d, r)))
+    PB = B @ B.T
+    hp = h @ (np.eye(d) + a * PB); hn = h @ (np.eye(d) - b * PB)
+    gamma = 0.55          # 0.5 would put the threshold exactly on the sum of the three leading values
+    out = oracle.learn_projections(h[:, None, :], hp[:, None, :], hn[:, None, :], gamma)
+    np.testing.assert_allclose(out["omega_pos"][0], np.eye(d) + a * PB, atol=1e-12)
+    np.testing.assert_allclose(out["S_pos"][0], [1 + a] * r + [1.0] * (d - r), atol=1e-12)
+    np.testing.assert_allclose(out["S_neg"][0], [1.0] * (d - r) + [1 - b] * r, atol=1e-12)
+    U = out["U_pos"][0]
+    np.testing.assert_allclose(U.T @ U, np.eye(d), atol=1e-12)
+    np.testing.assert_allclose(U[:, :r] @ U[:, :r].T, PB, atol=1e-10)                     # P+ of Eq. 2 with k+ = r
+    Un = out["U_neg"][0]
+    np.testing.assert_allclose(Un[:, d - r:] @ Un[:, d - r:].T, PB, atol=1e-10)           # P- of Eq. 2 with k- = d - r
+    # Eq. 3 in closed form: the total is d + a r; k leading values of 1 + a, then ones
+    total = d + a * r
+    k_expect = next(k for k in range(1, d + 1) if (min(k, r) * (1 + a) + max(0, k - r)) >= gamma * total - 1e-12)
+    assert out["k_pos"][0] == k_expect
+    assert out["k_pos"][0] == brute.rank_by_variance(out["S_pos"][0], gamma)
+    assert out["k_neg"][0] == brute.rank_by_variance(out["S_neg"][0], gamma)
+    # D: h+ - h- = (a + b) h B B^T, so each token's distance is (a + b) ||B^T h_i||
+    np.testing.assert_allclose(out["D"][0], ((a + b) * np.linalg.norm(h @ B, axis=1)).mean(), rtol=1e-12)
+
+
+def test_learner_invariants_on_the_synthetic_embeddings():
+    h, hp, hn, ans, bases, strength = inputs.contrastive_embeddings(seed=1, n=600, slots=5, head_dim=16, rank=3, dtype="f32")
+    out = oracle.learn_projections(h, hp, hn, 0.7, answer_tokens=ans)
+    for s in range(5):
+        for tag in ("pos", "neg"):
+            Om, U, S = out["omega_" + tag][s], out["U_" + tag][s], out["S_" + tag][s]
+            assert np.all(np.diff(S) <= 1e-15) and np.all(S >= 0)
+            np.testing.assert_allclose(U.T @ U, np.eye(16), atol=1e-12)
+            np.testing.assert_allclose(Om @ Om.T @ U, U * (S * S), atol=1e-12)            # left singular vectors
+            assert out["k_" + tag][s] == brute.rank_by_variance(S, 0.7)
+    # repeating every token leaves the cross-covariances and D unchanged (the 1/n of Section 3.1)
+    rep = oracle.learn_projections(np.tile(h, (2, 1, 1)), np.tile(hp, (2, 1, 1)), np.tile(hn, (2, 1, 1)), 0.7,
+                                   answer_tokens=np.tile(ans, 2))
+    np.testing.assert_allclose(rep["omega_pos"], out["omega_pos"], rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(rep["D"], out["D"], rtol=1e-12)
+    # slots are independent, and a head that does not react (strength 0) has the smallest distance
+    one = oracle.learn_projections(h[:, 2:3], hp[:, 2:3], hn[:, 2:3], 0.7, answer_tokens=ans)
+    np.testing.assert_array_equal(one["omega_neg"][0], out["omega_neg"][2])
+    assert np.argmin(out["D"]) == 3 and strength[3] == 0.0
+    # the planted directions lead the positive spectrum of a reacting head
+    lead = out["U_pos"][0][:, :3]
+    assert np.linalg.norm(bases[0].T @ lead) ** 2 > 2.9
