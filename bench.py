@@ -191,6 +191,37 @@ def decode_bench(w, peaks, batch: int = 64, steps: int = 30):
                 batch, L, Hkv, d, 2 * K.numel() * 2 / 1e9)}
 
 
+def learn_bench(peaks, n: int = 32768, slots: int = 288, d: int = 128, steps: int = 5):
+    """Offline spectral learning for a whole 8B-shaped model in one call: 36 layers x 8 KV heads = 288 slots,
+    n key embeddings each for the neutral / positive / negative prompts (bf16, 3 x 2.4 GB), gamma = 0.7.
+    Algorithmic bytes: the three tensors read once for the cross-covariances plus h+ and h- of the answer tokens
+    (30 %) once more for the head-selection distance."""
+    import torch
+    from paper_2603_01281_b200 import binding
+    gen = torch.Generator(device="cuda"); gen.manual_seed(260301283)
+    h = torch.randn((n, slots, d), device="cuda", dtype=torch.float32, generator=gen).to(torch.bfloat16)
+    hp = (h.float() * 1.5 + 0.1 * torch.randn((n, slots, d), device="cuda", generator=gen)).to(torch.bfloat16)
+    hn = (h.float() * 0.5 + 0.1 * torch.randn((n, slots, d), device="cuda", generator=gen)).to(torch.bfloat16)
+    ans = (torch.rand(n, device="cuda", generator=gen) < 0.3).to(torch.uint8)
+    for _ in range(2):
+        binding.seka_learn_projections(h, hp, hn, ans, 0.7)
+    torch.cuda.synchronize()
+    n0 = binding.seka_launch_count()
+    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        res = binding.seka_learn_projections(h, hp, hn, ans, 0.7)
+    e1.record(); torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    n_ans = int(ans.sum().item())
+    cov_bytes = 3.0 * n * slots * d * 2
+    alg_bytes = cov_bytes + 2.0 * n_ans * slots * d * 2
+    return {"ms": ms, "GB/s_whole_call": alg_bytes / (ms * 1e-3) / 1e9, "algorithmic_MB": alg_bytes / 1e6,
+            "covariance_flops": 2.0 * 2 * n * slots * d * d, "launches_per_call": (binding.seka_launch_count() - n0) / steps,
+            "embeddings": "bf16 3 x [%d, %d, %d] = %.2f GB" % (n, slots, d, cov_bytes / 1e9),
+            "k_pos_mean": float(res["k_pos"].float().mean().item())}
+
+
 def run_reference(args, rank: int):
     """The reference arm: the CPU oracle on a bounded sample of the same workload, K timed steps."""
     if rank != 0:
@@ -226,6 +257,7 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle work for cpu_baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-edit-bench", action="store_true", help="skip the stand-alone key-edit measurement")
+    ap.add_argument("--no-learn-bench", action="store_true", help="skip the offline spectral-learning measurement")
     ap.add_argument("--no-decode-bench", action="store_true", help="skip the decode-over-edited-cache measurement")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -329,6 +361,9 @@ def main():
     edit_res = None
     if rank == 0 and world == 1 and not args.no_edit_bench:
         edit_res = edit_keys_bench(w, measured_peaks())
+    learn_res = None
+    if rank == 0 and world == 1 and not args.no_learn_bench:
+        learn_res = learn_bench(measured_peaks())
     decode_res = None
     if rank == 0 and world == 1 and not args.no_decode_bench:
         decode_res = decode_bench(w, measured_peaks())
@@ -361,6 +396,8 @@ def main():
             line["extra"]["edit_keys"] = edit_res
         if decode_res is not None:
             line["extra"]["decode"] = decode_res
+        if learn_res is not None:
+            line["extra"]["learn"] = learn_res
         if world == 1 and not args.no_cpu_baseline:
             import oracle
             f, s, r = cpu_oracle_sample(w, args.cpu_budget)

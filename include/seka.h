@@ -187,6 +187,37 @@ seka_status seka_decode_attention(const seka_shape* shape, const void* Q, const 
                                   void* O, float* lse, void* workspace, size_t workspace_bytes,
                                   void* cuda_stream);
 
+/*
+ * Offline spectral learning of the projections (Section 3.1, Eq. 2-3; first loop of Algorithm 1) and the
+ * head-selection distance of Section 3.4, for every (layer, KV head) slot of a model in one call.
+ *   h, h_pos, h_neg   bf16 [n_tokens, n_slots, head_dim]: neutral / positive / negative key embeddings, token-major
+ *   answer_tokens     uint8 [n_tokens] (non-zero = the token counts for D) or NULL (all tokens)
+ * Per slot s (all outputs device fp32 unless noted, written by this call):
+ *   omega_pos[s], omega_neg[s]  [d, d] row-major: Omega+ = h^T h+ / n, Omega- = h^T h- / n  (bf16 products, fp32 sums)
+ *   U_pos[s], U_neg[s]          [d, d] row-major, COLUMNS = left singular vectors of Omega+ / Omega-, singular values
+ *                               descending (the layout seka_edit_keys / seka_attention_fwd take as U with rank = d;
+ *                               P+ of Eq. 2 uses columns [0, k_pos), P- columns [k_neg, d)); computed in fp64 from the
+ *                               fp32 Omega by one-sided Jacobi; a singular vector is defined up to its sign; columns
+ *                               of exactly zero singular value are returned as zeros
+ *   S_pos[s], S_neg[s]          [d] singular values
+ *   k_pos[s], k_neg[s]          int32: the smallest k with sum_{i<=k} S_i >= gamma * sum_i S_i (Eq. 3), decided in fp64
+ *   D[s]                        mean over the answer tokens of ||h+_t - h-_t||_2 (Section 3.4); 0 without answer tokens
+ * head_dim is 64 or 128 (64 needs an even number of slots: neighbouring heads share a tensor-core product).
+ * `workspace`: seka_learn_workspace_bytes(shape) bytes, 256-byte aligned, first 256 bytes the status block.
+ */
+typedef struct {
+    int32_t n_tokens;           /* n >= 1 */
+    int32_t n_slots;            /* number of (layer, KV head) pairs */
+    int32_t head_dim;           /* d: 64 or 128 */
+    float   gamma;              /* variance threshold of Eq. 3, in (0, 1] */
+} seka_learn_shape;
+size_t seka_learn_workspace_bytes(const seka_learn_shape* shape);
+seka_status seka_learn_projections(const seka_learn_shape* shape, const void* h, const void* h_pos,
+                                   const void* h_neg, const uint8_t* answer_tokens,
+                                   float* omega_pos, float* omega_neg, float* U_pos, float* U_neg,
+                                   float* S_pos, float* S_neg, int32_t* k_pos, int32_t* k_neg, float* D,
+                                   void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Clears the device status word (async on the stream); call once before first use of a workspace. */
 seka_status seka_reset_status(void* workspace, void* cuda_stream);
 /* Synchronises the stream and returns the device status word (SEKA_OK if no wait ran out). */

@@ -21,7 +21,7 @@ SEKA_F32, SEKA_BF16 = 0, 1
 EXPORTS = ["seka_workspace_bytes", "seka_edit_keys", "adaseka_route", "seka_attention_fwd",
            "seka_host_staging_bytes", "seka_attention_fwd_host", "seka_reset_status", "seka_poll_status",
            "seka_status_string", "seka_launch_count", "seka_edit_keys_static", "seka_decode_workspace_bytes",
-           "seka_decode_attention", "seka_attention_fwd_routed"]
+           "seka_decode_attention", "seka_attention_fwd_routed", "seka_learn_workspace_bytes", "seka_learn_projections"]
 SEKA_STATIC_MAX_TOKENS = 262144
 
 
@@ -30,6 +30,11 @@ class SekaShape(ctypes.Structure):
                 ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
                 ("rank", ctypes.c_int32), ("n_experts", ctypes.c_int32), ("dtype", ctypes.c_int32),
                 ("softmax_scale", ctypes.c_float), ("cu_seqlens", ctypes.c_void_p)]
+
+
+class SekaLearnShape(ctypes.Structure):
+    _fields_ = [("n_tokens", ctypes.c_int32), ("n_slots", ctypes.c_int32), ("head_dim", ctypes.c_int32),
+                ("gamma", ctypes.c_float)]
 
 
 class SekaError(RuntimeError):
@@ -69,6 +74,10 @@ def load() -> ctypes.CDLL:
         lib.seka_decode_workspace_bytes.argtypes = [sp]; lib.seka_decode_workspace_bytes.restype = ctypes.c_size_t
         lib.seka_decode_attention.argtypes = [sp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
         lib.seka_decode_attention.restype = ctypes.c_int
+        lp = ctypes.POINTER(SekaLearnShape)
+        lib.seka_learn_workspace_bytes.argtypes = [lp]; lib.seka_learn_workspace_bytes.restype = ctypes.c_size_t
+        lib.seka_learn_projections.argtypes = [lp] + [vp] * 14 + [ctypes.c_size_t, vp]
+        lib.seka_learn_projections.restype = ctypes.c_int
         lib.seka_reset_status.argtypes = [vp, vp]; lib.seka_reset_status.restype = ctypes.c_int
         lib.seka_poll_status.argtypes = [vp, vp]; lib.seka_poll_status.restype = ctypes.c_int
         lib.seka_status_string.argtypes = [ctypes.c_int]; lib.seka_status_string.restype = ctypes.c_char_p
@@ -183,6 +192,34 @@ def seka_decode_attention(shape: SekaShape, Q, K, V, O, lse, workspace) -> None:
     _check(load().seka_decode_attention(ctypes.byref(shape), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(lse),
                                         _ptr(workspace), workspace.numel() if workspace is not None else 0,
                                         _stream()), "seka_decode_attention")
+
+
+def seka_learn_projections(h, h_pos, h_neg, answer_tokens, gamma: float) -> dict:
+    """Offline spectral learning for every slot of bf16 embeddings [n, slots, d]; allocates the outputs with torch
+    and returns them in a dict (omega_pos, omega_neg, U_pos, U_neg, S_pos, S_neg, k_pos, k_neg, D)."""
+    n, slots, d = h.shape
+    assert h.dtype == torch.bfloat16 and h_pos.shape == h.shape and h_neg.shape == h.shape
+    shp = SekaLearnShape(n, slots, d, gamma)
+    nbytes = int(load().seka_learn_workspace_bytes(ctypes.byref(shp)))
+    if nbytes == 0:
+        raise SekaError(SEKA_ERR_UNSUPPORTED, "seka_learn_workspace_bytes")
+    ws = torch.zeros(nbytes, dtype=torch.uint8, device=h.device)
+    f32 = dict(dtype=torch.float32, device=h.device)
+    out = {"omega_pos": torch.empty((slots, d, d), **f32), "omega_neg": torch.empty((slots, d, d), **f32),
+           "U_pos": torch.empty((slots, d, d), **f32), "U_neg": torch.empty((slots, d, d), **f32),
+           "S_pos": torch.empty((slots, d), **f32), "S_neg": torch.empty((slots, d), **f32),
+           "k_pos": torch.empty(slots, dtype=torch.int32, device=h.device),
+           "k_neg": torch.empty(slots, dtype=torch.int32, device=h.device), "D": torch.empty(slots, **f32)}
+    _check(load().seka_learn_projections(ctypes.byref(shp), _ptr(h), _ptr(h_pos), _ptr(h_neg), _ptr(answer_tokens),
+                                         _ptr(out["omega_pos"]), _ptr(out["omega_neg"]), _ptr(out["U_pos"]),
+                                         _ptr(out["U_neg"]), _ptr(out["S_pos"]), _ptr(out["S_neg"]), _ptr(out["k_pos"]),
+                                         _ptr(out["k_neg"]), _ptr(out["D"]), _ptr(ws), ws.numel(), _stream()),
+           "seka_learn_projections")
+    st = seka_poll_status(ws)
+    if st != SEKA_OK:
+        raise SekaError(st, "seka_learn_projections (device status)")
+    out["workspace"] = ws
+    return out
 
 
 def seka_reset_status(workspace) -> None:

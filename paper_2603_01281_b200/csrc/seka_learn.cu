@@ -1,0 +1,486 @@
+// Offline spectral learning of the projections (Section 3.1, Eq. 2-3, first loop of Algorithm 1) and the
+// head-selection distance of Section 3.4, for all (layer, KV head) slots of a model in one call.
+//
+//   learn_cov_kernel      Omega+ = h^T h+ / n and Omega- = h^T h- / n.  The contraction runs over tokens, so the
+//                         key embeddings are read exactly once (three bf16 tensors [n, slots, d]); at 2 d / 3 FLOP
+//                         per byte the pass is bound by HBM bandwidth but needs the tensor cores to keep up.
+//                         Persistent CTAs, an item = (group of 128 columns, chunk of tokens): a producer warp
+//                         streams 128-token tiles of h, h+, h- with TMA through two stages; one thread issues
+//                         tcgen05 products with BOTH operands MN-major (the token axis is the contraction) into two
+//                         128 x 128 accumulators in tensor memory; four warps drain the finished accumulators of
+//                         item i while item i + 1 accumulates in the other half of tensor memory.
+//   learn_reduce_kernel   sums the per-chunk partials in chunk order, scales by 1 / n.
+//   learn_dist_kernel     D = mean over the answer tokens of ||h+ - h-||_2, per slot (fixed summation order).
+//   learn_svd_kernel      one CTA per matrix: one-sided Jacobi (Hestenes) in fp64 on the columns of Omega held in
+//                         shared memory, round-robin pair ordering, one warp per column pair; on convergence the
+//                         column norms are the singular values and the normalised columns the left singular
+//                         vectors; sorted descending; the rank of Eq. 3 from the sorted values.
+#include <math.h>
+
+#include "seka_kernels.h"
+
+namespace seka {
+namespace {
+
+// ------------------------------------------------------------------------------------ cross-covariances
+constexpr int LC_THREADS = 192;                 // warp 0 producer, warp 1 MMA issuer, warps 2..5 drain
+constexpr int LC_TOK = 128;                     // tokens per stage
+constexpr int LC_NS = 2;
+constexpr uint32_t LC_BLK = 128 * 128;          // [128 tokens x 64 columns] block, 128-byte swizzle
+constexpr uint32_t LC_TILE = 2 * LC_BLK;        // 128 columns of one tensor
+constexpr uint32_t LC_STAGE = 3 * LC_TILE;      // h, h+, h-
+constexpr uint32_t LC_BARS = LC_NS * LC_STAGE;  // full[2], empty[2], acc_full[2], acc_free[2]
+constexpr uint32_t LC_MISC = LC_BARS + 8 * 8;
+constexpr uint32_t LC_DYN_BYTES = LC_MISC + 16 + 1024;
+constexpr uint32_t LC_TMEM_COLS = 512;          // two sets of (Omega+, Omega-) accumulators
+
+struct LearnCovParams {
+    float* part;            // [n_chunks][slots][2][d][d]
+    int n_tokens, n_groups, d, slots, chunk_tokens, n_chunks;
+    int* status;
+};
+
+__device__ __forceinline__ bool lc_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status, int where) {
+    const bool ok = mbar_wait(bar, parity, abort_flag, status, where);
+    return __all_sync(0xffffffffu, ok);
+}
+
+// bf16 x bf16 -> fp32, M = N = 128, A and B both MN-major (their contraction axis, the tokens, is the slow one)
+constexpr uint32_t LC_IDESC = umma_idesc_bf16(128, true) | (1u << 15);
+
+__global__ void __launch_bounds__(LC_THREADS, 1)
+learn_cov_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmP,
+                 const __grid_constant__ CUtensorMap tmN, const LearnCovParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + LC_BARS);
+    uint64_t* full = bars;              // [2] the three tiles of a stage have landed
+    uint64_t* empty = bars + 2;         // [2] the products that read the stage have finished
+    uint64_t* acc_full = bars + 4;      // [2] every product of an item has finished: its accumulators can be read
+    uint64_t* acc_free = bars + 6;      // [2] four drain-warp arrivals: the accumulators have been read
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + LC_MISC);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + LC_MISC + 4);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (__syncthreads_or(*reinterpret_cast<volatile int*>(p.status) != 0)) return;
+
+    if (tid == 0) {
+        for (int i = 0; i < 2; ++i) { mbar_init(full + i, 1); mbar_init(empty + i, 1); mbar_init(acc_full + i, 1); mbar_init(acc_free + i, 4); }
+        *abort_flag = 0;
+        mbar_fence_init();
+        tma_prefetch_desc(&tmH); tma_prefetch_desc(&tmP); tma_prefetch_desc(&tmN);
+    }
+    __syncwarp();
+    if (warp == 0) { tmem_alloc(tmem_holder, LC_TMEM_COLS); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_holder;
+    const int n_items = p.n_groups * p.n_chunks;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ producer
+        uint32_t n_push = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+            const int g = item % p.n_groups, c = item / p.n_groups;
+            const int t0 = c * p.chunk_tokens, t1 = min(p.n_tokens, t0 + p.chunk_tokens);
+            const int n_tiles = (t1 - t0 + LC_TOK - 1) / LC_TOK;
+            for (int t = 0; t < n_tiles; ++t) {
+                const uint32_t s = n_push % LC_NS;
+                if (n_push >= LC_NS) {
+                    ok = lc_wait(empty + s, ((n_push / LC_NS) - 1) & 1, abort_flag, p.status, 70);
+                    if (!ok) break;
+                }
+                if (lane == 0) {
+                    uint8_t* st = smem + s * LC_STAGE;
+                    mbar_expect_tx(full + s, LC_STAGE);
+                    const int row = t0 + t * LC_TOK;            // rows beyond the last token are filled with zeros
+#pragma unroll
+                    for (int blk = 0; blk < 2; ++blk) {
+                        tma_load_3d(st + blk * LC_BLK, &tmH, full + s, blk * 64, g, row);
+                        tma_load_3d(st + LC_TILE + blk * LC_BLK, &tmP, full + s, blk * 64, g, row);
+                        tma_load_3d(st + 2 * LC_TILE + blk * LC_BLK, &tmN, full + s, blk * 64, g, row);
+                    }
+                }
+                __syncwarp();
+                ++n_push;
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        constexpr uint32_t DESC_HI = umma_desc_hi_sw128(1024);
+        const uint32_t d0 = umma_desc_lo(smem_u32(smem), LC_BLK);
+        uint32_t n_pop = 0, it = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
+            const int c = item / p.n_groups;
+            const int t0 = c * p.chunk_tokens, t1 = min(p.n_tokens, t0 + p.chunk_tokens);
+            const int n_tiles = (t1 - t0 + LC_TOK - 1) / LC_TOK;
+            const uint32_t set = it & 1;
+            if (it >= 2) {
+                ok = lc_wait(acc_free + set, ((it >> 1) - 1) & 1, abort_flag, p.status, 71);
+                if (!ok) break;
+            }
+            for (int t = 0; t < n_tiles; ++t) {
+                const uint32_t s = n_pop % LC_NS;
+                ok = lc_wait(full + s, (n_pop / LC_NS) & 1, abort_flag, p.status, 72);
+                if (!ok) break;
+                tc_fence_after();
+                if (lane == 0) {
+                    const uint32_t dh = d0 + s * (LC_STAGE >> 4), dp = dh + (LC_TILE >> 4), dn = dp + (LC_TILE >> 4);
+                    const uint32_t acc = tmem_base + set * 256;
+#pragma unroll
+                    for (int ks = 0; ks < LC_TOK / 16; ++ks) {        // 16 tokens per product: 16 rows x 128 B further on
+                        const uint32_t off = (uint32_t)ks * (2048 >> 4);
+                        const uint32_t accumulate = (t > 0 || ks > 0) ? 1u : 0u;
+                        umma_ss(acc, dh + off, DESC_HI, dp + off, DESC_HI, LC_IDESC, accumulate);
+                        umma_ss(acc + 128, dh + off, DESC_HI, dn + off, DESC_HI, LC_IDESC, accumulate);
+                    }
+                    umma_commit(empty + s);
+                    if (t == n_tiles - 1) umma_commit(acc_full + set);
+                }
+                __syncwarp();
+                ++n_pop;
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ drain: accumulators -> per-chunk partials
+        const int q = warp & 3;                                        // the quarter of tensor-memory lanes this warp may read
+        const int row = q * 32 + lane;
+        uint32_t it = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
+            const int g = item % p.n_groups, c = item / p.n_groups;
+            const uint32_t set = it & 1;
+            ok = lc_wait(acc_full + set, (it >> 1) & 1, abort_flag, p.status, 73);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16) + set * 256;
+#pragma unroll 1
+            for (int sign = 0; sign < 2; ++sign) {
+#pragma unroll 1
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    float* dst;
+                    if (p.d == 128) {
+                        dst = p.part + ((((size_t)c * p.slots + g) * 2 + sign) * 128 + row) * 128 + c4 * 32;
+                    } else {
+                        // two heads of 64 columns share the product: only the diagonal blocks are cross-covariances
+                        const int hd = q >> 1;
+                        if ((c4 >> 1) != hd) continue;                 // the same for the whole warp
+                        dst = p.part + ((((size_t)c * p.slots + 2 * g + hd) * 2 + sign) * 64 + (row & 63)) * 64 + (c4 & 1) * 32;
+                    }
+                    uint32_t v[32];
+                    tmem_ld32(t_lane + sign * 128 + c4 * 32, v);
+                    tmem_wait_ld_on(v);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e)
+                        reinterpret_cast<float4*>(dst)[e] = make_float4(__uint_as_float(v[4 * e]), __uint_as_float(v[4 * e + 1]),
+                                                                        __uint_as_float(v[4 * e + 2]), __uint_as_float(v[4 * e + 3]));
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_free + set);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        __syncwarp();
+        tmem_dealloc(tmem_base, LC_TMEM_COLS);
+    }
+}
+
+// omega[sign][slot][i][j] = sum over chunks (in order) of the partials, divided by the number of tokens
+__global__ void learn_reduce_kernel(const float* __restrict__ part, float* __restrict__ omega_pos,
+                                    float* __restrict__ omega_neg, int slots, int d, int n_chunks, float inv_n) {
+    const size_t per = (size_t)d * d, total = (size_t)slots * 2 * per;
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= total) return;
+    float acc = 0.f;
+    for (int c = 0; c < n_chunks; ++c) acc += part[(size_t)c * total + idx];
+    const size_t slot = idx / (2 * per), rest = idx % (2 * per);
+    float* out = rest < per ? omega_pos : omega_neg;
+    out[slot * per + rest % per] = acc * inv_n;
+}
+
+// ------------------------------------------------------------------------------------ head-selection distance
+// Block b takes a range of tokens; warp w owns the slots w, w + 8, ... (so that the eight warps read neighbouring
+// rows) and keeps their running sums in shared memory: one writer per slot, fixed order.
+constexpr int LD_THREADS = 256;
+__global__ void learn_dist_kernel(const __nv_bfloat16* __restrict__ hp, const __nv_bfloat16* __restrict__ hn,
+                                  const uint8_t* __restrict__ answer, int n, int slots, int d, int tokens_per_block,
+                                  float* __restrict__ part_sum, int* __restrict__ part_count) {
+    extern __shared__ float acc[];                  // [slots]
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int s = threadIdx.x; s < slots; s += LD_THREADS) acc[s] = 0.f;
+    __syncthreads();
+    const int t0 = blockIdx.x * tokens_per_block, t1 = min(n, t0 + tokens_per_block);
+    int count = 0;
+    for (int t = t0; t < t1; ++t) {
+        if (answer != nullptr && answer[t] == 0) continue;
+        ++count;
+        for (int s = warp; s < slots; s += LD_THREADS / 32) {
+            const size_t base = ((size_t)t * slots + s) * d;
+            float ss = 0.f;
+            for (int i = 2 * lane; i < d; i += 64) {
+                const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(hp + base + i));
+                const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(hn + base + i));
+                const float dx = a.x - b.x, dy = a.y - b.y;
+                ss = fmaf(dx, dx, fmaf(dy, dy, ss));
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+            if (lane == 0) acc[s] += sqrtf(ss);
+        }
+    }
+    __syncthreads();
+    for (int s = threadIdx.x; s < slots; s += LD_THREADS) part_sum[(size_t)blockIdx.x * slots + s] = acc[s];
+    if (threadIdx.x == 0) part_count[blockIdx.x] = count;
+}
+
+__global__ void learn_dist_reduce_kernel(const float* __restrict__ part_sum, const int* __restrict__ part_count,
+                                         int n_blocks, int slots, float* __restrict__ D) {
+    const int s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= slots) return;
+    double tot = 0.0;
+    long long cnt = 0;
+    for (int b = 0; b < n_blocks; ++b) { tot += (double)part_sum[(size_t)b * slots + s]; cnt += part_count[b]; }
+    D[s] = cnt > 0 ? (float)(tot / (double)cnt) : 0.f;
+}
+
+// ------------------------------------------------------------------------------------ SVD (one-sided Jacobi, fp64)
+constexpr int SV_THREADS = 512;
+constexpr int SV_MAX_SWEEPS = 60;
+
+// Column pair of position `i` in round `rd` of the round-robin tournament over d columns (d even): the last column
+// stays in place and the others rotate, so that the d / 2 pairs of a round are disjoint and d - 1 rounds meet every pair.
+__device__ __forceinline__ void sv_pair(int d, int rd, int i, int& a, int& b) {
+    const int m = d - 1;
+    if (i == 0) { a = m; b = rd % m; }
+    else { a = (rd + i) % m; b = (rd - i + m) % m; }
+    if (a > b) { const int t = a; a = b; b = t; }
+}
+
+// One CTA per (sign, slot).  G (column-major, fp64, shared memory) starts as Omega; plane rotations from the right
+// make its columns mutually orthogonal: Omega V = U S.  Outputs: U [d x d] row-major with the singular vectors as
+// columns, S descending, and the smallest k with sum_{i<=k} S_i >= gamma * sum_i S_i (Eq. 3).
+__global__ void __launch_bounds__(SV_THREADS, 1)
+learn_svd_kernel(const float* __restrict__ omega_pos, const float* __restrict__ omega_neg, int slots, int d, float gamma,
+                 float* __restrict__ U_pos, float* __restrict__ U_neg, float* __restrict__ S_pos, float* __restrict__ S_neg,
+                 int* __restrict__ k_pos, int* __restrict__ k_neg, int* __restrict__ sweeps_out) {
+    extern __shared__ double sv_sm[];
+    double* G = sv_sm;                      // [d][d], column j at G + j * d
+    double* sig = G + (size_t)d * d;        // [d]
+    int* order = reinterpret_cast<int*>(sig + d);   // [d]: position of column j in the sorted output
+    __shared__ int rotated;
+    const int sign = blockIdx.x / slots, slot = blockIdx.x % slots;
+    const float* om = (sign == 0 ? omega_pos : omega_neg) + (size_t)slot * d * d;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, n_warps = SV_THREADS / 32;
+    for (int idx = tid; idx < d * d; idx += SV_THREADS) {
+        const int i = idx / d, j = idx - i * d;     // Omega[i][j], coalesced read
+        G[(size_t)j * d + i] = (double)om[idx];
+    }
+    __syncthreads();
+    const int per_lane = d / 32;                    // d is 64 or 128
+    int sweep = 0;
+    for (; sweep < SV_MAX_SWEEPS; ++sweep) {
+        if (tid == 0) rotated = 0;
+        __syncthreads();
+        for (int rd = 0; rd < d - 1; ++rd) {
+            for (int i = warp; i < d / 2; i += n_warps) {
+                int a, b;
+                sv_pair(d, rd, i, a, b);
+                double* ga = G + (size_t)a * d;
+                double* gb = G + (size_t)b * d;
+                double x[4], y[4];
+                double aa = 0.0, bb = 0.0, ab = 0.0;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    if (e < per_lane) {
+                        x[e] = ga[lane + 32 * e]; y[e] = gb[lane + 32 * e];
+                        aa = fma(x[e], x[e], aa); bb = fma(y[e], y[e], bb); ab = fma(x[e], y[e], ab);
+                    }
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    aa += __shfl_xor_sync(0xffffffffu, aa, o);
+                    bb += __shfl_xor_sync(0xffffffffu, bb, o);
+                    ab += __shfl_xor_sync(0xffffffffu, ab, o);
+                }
+                // every lane holds the same three sums (the butterfly adds in the same order on every lane)
+                if (fabs(ab) > 1e-13 * sqrt(aa * bb) && aa > 0.0 && bb > 0.0) {     // well above the rounding noise of the dot product
+                    const double zeta = (bb - aa) / (2.0 * ab);
+                    const double t = (zeta >= 0.0 ? 1.0 : -1.0) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
+                    const double cs = 1.0 / sqrt(1.0 + t * t), sn = cs * t;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        if (e < per_lane) {
+                            ga[lane + 32 * e] = cs * x[e] - sn * y[e];
+                            gb[lane + 32 * e] = sn * x[e] + cs * y[e];
+                        }
+                    }
+                    if (lane == 0) rotated = 1;
+                }
+            }
+            __syncthreads();
+        }
+        if (rotated == 0) break;                    // a whole sweep without a rotation: the columns are orthogonal
+        __syncthreads();
+    }
+    // singular values = column norms
+    for (int j = warp; j < d; j += n_warps) {
+        double ss = 0.0;
+        for (int i = lane; i < d; i += 32) ss = fma(G[(size_t)j * d + i], G[(size_t)j * d + i], ss);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        if (lane == 0) sig[j] = sqrt(ss);
+    }
+    __syncthreads();
+    // descending order (ties: the earlier column first)
+    for (int j = tid; j < d; j += SV_THREADS) {
+        int r = 0;
+        for (int i = 0; i < d; ++i) r += (sig[i] > sig[j] || (sig[i] == sig[j] && i < j)) ? 1 : 0;
+        order[j] = r;
+    }
+    __syncthreads();
+    float* Uo = (sign == 0 ? U_pos : U_neg) + (size_t)slot * d * d;
+    float* So = (sign == 0 ? S_pos : S_neg) + (size_t)slot * d;
+    for (int idx = tid; idx < d * d; idx += SV_THREADS) {
+        const int i = idx / d, j = idx - i * d;     // component i of column j
+        const double s = sig[j];
+        Uo[(size_t)i * d + order[j]] = s > 0.0 ? (float)(G[(size_t)j * d + i] / s) : 0.f;
+    }
+    for (int j = tid; j < d; j += SV_THREADS) So[order[j]] = (float)sig[j];
+    __syncthreads();
+    if (tid == 0) {
+        // Eq. 3 on the sorted values, in fp64
+        double* sorted = G;                         // the matrix has been written out: reuse its first d entries
+        for (int j = 0; j < d; ++j) sorted[order[j]] = sig[j];
+        double total = 0.0;
+        for (int j = 0; j < d; ++j) total += sorted[j];
+        double run = 0.0;
+        int k = d;
+        for (int j = 0; j < d; ++j) {
+            run += sorted[j];
+            if (run >= (double)gamma * total) { k = j + 1; break; }
+        }
+        (sign == 0 ? k_pos : k_neg)[slot] = k;
+        if (sweeps_out != nullptr) sweeps_out[blockIdx.x] = sweep;
+    }
+}
+
+struct LearnPlan {
+    int n_groups, chunk_tokens, n_chunks, dist_tokens, dist_blocks;
+    size_t part_off, part_bytes, dsum_off, dsum_bytes, dcnt_off, dcnt_bytes, sweeps_off, sweeps_bytes, total;
+};
+
+seka_status validate_learn(const seka_learn_shape* s) {
+    if (s == nullptr) return SEKA_ERR_INVALID_ARG;
+    if (s->n_tokens <= 0 || s->n_slots <= 0) return SEKA_ERR_INVALID_ARG;
+    if (!(s->gamma > 0.f) || !(s->gamma <= 1.f)) return SEKA_ERR_INVALID_ARG;
+    if (s->head_dim != 64 && s->head_dim != 128) return SEKA_ERR_UNSUPPORTED;
+    if (s->head_dim == 64 && (s->n_slots & 1)) return SEKA_ERR_UNSUPPORTED;       // heads of 64 are processed in pairs
+    if ((long long)s->n_tokens * s->n_slots > 0x7fffffffLL) return SEKA_ERR_UNSUPPORTED;
+    return SEKA_OK;
+}
+
+// Chunks of tokens: a few items per SM so that the accumulator drain of one item hides under the next, but long
+// enough (>= 2048 tokens) that the partials stay small next to the embeddings.
+LearnPlan learn_plan(const seka_learn_shape* s) {
+    LearnPlan pl;
+    const int d = s->head_dim;
+    pl.n_groups = d == 128 ? s->n_slots : s->n_slots / 2;
+    long long want = (4LL * 148 + pl.n_groups - 1) / pl.n_groups;          // chunks that give about 4 items per SM
+    if (want < 1) want = 1;
+    long long chunk = (s->n_tokens + want - 1) / want;
+    if (chunk < 2048) chunk = 2048;
+    chunk = (chunk + LC_TOK - 1) / LC_TOK * LC_TOK;
+    pl.chunk_tokens = (int)chunk;
+    pl.n_chunks = (int)((s->n_tokens + chunk - 1) / chunk);
+    pl.dist_tokens = 64;
+    pl.dist_blocks = (s->n_tokens + pl.dist_tokens - 1) / pl.dist_tokens;
+    if (pl.dist_blocks > 2048) { pl.dist_tokens = (s->n_tokens + 2047) / 2048; pl.dist_blocks = (s->n_tokens + pl.dist_tokens - 1) / pl.dist_tokens; }
+    pl.part_off = kStatusBytes;
+    pl.part_bytes = align_up((size_t)pl.n_chunks * s->n_slots * 2 * d * d * sizeof(float), 256);
+    pl.dsum_off = pl.part_off + pl.part_bytes;
+    pl.dsum_bytes = align_up((size_t)pl.dist_blocks * s->n_slots * sizeof(float), 256);
+    pl.dcnt_off = pl.dsum_off + pl.dsum_bytes;
+    pl.dcnt_bytes = align_up((size_t)pl.dist_blocks * sizeof(int), 256);
+    pl.sweeps_off = pl.dcnt_off + pl.dcnt_bytes;
+    pl.sweeps_bytes = align_up((size_t)2 * s->n_slots * sizeof(int), 256);
+    pl.total = pl.sweeps_off + pl.sweeps_bytes;
+    return pl;
+}
+
+}  // namespace
+}  // namespace seka
+
+extern "C" size_t seka_learn_workspace_bytes(const seka_learn_shape* shape) {
+    if (seka::validate_learn(shape) != SEKA_OK) return 0;
+    return seka::learn_plan(shape).total;
+}
+
+extern "C" seka_status seka_learn_projections(const seka_learn_shape* shape, const void* h, const void* h_pos,
+                                              const void* h_neg, const uint8_t* answer_tokens,
+                                              float* omega_pos, float* omega_neg, float* U_pos, float* U_neg,
+                                              float* S_pos, float* S_neg, int32_t* k_pos, int32_t* k_neg, float* D,
+                                              void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    using namespace seka;
+    seka_status stc = validate_learn(shape);
+    if (stc != SEKA_OK) return stc;
+    if (!h || !h_pos || !h_neg || !omega_pos || !omega_neg || !U_pos || !U_neg || !S_pos || !S_neg || !k_pos || !k_neg || !D)
+        return SEKA_ERR_INVALID_ARG;
+    if (((uintptr_t)h | (uintptr_t)h_pos | (uintptr_t)h_neg | (uintptr_t)omega_pos | (uintptr_t)omega_neg) & 15) return SEKA_ERR_INVALID_ARG;
+    const LearnPlan pl = learn_plan(shape);
+    if (!workspace || workspace_bytes < pl.total || ((uintptr_t)workspace & 255)) return SEKA_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    char* ws = static_cast<char*>(workspace);
+    const int d = shape->head_dim, slots = shape->n_slots, n = shape->n_tokens;
+
+    static bool configured = false;
+    static int n_sm = 0;
+    if (!configured) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm <= 0) return SEKA_ERR_CUDA;
+        if (cudaFuncSetAttribute(learn_cov_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LC_DYN_BYTES) != cudaSuccess ||
+            cudaFuncSetAttribute(learn_svd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)(sizeof(double) * (128 * 128 + 128) + sizeof(int) * 128)) != cudaSuccess)
+            return SEKA_ERR_CUDA;
+        configured = true;
+    }
+
+    // cross-covariances: columns in groups of 128 (one head of 128, or two neighbouring heads of 64)
+    CUtensorMap tmH, tmP, tmN;
+    if (!make_tile_map(&tmH, h, 128, pl.n_groups, n, LC_TOK) || !make_tile_map(&tmP, h_pos, 128, pl.n_groups, n, LC_TOK) ||
+        !make_tile_map(&tmN, h_neg, 128, pl.n_groups, n, LC_TOK))
+        return SEKA_ERR_CUDA;
+    LearnCovParams p;
+    p.part = reinterpret_cast<float*>(ws + pl.part_off);
+    p.n_tokens = n; p.n_groups = pl.n_groups; p.d = d; p.slots = slots;
+    p.chunk_tokens = pl.chunk_tokens; p.n_chunks = pl.n_chunks; p.status = reinterpret_cast<int*>(ws);
+    const int n_items = pl.n_groups * pl.n_chunks;
+    learn_cov_kernel<<<n_items < n_sm ? n_items : n_sm, LC_THREADS, LC_DYN_BYTES, st>>>(tmH, tmP, tmN, p);
+    ++g_launches;
+    const size_t total = (size_t)slots * 2 * d * d;
+    learn_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(p.part, omega_pos, omega_neg, slots, d, pl.n_chunks, 1.f / (float)n);
+    ++g_launches;
+
+    // head-selection distance
+    float* dsum = reinterpret_cast<float*>(ws + pl.dsum_off);
+    int* dcnt = reinterpret_cast<int*>(ws + pl.dcnt_off);
+    learn_dist_kernel<<<pl.dist_blocks, LD_THREADS, slots * sizeof(float), st>>>(
+        static_cast<const __nv_bfloat16*>(h_pos), static_cast<const __nv_bfloat16*>(h_neg), answer_tokens, n, slots, d,
+        pl.dist_tokens, dsum, dcnt);
+    ++g_launches;
+    learn_dist_reduce_kernel<<<(slots + 127) / 128, 128, 0, st>>>(dsum, dcnt, pl.dist_blocks, slots, D);
+    ++g_launches;
+
+    // SVD of every Omega, rank rule
+    const size_t sv_smem = sizeof(double) * ((size_t)d * d + d) + sizeof(int) * d;
+    learn_svd_kernel<<<2 * slots, SV_THREADS, sv_smem, st>>>(omega_pos, omega_neg, slots, d, shape->gamma, U_pos, U_neg,
+                                                           S_pos, S_neg, k_pos, k_neg, reinterpret_cast<int*>(ws + pl.sweeps_off));
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? SEKA_OK : SEKA_ERR_CUDA;
+}
