@@ -257,6 +257,7 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle work for cpu_baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-edit-bench", action="store_true", help="skip the stand-alone key-edit measurement")
+    ap.add_argument("--learn-tokens", type=int, default=32768, help="tokens per embedding tensor in the learning measurement")
     ap.add_argument("--no-learn-bench", action="store_true", help="skip the offline spectral-learning measurement")
     ap.add_argument("--no-decode-bench", action="store_true", help="skip the decode-over-edited-cache measurement")
     args = ap.parse_args()
@@ -363,7 +364,7 @@ def main():
         edit_res = edit_keys_bench(w, measured_peaks())
     learn_res = None
     if rank == 0 and world == 1 and not args.no_learn_bench:
-        learn_res = learn_bench(measured_peaks())
+        learn_res = learn_bench(measured_peaks(), n=args.learn_tokens)
     decode_res = None
     if rank == 0 and world == 1 and not args.no_decode_bench:
         decode_res = decode_bench(w, measured_peaks())

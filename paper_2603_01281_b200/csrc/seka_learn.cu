@@ -220,18 +220,35 @@ __global__ void learn_dist_kernel(const __nv_bfloat16* __restrict__ hp, const __
     for (int t = t0; t < t1; ++t) {
         if (answer != nullptr && answer[t] == 0) continue;
         ++count;
-        for (int s = warp; s < slots; s += LD_THREADS / 32) {
-            const size_t base = ((size_t)t * slots + s) * d;
-            float ss = 0.f;
-            for (int i = 2 * lane; i < d; i += 64) {
-                const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(hp + base + i));
-                const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(hn + base + i));
-                const float dx = a.x - b.x, dy = a.y - b.y;
-                ss = fmaf(dx, dx, fmaf(dy, dy, ss));
+        // four slots of the warp at a time: their loads and reductions are independent
+        for (int s0 = warp; s0 < slots; s0 += 4 * (LD_THREADS / 32)) {
+            float ss[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int s = s0 + u * (LD_THREADS / 32);
+                ss[u] = 0.f;
+                if (s < slots) {
+                    const size_t base = ((size_t)t * slots + s) * d;
+                    for (int i = 2 * lane; i < d; i += 64) {
+                        const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(hp + base + i));
+                        const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(hn + base + i));
+                        const float dx = a.x - b.x, dy = a.y - b.y;
+                        ss[u] = fmaf(dx, dx, fmaf(dy, dy, ss[u]));
+                    }
+                }
             }
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-            if (lane == 0) acc[s] += sqrtf(ss);
+            for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u) ss[u] += __shfl_xor_sync(0xffffffffu, ss[u], o);
+            }
+            if (lane == 0) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int s = s0 + u * (LD_THREADS / 32);
+                    if (s < slots) acc[s] += sqrtf(ss[u]);
+                }
+            }
         }
     }
     __syncthreads();
@@ -239,18 +256,28 @@ __global__ void learn_dist_kernel(const __nv_bfloat16* __restrict__ hp, const __
     if (threadIdx.x == 0) part_count[blockIdx.x] = count;
 }
 
+// One CTA per slot: thread i adds the partials of blocks i, i + 256, ... in order, then thread 0 adds the 256 sums in order.
 __global__ void learn_dist_reduce_kernel(const float* __restrict__ part_sum, const int* __restrict__ part_count,
                                          int n_blocks, int slots, float* __restrict__ D) {
-    const int s = blockIdx.x * blockDim.x + threadIdx.x;
-    if (s >= slots) return;
-    double tot = 0.0;
-    long long cnt = 0;
-    for (int b = 0; b < n_blocks; ++b) { tot += (double)part_sum[(size_t)b * slots + s]; cnt += part_count[b]; }
-    D[s] = cnt > 0 ? (float)(tot / (double)cnt) : 0.f;
+    __shared__ double tot[256];
+    __shared__ long long cnt[256];
+    const int s = blockIdx.x, i = threadIdx.x;
+    double t = 0.0;
+    long long c = 0;
+    for (int b = i; b < n_blocks; b += 256) { t += (double)part_sum[(size_t)b * slots + s]; c += part_count[b]; }
+    tot[i] = t; cnt[i] = c;
+    __syncthreads();
+    if (i == 0) {
+        double tt = 0.0;
+        long long cc = 0;
+        for (int k = 0; k < 256; ++k) { tt += tot[k]; cc += cnt[k]; }
+        D[s] = cc > 0 ? (float)(tt / (double)cc) : 0.f;
+    }
 }
 
 // ------------------------------------------------------------------------------------ SVD (one-sided Jacobi, fp64)
-constexpr int SV_THREADS = 512;
+constexpr int SV_THREADS = 1024;
+constexpr int SV_PPW = 2;                       // column pairs per warp and round: 64 pairs over 32 warps
 constexpr int SV_MAX_SWEEPS = 60;
 
 // Column pair of position `i` in round `rd` of the round-robin tournament over d columns (d even): the last column
@@ -274,6 +301,8 @@ learn_svd_kernel(const float* __restrict__ omega_pos, const float* __restrict__ 
     double* sig = G + (size_t)d * d;        // [d]
     int* order = reinterpret_cast<int*>(sig + d);   // [d]: position of column j in the sorted output
     __shared__ int rotated;
+    uint8_t* sched = reinterpret_cast<uint8_t*>(order + d);      // [d - 1][d / 2][2]: the pairs of every round
+    __shared__ double pr[64], rot[2 * 64], nrm2[128], scale;
     const int sign = blockIdx.x / slots, slot = blockIdx.x % slots;
     const float* om = (sign == 0 ? omega_pos : omega_neg) + (size_t)slot * d * d;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, n_warps = SV_THREADS / 32;
@@ -282,45 +311,107 @@ learn_svd_kernel(const float* __restrict__ omega_pos, const float* __restrict__ 
         G[(size_t)j * d + i] = (double)om[idx];
     }
     __syncthreads();
+    // scale the matrix to unit largest entry (squares of column norms stay far from under- and overflow)
+    {
+        double mx = 0.0;
+        for (int idx = tid; idx < d * d; idx += SV_THREADS) mx = fmax(mx, fabs(G[idx]));
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx = fmax(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        if (lane == 0) pr[warp] = mx;
+        __syncthreads();
+        if (tid == 0) {
+            double m2 = 0.0;
+            for (int w = 0; w < n_warps; ++w) m2 = fmax(m2, pr[w]);
+            scale = m2;
+        }
+        __syncthreads();
+        const double inv = scale > 0.0 ? 1.0 / scale : 0.0;
+        for (int idx = tid; idx < d * d; idx += SV_THREADS) G[idx] *= inv;
+        __syncthreads();
+    }
     const int per_lane = d / 32;                    // d is 64 or 128
+    const int n_pairs = d / 2;
+    // the tournament schedule, once: pair (a, b) of position i in round rd
+    for (int idx = tid; idx < (d - 1) * n_pairs; idx += SV_THREADS) {
+        int pa, pb;
+        sv_pair(d, idx / n_pairs, idx % n_pairs, pa, pb);
+        sched[2 * idx] = (uint8_t)pa; sched[2 * idx + 1] = (uint8_t)pb;
+    }
     int sweep = 0;
     for (; sweep < SV_MAX_SWEEPS; ++sweep) {
         if (tid == 0) rotated = 0;
+        // squared column norms, exact at the start of every sweep; inside the sweep they follow the rotations
+        // (a' . a' = a . a - t a . b,  b' . b' = b . b + t a . b), so that a pair costs one inner product, not three
+        for (int j = warp; j < d; j += n_warps) {
+            double ss = 0.0;
+            for (int i = lane; i < d; i += 32) ss = fma(G[(size_t)j * d + i], G[(size_t)j * d + i], ss);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+            if (lane == 0) nrm2[j] = ss;
+        }
         __syncthreads();
         for (int rd = 0; rd < d - 1; ++rd) {
-            for (int i = warp; i < d / 2; i += n_warps) {
-                int a, b;
-                sv_pair(d, rd, i, a, b);
-                double* ga = G + (size_t)a * d;
-                double* gb = G + (size_t)b * d;
-                double x[4], y[4];
-                double aa = 0.0, bb = 0.0, ab = 0.0;
+            // phase 1: the inner product of every pair of the round (one warp per pair, SV_PPW pairs per warp)
+            double x[SV_PPW][4], y[SV_PPW][4];
+            int ca[SV_PPW], cb[SV_PPW];
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    if (e < per_lane) {
-                        x[e] = ga[lane + 32 * e]; y[e] = gb[lane + 32 * e];
-                        aa = fma(x[e], x[e], aa); bb = fma(y[e], y[e], bb); ab = fma(x[e], y[e], ab);
-                    }
-                }
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) {
-                    aa += __shfl_xor_sync(0xffffffffu, aa, o);
-                    bb += __shfl_xor_sync(0xffffffffu, bb, o);
-                    ab += __shfl_xor_sync(0xffffffffu, ab, o);
-                }
-                // every lane holds the same three sums (the butterfly adds in the same order on every lane)
-                if (fabs(ab) > 1e-13 * sqrt(aa * bb) && aa > 0.0 && bb > 0.0) {     // well above the rounding noise of the dot product
-                    const double zeta = (bb - aa) / (2.0 * ab);
-                    const double t = (zeta >= 0.0 ? 1.0 : -1.0) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
-                    const double cs = 1.0 / sqrt(1.0 + t * t), sn = cs * t;
+            for (int j = 0; j < SV_PPW; ++j) {
+                const int i = warp + n_warps * j;
+                if (i < n_pairs) {
+                    ca[j] = sched[2 * (rd * n_pairs + i)]; cb[j] = sched[2 * (rd * n_pairs + i) + 1];
+                    const double* ga = G + (size_t)ca[j] * d;
+                    const double* gb = G + (size_t)cb[j] * d;
+                    double ab = 0.0;
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         if (e < per_lane) {
-                            ga[lane + 32 * e] = cs * x[e] - sn * y[e];
-                            gb[lane + 32 * e] = sn * x[e] + cs * y[e];
+                            x[j][e] = ga[lane + 32 * e]; y[j][e] = gb[lane + 32 * e];
+                            ab = fma(x[j][e], y[j][e], ab);
                         }
                     }
-                    if (lane == 0) rotated = 1;
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) ab += __shfl_xor_sync(0xffffffffu, ab, o);
+                    if (lane == 0) pr[i] = ab;
+                }
+            }
+            __syncthreads();
+            // phase 2: one thread per pair works out the plane rotation that makes the two columns orthogonal
+            // (the scalar chain of a square root, a division and a reciprocal square root runs once, side by side
+            // in the lanes of two warps, instead of once per warp)
+            if (tid < n_pairs) {
+                const int pa = sched[2 * (rd * n_pairs + tid)], pb = sched[2 * (rd * n_pairs + tid) + 1];
+                const double aa = nrm2[pa], bb = nrm2[pb], ab = pr[tid];
+                double cs = 1.0, sn = 0.0;
+                if (ab * ab > 1e-26 * aa * bb && aa > 0.0 && bb > 0.0) {     // |cos| > 1e-13: well above the rounding noise
+                    const double delta = bb - aa, tau = 2.0 * ab;
+                    const double hyp = sqrt(fma(delta, delta, tau * tau));
+                    const double t = (delta >= 0.0 ? tau : -tau) / (fabs(delta) + hyp);
+                    cs = rsqrt(fma(t, t, 1.0));
+                    sn = cs * t;
+                    nrm2[pa] = fmax(aa - t * ab, 0.0);
+                    nrm2[pb] = bb + t * ab;
+                    rotated = 1;
+                }
+                rot[2 * tid] = cs; rot[2 * tid + 1] = sn;
+            }
+            __syncthreads();
+            // phase 3: apply
+#pragma unroll
+            for (int j = 0; j < SV_PPW; ++j) {
+                const int i = warp + n_warps * j;
+                if (i < n_pairs) {
+                    const double cs = rot[2 * i], sn = rot[2 * i + 1];
+                    if (sn != 0.0) {
+                        double* ga = G + (size_t)ca[j] * d;
+                        double* gb = G + (size_t)cb[j] * d;
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            if (e < per_lane) {
+                                ga[lane + 32 * e] = cs * x[j][e] - sn * y[j][e];
+                                gb[lane + 32 * e] = sn * x[j][e] + cs * y[j][e];
+                            }
+                        }
+                    }
                 }
             }
             __syncthreads();
@@ -334,7 +425,7 @@ learn_svd_kernel(const float* __restrict__ omega_pos, const float* __restrict__ 
         for (int i = lane; i < d; i += 32) ss = fma(G[(size_t)j * d + i], G[(size_t)j * d + i], ss);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-        if (lane == 0) sig[j] = sqrt(ss);
+        if (lane == 0) sig[j] = sqrt(ss);           // of the scaled matrix; the scale goes back on at the output
     }
     __syncthreads();
     // descending order (ties: the earlier column first)
@@ -351,7 +442,7 @@ learn_svd_kernel(const float* __restrict__ omega_pos, const float* __restrict__ 
         const double s = sig[j];
         Uo[(size_t)i * d + order[j]] = s > 0.0 ? (float)(G[(size_t)j * d + i] / s) : 0.f;
     }
-    for (int j = tid; j < d; j += SV_THREADS) So[order[j]] = (float)sig[j];
+    for (int j = tid; j < d; j += SV_THREADS) So[order[j]] = (float)(sig[j] * scale);
     __syncthreads();
     if (tid == 0) {
         // Eq. 3 on the sorted values, in fp64
@@ -398,9 +489,9 @@ LearnPlan learn_plan(const seka_learn_shape* s) {
     chunk = (chunk + LC_TOK - 1) / LC_TOK * LC_TOK;
     pl.chunk_tokens = (int)chunk;
     pl.n_chunks = (int)((s->n_tokens + chunk - 1) / chunk);
-    pl.dist_tokens = 64;
+    pl.dist_tokens = 8;
     pl.dist_blocks = (s->n_tokens + pl.dist_tokens - 1) / pl.dist_tokens;
-    if (pl.dist_blocks > 2048) { pl.dist_tokens = (s->n_tokens + 2047) / 2048; pl.dist_blocks = (s->n_tokens + pl.dist_tokens - 1) / pl.dist_tokens; }
+    if (pl.dist_blocks > 8192) { pl.dist_tokens = (s->n_tokens + 8191) / 8192; pl.dist_blocks = (s->n_tokens + pl.dist_tokens - 1) / pl.dist_tokens; }
     pl.part_off = kStatusBytes;
     pl.part_bytes = align_up((size_t)pl.n_chunks * s->n_slots * 2 * d * d * sizeof(float), 256);
     pl.dsum_off = pl.part_off + pl.part_bytes;
@@ -446,7 +537,7 @@ extern "C" seka_status seka_learn_projections(const seka_learn_shape* shape, con
             cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm <= 0) return SEKA_ERR_CUDA;
         if (cudaFuncSetAttribute(learn_cov_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LC_DYN_BYTES) != cudaSuccess ||
             cudaFuncSetAttribute(learn_svd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)(sizeof(double) * (128 * 128 + 128) + sizeof(int) * 128)) != cudaSuccess)
+                                 (int)(sizeof(double) * (128 * 128 + 128) + sizeof(int) * 128 + 127 * 128)) != cudaSuccess)
             return SEKA_ERR_CUDA;
         configured = true;
     }
@@ -474,11 +565,11 @@ extern "C" seka_status seka_learn_projections(const seka_learn_shape* shape, con
         static_cast<const __nv_bfloat16*>(h_pos), static_cast<const __nv_bfloat16*>(h_neg), answer_tokens, n, slots, d,
         pl.dist_tokens, dsum, dcnt);
     ++g_launches;
-    learn_dist_reduce_kernel<<<(slots + 127) / 128, 128, 0, st>>>(dsum, dcnt, pl.dist_blocks, slots, D);
+    learn_dist_reduce_kernel<<<slots, 256, 0, st>>>(dsum, dcnt, pl.dist_blocks, slots, D);
     ++g_launches;
 
     // SVD of every Omega, rank rule
-    const size_t sv_smem = sizeof(double) * ((size_t)d * d + d) + sizeof(int) * d;
+    const size_t sv_smem = sizeof(double) * ((size_t)d * d + d) + sizeof(int) * d + (size_t)(d - 1) * d;
     learn_svd_kernel<<<2 * slots, SV_THREADS, sv_smem, st>>>(omega_pos, omega_neg, slots, d, shape->gamma, U_pos, U_neg,
                                                            S_pos, S_neg, k_pos, k_neg, reinterpret_cast<int*>(ws + pl.sweeps_off));
     ++g_launches;
