@@ -71,3 +71,42 @@ def test_workspace_bytes_and_validation(lib):
                                   None, None, None, 0, None) == binding.SEKA_OK
     assert binding.status_string(binding.SEKA_ERR_TIMEOUT).startswith("a bounded")
     assert binding.seka_launch_count() == 0
+
+
+def test_decode_routed_and_learner_validation(lib):
+    one = ctypes.c_void_p(256)
+    s = shape()
+    # decode: partial results per (sequence, KV head, chunk, group head): at least the status block and one chunk
+    n = binding.seka_decode_workspace_bytes(s)
+    assert n >= 256 + 2 * 2 * 4 * (128 + 2) * 4
+    assert binding.seka_decode_workspace_bytes(shape(dtype=binding.SEKA_F32)) == 0        # bf16 caches only
+    assert binding.seka_decode_workspace_bytes(shape(n_q_heads=34)) == 0                  # 17 heads per KV head
+    assert binding.seka_decode_workspace_bytes(shape(head_dim=96)) == 0
+    assert lib.seka_decode_attention(ctypes.byref(shape(n_q_heads=34)), one, one, one, one, None, one, 1 << 30,
+                                     None) == binding.SEKA_ERR_UNSUPPORTED
+    assert lib.seka_decode_attention(ctypes.byref(s), None, one, one, one, None, one, 1 << 30, None) == binding.SEKA_ERR_INVALID_ARG
+    assert lib.seka_decode_attention(ctypes.byref(s), ctypes.c_void_p(264), one, one, one, None, one, 1 << 30,
+                                     None) == binding.SEKA_ERR_INVALID_ARG
+    assert lib.seka_decode_attention(ctypes.byref(s), one, one, one, one, None, one, 16, None) == binding.SEKA_ERR_WORKSPACE
+    assert lib.seka_decode_attention(ctypes.byref(shape(batch=0)), None, None, None, None, None, None, 0, None) == binding.SEKA_OK
+    # routed forward: needs mask, U and sigma, and k_route within the rank
+    args = [one, one, one, one, None]
+    assert lib.seka_attention_fwd_routed(ctypes.byref(s), *args, one, one, None, 0, None, one, None, one, 1 << 30,
+                                         None) == binding.SEKA_ERR_INVALID_ARG
+    assert lib.seka_attention_fwd_routed(ctypes.byref(s), *args, None, one, one, 0, None, one, None, one, 1 << 30,
+                                         None) == binding.SEKA_ERR_INVALID_ARG
+    assert lib.seka_attention_fwd_routed(ctypes.byref(s), *args, one, one, one, 33, None, one, None, one, 1 << 30,
+                                         None) == binding.SEKA_ERR_INVALID_ARG
+    assert lib.seka_attention_fwd_routed(ctypes.byref(s), *args, one, one, one, 0, None, one, None, one, 16,
+                                         None) == binding.SEKA_ERR_WORKSPACE
+    # learner
+    L = binding.SekaLearnShape
+    assert lib.seka_learn_workspace_bytes(ctypes.byref(L(1000, 4, 128, 0.7))) > 256 + 4 * 2 * 128 * 128 * 4
+    for bad in (L(0, 4, 128, 0.7), L(1000, 0, 128, 0.7), L(1000, 4, 96, 0.7), L(1000, 3, 64, 0.7),
+                L(1000, 4, 128, 0.0), L(1000, 4, 128, 1.5)):
+        assert lib.seka_learn_workspace_bytes(ctypes.byref(bad)) == 0
+        assert lib.seka_learn_projections(ctypes.byref(bad), *([one] * 14), 1 << 30, None) != 0
+    ok = L(1000, 4, 128, 0.7)
+    assert lib.seka_learn_projections(ctypes.byref(ok), None, *([one] * 13), 1 << 30, None) == binding.SEKA_ERR_INVALID_ARG
+    assert lib.seka_learn_projections(ctypes.byref(ok), *([one] * 14), 16, None) == binding.SEKA_ERR_WORKSPACE
+    assert binding.seka_launch_count() == 0
