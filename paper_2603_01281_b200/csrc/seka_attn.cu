@@ -600,10 +600,21 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             const int nX = x ? it.nB : it.nA;
             const int hqX = x ? it.hqB : it.hqA, qtX = x ? it.qtB : it.qtA;
             const uint8_t* hot_g = p.tile_hot + (size_t)it.b * p.n_qt;
+            // Every softmax warp waits for dK of EVERY highlighted key tile, in order, whether or not it helps to drain
+            // it: a warp that skipped a phase of e_full could find its next phase "complete" while the skipped one is
+            // still running (a parity wait only tells the current phase from the one before).  The waits cost nothing:
+            // the scores a warp needs next are issued after the edit anyway.
+            auto see_edit = [&](int j0, int j1) {
+                for (int j = j0; j < j1 && ok; ++j) {
+                    if (hot_g[j] == 0) continue;
+                    ok = warp_wait(e_full, n_hot & 1, abort_flag, p.status, 38);
+                    ++n_hot;
+                }
+            };
             if (nX == 0) {      // tile B lies beyond the sequence: only the counts move
-                if (it.steer)
-                    for (int j = 0; j < it.n_kv; ++j) n_hot += hot_g[j] != 0 ? 1u : 0u;
+                if (it.steer) see_edit(0, it.n_kv);
                 pr += it.n_kv;
+                if (!ok) break;
                 continue;
             }
             float m_run = -INFINITY, l_run = 0.f;
@@ -613,11 +624,11 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                 // scores anyway, these warps add the upper half of the columns of dK to the staged K tile (the
                 // key editors take the lower half).  Every softmax warp counts the highlighted tiles.
                 if (it.steer && hot_g[j] != 0) {
+                    ok = warp_wait(e_full, n_hot & 1, abort_flag, p.status, 36 + x);
+                    if (!ok) break;
                     if ((j < it.nA ? 0 : 1) == x) {
                         const int kpos = j * BN + row;
                         const bool hl = kpos < it.Lb && p.mask[it.seq0 + kpos] != 0;
-                        ok = warp_wait(e_full, n_hot & 1, abort_flag, p.status, 36 + x);
-                        if (!ok) break;
                         tc_fence_after();
                         drain_edit(EDIT_OWN_COLS ? t_lane + COL_E : tS, smem + SL::K + ((pr + (uint32_t)j) % NK) * SL::TILE, row, hl, D / 64, D / 32);
                         fence_proxy_async();
@@ -698,9 +709,6 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                 const float2 s2 = __fadd2_rn(sum[0], sum[1]);
                 l_run = l_run * factor + (s2.x + s2.y);
             }
-            // highlighted tiles that only the other tile uses are counted too
-            if (it.steer)
-                for (int j = nX; j < it.n_kv; ++j) n_hot += hot_g[j] != 0 ? 1u : 0u;
             cX += nX; pr += it.n_kv;
             if (ok) ok = warp_wait(o_full + x, n_o & 1, abort_flag, p.status, 44 + x);
             ++n_o;
@@ -722,6 +730,8 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                 if (valid && p.lse != nullptr) p.lse[orow] = (m_run + log2f(l_run)) * 0.6931471805599453f;
                 tc_fence_before();
             }
+            // highlighted tiles that only the other tile uses are seen too (after the output is on its way)
+            if (it.steer && ok) see_edit(nX, it.n_kv);
         }
     }
 

@@ -278,6 +278,21 @@ def test_more_items_than_sms():
     _fused_vs_oracle(w, head_enable=he, rows=rows, label="152 items")
 
 
+@pytest.mark.parametrize("d", [64, 128])
+def test_every_tile_highlighted_with_odd_group(d):
+    """Odd group size (here MHA): an item pairs two consecutive row tiles, so the last key tile of an item is used
+    by its second tile only.  With every token highlighted and many short sequences each persistent CTA walks items
+    whose first and last key tiles are both edited, back to back: the softmax warps of the first tile then reach
+    the next item's first edit while the previous item's last one is still being formed."""
+    rng = np.random.default_rng(61)
+    lens = [int(x) for x in rng.integers(130, 640, size=96)]
+    w = inputs.make_custom(seed=61, dtype="bf16", lens=lens, n_q_heads=3, n_kv_heads=3, head_dim=d, rank=16,
+                           mask_kind="all", gain=0.5)
+    rows = H.sampled_rows(w, 6, seed=4)
+    for _ in range(3):
+        _fused_vs_oracle(w, rows=rows, label="all tiles hot, d=%d" % d, short_rows=True)
+
+
 # ----------------------------------------------------------------- AdaSEKA in one call (routing inside the preparation launch)
 
 @pytest.mark.parametrize("case", ["C3", "small_f32", "small_varlen"])
