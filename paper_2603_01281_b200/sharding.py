@@ -2,6 +2,7 @@
 
 The path has no exchange step: a sequence (and within it a KV-head group) needs only its own Q, K, V, mask,
 gain and routing coefficients, so N ranks take N disjoint sets of sequences and never talk on the data path.
+The decode step shards the same way (by sequence), the offline learner by slot (`shard_slots`).
 What crosses ranks is bookkeeping only: a barrier around timed regions and the maximum of the ranks' device
 times.  These helpers hold that bookkeeping; they work on any torch.distributed backend (NCCL on GPUs, gloo in
 the CPU tests).
@@ -29,6 +30,19 @@ def shard_tokens(cu_seqlens: Sequence[int], world: int, rank: int) -> Tuple[int,
     first, last = shard_sequences(len(cu_seqlens) - 1, world, rank)
     t0, t1 = int(cu_seqlens[first]), int(cu_seqlens[last])
     return t0, t1, [int(c) - t0 for c in cu_seqlens[first:last + 1]]
+
+
+def shard_slots(n_slots: int, world: int, rank: int, pair: bool = False) -> Tuple[int, int]:
+    """Range [first, last) of (layer, KV head) slots of the offline learner owned by `rank`: slots are learned
+    independently (one cross-covariance pair and two SVDs each), so N ranks take N disjoint ranges of the slot axis
+    and exchange nothing.  With `pair` (head_dim 64: neighbouring heads share a tensor-core product) the ranges
+    start and end on even slots."""
+    if pair:
+        if n_slots % 2:
+            raise ValueError("an even number of slots is needed when heads are processed in pairs")
+        first, last = shard_sequences(n_slots // 2, world, rank)
+        return 2 * first, 2 * last
+    return shard_sequences(n_slots, world, rank)
 
 
 def rank_seed_offset(rank: int) -> int:

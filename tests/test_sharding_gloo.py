@@ -32,6 +32,16 @@ def _worker(rank, world, port, out_dir):
         O, lse, _ = oracle.seka_attention(w.Q[t0:t1], w.K[t0:t1], w.V[t0:t1], w.mask[t0:t1], np.asarray(cu, dtype=np.int32),
                                           w.U, gain=w.gain[first:last])
         np.save(os.path.join(out_dir, "O_%d.npy" % rank), O)
+        # the decode step over the (edited) cache shards by sequence in the same way
+        q = np.stack([w.Q[c - 1] if c > w.cu_seqlens[i] else np.zeros_like(w.Q[0])
+                      for i, c in enumerate(w.cu_seqlens[1:])])
+        Od, _ = oracle.seka_decode(q[first:last], w.K[t0:t1], w.V[t0:t1], w.mask[t0:t1], cu, w.U, gain=w.gain[first:last])
+        np.save(os.path.join(out_dir, "Od_%d.npy" % rank), Od)
+        # the offline learner shards by slot
+        h, hp, hn, ans, _, _ = inputs.contrastive_embeddings(seed=2, n=300, slots=6, head_dim=16, rank=3, dtype="f32")
+        s0, s1 = sharding.shard_slots(6, world, rank, pair=True)
+        res = oracle.learn_projections(h[:, s0:s1], hp[:, s0:s1], hn[:, s0:s1], 0.7, answer_tokens=ans)
+        np.save(os.path.join(out_dir, "S_%d.npy" % rank), np.concatenate([res["S_pos"], res["D"][:, None]], axis=1))
         # timing bookkeeping: the slowest rank decides, every rank learns it
         slow = sharding.max_over_ranks(10.0 + rank)
         assert slow == 10.0 + world - 1
@@ -53,6 +63,23 @@ def test_two_ranks_shard_by_sequence_without_exchange(tmp_path):
     parts = np.concatenate([np.load(tmp_path / ("O_%d.npy" % r)) for r in range(world)], axis=0)
     assert parts.shape == whole.shape
     assert np.array_equal(parts, whole)         # the same arithmetic on the same rows: bit-identical
+    q = np.stack([w.Q[c - 1] if c > w.cu_seqlens[i] else np.zeros_like(w.Q[0]) for i, c in enumerate(w.cu_seqlens[1:])])
+    whole_d, _ = oracle.seka_decode(q, w.K, w.V, w.mask, w.cu_seqlens, w.U, gain=w.gain)
+    parts_d = np.concatenate([np.load(tmp_path / ("Od_%d.npy" % r)) for r in range(world)], axis=0)
+    assert np.array_equal(parts_d, whole_d)
+    h, hp, hn, ans, _, _ = inputs.contrastive_embeddings(seed=2, n=300, slots=6, head_dim=16, rank=3, dtype="f32")
+    res = oracle.learn_projections(h, hp, hn, 0.7, answer_tokens=ans)
+    parts_s = np.concatenate([np.load(tmp_path / ("S_%d.npy" % r)) for r in range(world)], axis=0)
+    assert np.array_equal(parts_s, np.concatenate([res["S_pos"], res["D"][:, None]], axis=1))
+
+
+def test_slot_ranges_partition_the_slots():
+    for n in (2, 6, 288):
+        for world in (1, 2, 4, 8):
+            for pair in (False, True):
+                r = [sharding.shard_slots(n, world, k, pair=pair) for k in range(world)]
+                assert r[0][0] == 0 and r[-1][1] == n and all(r[k][1] == r[k + 1][0] for k in range(world - 1))
+                assert not pair or all(a % 2 == 0 and b % 2 == 0 for a, b in r)
 
 
 def test_shard_ranges_partition_the_batch():
