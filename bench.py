@@ -33,7 +33,7 @@ METRIC = "SEKA fused attention TFLOP/s (% BF16 peak); overhead vs g=0, 8B shape"
 WORKLOAD = "C2: 8B-shaped prefill layer B=4 Hq=32 Hkv=8 d=128 L=4096 bf16, rank 32, ~10% highlighted spans, g=1"
 # DRAM bytes of one fused-kernel launch on this workload from the ncu capture summarised in
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture exists.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 437662720  # profiles/seka_attn_fwd_kernel_d128_C2.md (324.03 MB read + 96.06 MB written)
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 437662720  # profiles/seka_attn_fwd_kernel_d128_C2.md (341.05 MB read + 96.61 MB written)
 
 
 def measured_peaks():
