@@ -277,7 +277,6 @@ __global__ void learn_dist_reduce_kernel(const float* __restrict__ part_sum, con
 
 // ------------------------------------------------------------------------------------ SVD (one-sided Jacobi, fp64)
 constexpr int SV_THREADS = 1024;
-constexpr int SV_PPW = 2;                       // column pairs per warp and round: 64 pairs over 32 warps
 constexpr int SV_MAX_SWEEPS = 60;
 
 // Column pair of position `i` in round `rd` of the round-robin tournament over d columns (d even): the last column
@@ -302,7 +301,7 @@ learn_svd_kernel(const float* __restrict__ omega_pos, const float* __restrict__ 
     int* order = reinterpret_cast<int*>(sig + d);   // [d]: position of column j in the sorted output
     __shared__ int rotated;
     uint8_t* sched = reinterpret_cast<uint8_t*>(order + d);      // [d - 1][d / 2][2]: the pairs of every round
-    __shared__ double pr[64], rot[2 * 64], nrm2[128], scale;
+    __shared__ double pr[64], rot[2 * 64], nrm2[128], scl[128], iscl[128], scale;
     const int sign = blockIdx.x / slots, slot = blockIdx.x % slots;
     const float* om = (sign == 0 ? omega_pos : omega_neg) + (size_t)slot * d * d;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, n_warps = SV_THREADS / 32;
@@ -329,7 +328,7 @@ learn_svd_kernel(const float* __restrict__ omega_pos, const float* __restrict__ 
         for (int idx = tid; idx < d * d; idx += SV_THREADS) G[idx] *= inv;
         __syncthreads();
     }
-    const int per_lane = d / 32;                    // d is 64 or 128
+    const int per_lane = d / 16;                    // rows per lane: a column pair is worked by 16 lanes (d is 64 or 128)
     const int n_pairs = d / 2;
     // the tournament schedule, once: pair (a, b) of position i in round rd
     for (int idx = tid; idx < (d - 1) * n_pairs; idx += SV_THREADS) {
@@ -337,79 +336,105 @@ learn_svd_kernel(const float* __restrict__ omega_pos, const float* __restrict__ 
         sv_pair(d, idx / n_pairs, idx % n_pairs, pa, pb);
         sched[2 * idx] = (uint8_t)pa; sched[2 * idx + 1] = (uint8_t)pb;
     }
+    // Scaled (fast) rotations: column j of the matrix is scl[j] * g_j with g_j the stored column.  A rotation
+    //   A' = c (A - t B),  B' = c (B + t A)   becomes   g_a' = g_a - (t s_b / s_a) g_b,  g_b' = g_b + (t s_a / s_b) g_a
+    // (two multiply-adds per row instead of four operations) with s_a' = c s_a, s_b' = c s_b; the reciprocals are
+    // tracked too (1 / c = (1 + t^2) c), so no division is needed for the ratios.  The scales are folded back into
+    // the columns at the start of every sweep (c >= 1 / sqrt 2 per rotation, 127 rotations per sweep at most).
+    for (int j = tid; j < d; j += SV_THREADS) { scl[j] = 1.0; iscl[j] = 1.0; }
+    const int half = lane >> 4, l16 = lane & 15;
+    const int my_pair = 2 * warp + half;            // two pairs per warp, one per half-warp: 64 pairs over 32 warps
     int sweep = 0;
     for (; sweep < SV_MAX_SWEEPS; ++sweep) {
         if (tid == 0) rotated = 0;
-        // squared column norms, exact at the start of every sweep; inside the sweep they follow the rotations
-        // (a' . a' = a . a - t a . b,  b' . b' = b . b + t a . b), so that a pair costs one inner product, not three
+        __syncthreads();
+        // fold the scales, and the squared column norms, exact at the start of every sweep; inside the sweep they
+        // follow the rotations (A' . A' = A . A - t A . B,  B' . B' = B . B + t A . B): a pair costs one inner product
         for (int j = warp; j < d; j += n_warps) {
+            const double sj = scl[j];
             double ss = 0.0;
-            for (int i = lane; i < d; i += 32) ss = fma(G[(size_t)j * d + i], G[(size_t)j * d + i], ss);
+            for (int i = lane; i < d; i += 32) {
+                const double v = G[(size_t)j * d + i] * sj;
+                G[(size_t)j * d + i] = v;
+                ss = fma(v, v, ss);
+            }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-            if (lane == 0) nrm2[j] = ss;
+            __syncwarp();
+            if (lane == 0) { nrm2[j] = ss; scl[j] = 1.0; iscl[j] = 1.0; }
         }
         __syncthreads();
         for (int rd = 0; rd < d - 1; ++rd) {
-            // phase 1: the inner product of every pair of the round (one warp per pair, SV_PPW pairs per warp)
-            double x[SV_PPW][4], y[SV_PPW][4];
-            int ca[SV_PPW], cb[SV_PPW];
+            // phase 1: the inner product of the stored columns of every pair of the round
+            double x[8], y[8];
+            int ca = 0, cb = 0;
+            if (my_pair < n_pairs) {
+                ca = sched[2 * (rd * n_pairs + my_pair)]; cb = sched[2 * (rd * n_pairs + my_pair) + 1];
+                const double* ga = G + (size_t)ca * d;
+                const double* gb = G + (size_t)cb * d;
+                double ab = 0.0, ab1 = 0.0;              // two chains: dependent fp64 operations are slow
 #pragma unroll
-            for (int j = 0; j < SV_PPW; ++j) {
-                const int i = warp + n_warps * j;
-                if (i < n_pairs) {
-                    ca[j] = sched[2 * (rd * n_pairs + i)]; cb[j] = sched[2 * (rd * n_pairs + i) + 1];
-                    const double* ga = G + (size_t)ca[j] * d;
-                    const double* gb = G + (size_t)cb[j] * d;
-                    double ab = 0.0;
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        if (e < per_lane) {
-                            x[j][e] = ga[lane + 32 * e]; y[j][e] = gb[lane + 32 * e];
-                            ab = fma(x[j][e], y[j][e], ab);
-                        }
+                for (int e = 0; e < 8; e += 2) {
+                    if (e < per_lane) {
+                        x[e] = ga[l16 + 16 * e]; y[e] = gb[l16 + 16 * e];
+                        x[e + 1] = ga[l16 + 16 * (e + 1)]; y[e + 1] = gb[l16 + 16 * (e + 1)];
+                        ab = fma(x[e], y[e], ab);
+                        ab1 = fma(x[e + 1], y[e + 1], ab1);
                     }
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) ab += __shfl_xor_sync(0xffffffffu, ab, o);
-                    if (lane == 0) pr[i] = ab;
                 }
+                ab += ab1;
+#pragma unroll
+                for (int o = 8; o > 0; o >>= 1) ab += __shfl_xor_sync(0xffffffffu, ab, o);      // within the half-warp
+                if (l16 == 0) pr[my_pair] = ab;
             }
             __syncthreads();
-            // phase 2: one thread per pair works out the plane rotation that makes the two columns orthogonal
-            // (the scalar chain of a square root, a division and a reciprocal square root runs once, side by side
-            // in the lanes of two warps, instead of once per warp)
+            // phase 2: one thread per pair works out the rotation that makes the two columns orthogonal (the scalar
+            // chain of a square root, a division and a reciprocal square root runs once per pair, side by side)
             if (tid < n_pairs) {
                 const int pa = sched[2 * (rd * n_pairs + tid)], pb = sched[2 * (rd * n_pairs + tid) + 1];
-                const double aa = nrm2[pa], bb = nrm2[pb], ab = pr[tid];
-                double cs = 1.0, sn = 0.0;
+                const double sa = scl[pa], sb = scl[pb];
+                const double aa = nrm2[pa], bb = nrm2[pb], ab = sa * sb * pr[tid];
+                double ta = 0.0, tb = 0.0;
+                // The tangent of the rotation angle needs no more than single precision: an error eps in t leaves
+                // eps times the old inner product behind, which the next sweep removes; the rotation itself stays
+                // exact because the same t goes into both columns and into the scales.  Dependent fp64 operations
+                // are slow on this part, so the square root and the division of the textbook formula run in fp32
+                // and the cosine is one Newton step from an fp32 seed.
+                double t = 0.0;
                 if (ab * ab > 1e-26 * aa * bb && aa > 0.0 && bb > 0.0) {     // |cos| > 1e-13: well above the rounding noise
-                    const double delta = bb - aa, tau = 2.0 * ab;
-                    const double hyp = sqrt(fma(delta, delta, tau * tau));
-                    const double t = (delta >= 0.0 ? tau : -tau) / (fabs(delta) + hyp);
-                    cs = rsqrt(fma(t, t, 1.0));
-                    sn = cs * t;
+                    const float df = (float)(bb - aa), tf = (float)(2.0 * ab);
+                    const float mf = fmaxf(fabsf(df), fabsf(tf));
+                    if (mf > 0.f) {
+                        const float dn = df / mf, tn = tf / mf;
+                        t = (double)((dn >= 0.f ? tn : -tn) / (fabsf(dn) + sqrtf(fmaf(dn, dn, tn * tn))));
+                    }
+                }
+                if (t != 0.0) {
+                    const double t2 = fma(t, t, 1.0);
+                    const double c0 = (double)rsqrtf((float)t2);
+                    const double cs = c0 * fma(-0.5 * t2, c0 * c0, 1.5), ics = t2 * cs;
+                    ta = t * sb * iscl[pa];
+                    tb = t * sa * iscl[pb];
+                    scl[pa] = cs * sa; scl[pb] = cs * sb;
+                    iscl[pa] *= ics; iscl[pb] *= ics;
                     nrm2[pa] = fmax(aa - t * ab, 0.0);
                     nrm2[pb] = bb + t * ab;
                     rotated = 1;
                 }
-                rot[2 * tid] = cs; rot[2 * tid + 1] = sn;
+                rot[2 * tid] = ta; rot[2 * tid + 1] = tb;
             }
             __syncthreads();
             // phase 3: apply
+            if (my_pair < n_pairs) {
+                const double ta = rot[2 * my_pair], tb = rot[2 * my_pair + 1];
+                if (ta != 0.0 || tb != 0.0) {
+                    double* ga = G + (size_t)ca * d;
+                    double* gb = G + (size_t)cb * d;
 #pragma unroll
-            for (int j = 0; j < SV_PPW; ++j) {
-                const int i = warp + n_warps * j;
-                if (i < n_pairs) {
-                    const double cs = rot[2 * i], sn = rot[2 * i + 1];
-                    if (sn != 0.0) {
-                        double* ga = G + (size_t)ca[j] * d;
-                        double* gb = G + (size_t)cb[j] * d;
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            if (e < per_lane) {
-                                ga[lane + 32 * e] = cs * x[j][e] - sn * y[j][e];
-                                gb[lane + 32 * e] = sn * x[j][e] + cs * y[j][e];
-                            }
+                    for (int e = 0; e < 8; ++e) {
+                        if (e < per_lane) {
+                            ga[l16 + 16 * e] = fma(-ta, y[e], x[e]);
+                            gb[l16 + 16 * e] = fma(tb, x[e], y[e]);
                         }
                     }
                 }
@@ -419,6 +444,12 @@ learn_svd_kernel(const float* __restrict__ omega_pos, const float* __restrict__ 
         if (rotated == 0) break;                    // a whole sweep without a rotation: the columns are orthogonal
         __syncthreads();
     }
+    // fold the scales of the last sweep
+    for (int j = warp; j < d; j += n_warps) {
+        const double sj = scl[j];
+        for (int i = lane; i < d; i += 32) G[(size_t)j * d + i] *= sj;
+    }
+    __syncthreads();
     // singular values = column norms
     for (int j = warp; j < d; j += n_warps) {
         double ss = 0.0;
