@@ -276,17 +276,9 @@ __global__ void learn_dist_reduce_kernel(const float* __restrict__ part_sum, con
 }
 
 // ------------------------------------------------------------------------------------ SVD (one-sided Jacobi, fp64)
-constexpr int SV_THREADS = 1024;
+constexpr int SV_LP = 8;                        // lanes that share a column pair: four pairs per warp
+constexpr int SV_THREADS = 64 * SV_LP;          // 64 pairs per round at head_dim 128
 constexpr int SV_MAX_SWEEPS = 60;
-
-// Column pair of position `i` in round `rd` of the round-robin tournament over d columns (d even): the last column
-// stays in place and the others rotate, so that the d / 2 pairs of a round are disjoint and d - 1 rounds meet every pair.
-__device__ __forceinline__ void sv_pair(int d, int rd, int i, int& a, int& b) {
-    const int m = d - 1;
-    if (i == 0) { a = m; b = rd % m; }
-    else { a = (rd + i) % m; b = (rd - i + m) % m; }
-    if (a > b) { const int t = a; a = b; b = t; }
-}
 
 // One CTA per (sign, slot).  G (column-major, fp64, shared memory) starts as Omega; plane rotations from the right
 // make its columns mutually orthogonal: Omega V = U S.  Outputs: U [d x d] row-major with the singular vectors as
@@ -300,8 +292,8 @@ learn_svd_kernel(const float* __restrict__ omega_pos, const float* __restrict__ 
     double* sig = G + (size_t)d * d;        // [d]
     int* order = reinterpret_cast<int*>(sig + d);   // [d]: position of column j in the sorted output
     __shared__ int rotated;
-    uint8_t* sched = reinterpret_cast<uint8_t*>(order + d);      // [d - 1][d / 2][2]: the pairs of every round
-    __shared__ double pr[64], rot[2 * 64], nrm2[128], scl[128], iscl[128], scale;
+    __shared__ double pr[64], scl[128], iscl[128], scale;
+    __shared__ float nrm2[128];
     const int sign = blockIdx.x / slots, slot = blockIdx.x % slots;
     const float* om = (sign == 0 ? omega_pos : omega_neg) + (size_t)slot * d * d;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, n_warps = SV_THREADS / 32;
@@ -328,28 +320,37 @@ learn_svd_kernel(const float* __restrict__ omega_pos, const float* __restrict__ 
         for (int idx = tid; idx < d * d; idx += SV_THREADS) G[idx] *= inv;
         __syncthreads();
     }
-    const int per_lane = d / 16;                    // rows per lane: a column pair is worked by 16 lanes (d is 64 or 128)
+    constexpr int RPL = 128 / SV_LP;                // rows per lane at d = 128 (d = 64 uses the first half)
+    const int per_lane = d / SV_LP;
     const int n_pairs = d / 2;
-    // the tournament schedule, once: pair (a, b) of position i in round rd
-    for (int idx = tid; idx < (d - 1) * n_pairs; idx += SV_THREADS) {
-        int pa, pb;
-        sv_pair(d, idx / n_pairs, idx % n_pairs, pa, pb);
-        sched[2 * idx] = (uint8_t)pa; sched[2 * idx + 1] = (uint8_t)pb;
-    }
     // Scaled (fast) rotations: column j of the matrix is scl[j] * g_j with g_j the stored column.  A rotation
     //   A' = c (A - t B),  B' = c (B + t A)   becomes   g_a' = g_a - (t s_b / s_a) g_b,  g_b' = g_b + (t s_a / s_b) g_a
     // (two multiply-adds per row instead of four operations) with s_a' = c s_a, s_b' = c s_b; the reciprocals are
     // tracked too (1 / c = (1 + t^2) c), so no division is needed for the ratios.  The scales are folded back into
     // the columns at the start of every sweep (c >= 1 / sqrt 2 per rotation, 127 rotations per sweep at most).
+    //
+    // Ordering of a sweep (every pair of columns meets once, d - 1 rounds of d / 2 disjoint pairs): level l cuts
+    // the columns into blocks of 2 m, m = d / 2, d / 4, ..., 1; in round r of the level the i-th column of the first
+    // half of a block meets the ((i + r) mod m)-th column of its second half.  A group of SV_LP lanes owns one
+    // first-half column for the whole level and keeps it in registers; only the second-half columns go through
+    // shared memory (read, rotated, written back in place), and there is one barrier per round, since every group
+    // works out its own rotation.
+    //
+    // What bounds the kernel is the fp64 pipe (one warp instruction every 8-11 cycles per scheduler on this part),
+    // so the aim is few fp64 warp instructions per round: several pairs share a warp (the scalar work of a rotation
+    // is then issued once for all of them), the tangent and the squared norms are fp32, only what decides the
+    // orthogonality of the result stays fp64.
     for (int j = tid; j < d; j += SV_THREADS) { scl[j] = 1.0; iscl[j] = 1.0; }
-    const int half = lane >> 4, l16 = lane & 15;
-    const int my_pair = 2 * warp + half;            // two pairs per warp, one per half-warp: 64 pairs over 32 warps
+    const int grp = lane / SV_LP, lg = lane % SV_LP;
+    const int hw = (32 / SV_LP) * warp + grp;       // pair slot of a round
+    const bool active = hw < n_pairs;
     int sweep = 0;
     for (; sweep < SV_MAX_SWEEPS; ++sweep) {
         if (tid == 0) rotated = 0;
         __syncthreads();
         // fold the scales, and the squared column norms, exact at the start of every sweep; inside the sweep they
-        // follow the rotations (A' . A' = A . A - t A . B,  B' . B' = B . B + t A . B): a pair costs one inner product
+        // follow the rotations (A' . A' = A . A - t A . B,  B' . B' = B . B + t A . B) in fp32: they only feed the
+        // tangent.  A pair then costs one inner product.
         for (int j = warp; j < d; j += n_warps) {
             const double sj = scl[j];
             double ss = 0.0;
@@ -361,83 +362,88 @@ learn_svd_kernel(const float* __restrict__ omega_pos, const float* __restrict__ 
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
             __syncwarp();
-            if (lane == 0) { nrm2[j] = ss; scl[j] = 1.0; iscl[j] = 1.0; }
+            if (lane == 0) { nrm2[j] = (float)ss; scl[j] = 1.0; iscl[j] = 1.0; }
         }
         __syncthreads();
-        for (int rd = 0; rd < d - 1; ++rd) {
-            // phase 1: the inner product of the stored columns of every pair of the round
-            double x[8], y[8];
-            int ca = 0, cb = 0;
-            if (my_pair < n_pairs) {
-                ca = sched[2 * (rd * n_pairs + my_pair)]; cb = sched[2 * (rd * n_pairs + my_pair) + 1];
+        for (int m = n_pairs; m >= 1; m >>= 1) {
+            // the resident column of this group for the level, with its scale, reciprocal scale and squared norm
+            const int blk = hw / m, idx = hw - blk * m;
+            const int ca = blk * 2 * m + idx;
+            double x[RPL];
+            double sa = 1.0, isa = 1.0;
+            float aa = 0.f, saf = 1.f;
+            if (active) {
                 const double* ga = G + (size_t)ca * d;
-                const double* gb = G + (size_t)cb * d;
-                double ab = 0.0, ab1 = 0.0;              // two chains: dependent fp64 operations are slow
 #pragma unroll
-                for (int e = 0; e < 8; e += 2) {
-                    if (e < per_lane) {
-                        x[e] = ga[l16 + 16 * e]; y[e] = gb[l16 + 16 * e];
-                        x[e + 1] = ga[l16 + 16 * (e + 1)]; y[e + 1] = gb[l16 + 16 * (e + 1)];
-                        ab = fma(x[e], y[e], ab);
-                        ab1 = fma(x[e + 1], y[e + 1], ab1);
-                    }
-                }
-                ab += ab1;
-#pragma unroll
-                for (int o = 8; o > 0; o >>= 1) ab += __shfl_xor_sync(0xffffffffu, ab, o);      // within the half-warp
-                if (l16 == 0) pr[my_pair] = ab;
+                for (int e = 0; e < RPL; ++e)
+                    if (e < per_lane) x[e] = ga[lg + SV_LP * e];
+                sa = scl[ca]; isa = iscl[ca]; aa = nrm2[ca]; saf = (float)sa;
             }
-            __syncthreads();
-            // phase 2: one thread per pair works out the rotation that makes the two columns orthogonal (the scalar
-            // chain of a square root, a division and a reciprocal square root runs once per pair, side by side)
-            if (tid < n_pairs) {
-                const int pa = sched[2 * (rd * n_pairs + tid)], pb = sched[2 * (rd * n_pairs + tid) + 1];
-                const double sa = scl[pa], sb = scl[pb];
-                const double aa = nrm2[pa], bb = nrm2[pb], ab = sa * sb * pr[tid];
-                double ta = 0.0, tb = 0.0;
-                // The tangent of the rotation angle needs no more than single precision: an error eps in t leaves
-                // eps times the old inner product behind, which the next sweep removes; the rotation itself stays
-                // exact because the same t goes into both columns and into the scales.  Dependent fp64 operations
-                // are slow on this part, so the square root and the division of the textbook formula run in fp32
-                // and the cosine is one Newton step from an fp32 seed.
-                double t = 0.0;
-                if (ab * ab > 1e-26 * aa * bb && aa > 0.0 && bb > 0.0) {     // |cos| > 1e-13: well above the rounding noise
-                    const float df = (float)(bb - aa), tf = (float)(2.0 * ab);
-                    const float mf = fmaxf(fabsf(df), fabsf(tf));
-                    if (mf > 0.f) {
-                        const float dn = df / mf, tn = tf / mf;
-                        t = (double)((dn >= 0.f ? tn : -tn) / (fabsf(dn) + sqrtf(fmaf(dn, dn, tn * tn))));
-                    }
-                }
-                if (t != 0.0) {
-                    const double t2 = fma(t, t, 1.0);
-                    const double c0 = (double)rsqrtf((float)t2);
-                    const double cs = c0 * fma(-0.5 * t2, c0 * c0, 1.5), ics = t2 * cs;
-                    ta = t * sb * iscl[pa];
-                    tb = t * sa * iscl[pb];
-                    scl[pa] = cs * sa; scl[pb] = cs * sb;
-                    iscl[pa] *= ics; iscl[pb] *= ics;
-                    nrm2[pa] = fmax(aa - t * ab, 0.0);
-                    nrm2[pb] = bb + t * ab;
-                    rotated = 1;
-                }
-                rot[2 * tid] = ta; rot[2 * tid + 1] = tb;
-            }
-            __syncthreads();
-            // phase 3: apply
-            if (my_pair < n_pairs) {
-                const double ta = rot[2 * my_pair], tb = rot[2 * my_pair + 1];
-                if (ta != 0.0 || tb != 0.0) {
-                    double* ga = G + (size_t)ca * d;
+            for (int r = 0; r < m; ++r) {
+                if (active) {
+                    int ib = idx + r;
+                    if (ib >= m) ib -= m;
+                    const int cb = blk * 2 * m + m + ib;
                     double* gb = G + (size_t)cb * d;
+                    double y[RPL];
+                    double dsum[4] = {0.0, 0.0, 0.0, 0.0};      // four chains: dependent fp64 operations are slow
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) {
+                    for (int e = 0; e < RPL; ++e) {
                         if (e < per_lane) {
-                            ga[l16 + 16 * e] = fma(-ta, y[e], x[e]);
-                            gb[l16 + 16 * e] = fma(tb, x[e], y[e]);
+                            y[e] = gb[lg + SV_LP * e];
+                            dsum[e & 3] = fma(x[e], y[e], dsum[e & 3]);
                         }
                     }
+                    double dot = (dsum[0] + dsum[1]) + (dsum[2] + dsum[3]);
+#pragma unroll
+                    for (int o = SV_LP / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);   // within the group
+                    // every lane of the group holds the same sums and works out the same rotation
+                    const double sb = scl[cb], isb = iscl[cb];
+                    const float bb = nrm2[cb];
+                    // The tangent of the rotation angle needs no more than single precision: an error eps in t leaves
+                    // eps times the old inner product behind, which the next sweep removes; the rotation itself stays
+                    // exact because the same t goes into both columns and into the scales.
+                    const float ab = saf * (float)sb * (float)dot;
+                    float tf = 0.f;
+                    // |cos| > 1e-13 (well above the rounding noise of the inner product), as a product of ratios so
+                    // that columns of very different size neither overflow nor underflow the test
+                    if (aa > 0.f && bb > 0.f && (ab / aa) * (ab / bb) > 1e-26f) {
+                        const float df = bb - aa, t2ab = 2.f * ab;
+                        const float mf = fmaxf(fabsf(df), fabsf(t2ab));
+                        const float dn = df / mf, tn = t2ab / mf;
+                        tf = (dn >= 0.f ? tn : -tn) / (fabsf(dn) + sqrtf(fmaf(dn, dn, tn * tn)));
+                    }
+                    if (tf != 0.f) {                    // the same decision on all lanes of the group
+                        // the cosine: one Newton step in fp64 from an fp32 seed
+                        const double t = (double)tf;
+                        const double t2 = fma(t, t, 1.0);
+                        const double c0 = (double)rsqrtf(fmaf(tf, tf, 1.f));
+                        const double cs = c0 * fma(-0.5 * t2, c0 * c0, 1.5), ics = t2 * cs;
+                        const double ta = t * sb * isa, tb = t * sa * isb;
+#pragma unroll
+                        for (int e = 0; e < RPL; ++e) {
+                            if (e < per_lane) {
+                                const double xo = x[e];
+                                x[e] = fma(-ta, y[e], xo);
+                                gb[lg + SV_LP * e] = fma(tb, xo, y[e]);
+                            }
+                        }
+                        if (lg == 0) {
+                            scl[cb] = cs * sb; iscl[cb] = isb * ics; nrm2[cb] = bb + tf * ab;
+                            rotated = 1;
+                        }
+                        sa *= cs; isa *= ics; saf = (float)sa; aa = fmaxf(aa - tf * ab, 0.f);
+                    }
                 }
+                __syncthreads();                        // the second-half columns change hands
+            }
+            // the level ends: the resident columns go back
+            if (active) {
+                double* ga = G + (size_t)ca * d;
+#pragma unroll
+                for (int e = 0; e < RPL; ++e)
+                    if (e < per_lane) ga[lg + SV_LP * e] = x[e];
+                if (lg == 0) { scl[ca] = sa; iscl[ca] = isa; nrm2[ca] = aa; }
             }
             __syncthreads();
         }
@@ -568,7 +574,7 @@ extern "C" seka_status seka_learn_projections(const seka_learn_shape* shape, con
             cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm <= 0) return SEKA_ERR_CUDA;
         if (cudaFuncSetAttribute(learn_cov_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LC_DYN_BYTES) != cudaSuccess ||
             cudaFuncSetAttribute(learn_svd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)(sizeof(double) * (128 * 128 + 128) + sizeof(int) * 128 + 127 * 128)) != cudaSuccess)
+                                 (int)(sizeof(double) * (128 * 128 + 128) + sizeof(int) * 128)) != cudaSuccess)
             return SEKA_ERR_CUDA;
         configured = true;
     }
@@ -600,7 +606,7 @@ extern "C" seka_status seka_learn_projections(const seka_learn_shape* shape, con
     ++g_launches;
 
     // SVD of every Omega, rank rule
-    const size_t sv_smem = sizeof(double) * ((size_t)d * d + d) + sizeof(int) * d + (size_t)(d - 1) * d;
+    const size_t sv_smem = sizeof(double) * ((size_t)d * d + d) + sizeof(int) * d;
     learn_svd_kernel<<<2 * slots, SV_THREADS, sv_smem, st>>>(omega_pos, omega_neg, slots, d, shape->gamma, U_pos, U_neg,
                                                            S_pos, S_neg, k_pos, k_neg, reinterpret_cast<int*>(ws + pl.sweeps_off));
     ++g_launches;
