@@ -277,6 +277,7 @@ __global__ void learn_dist_reduce_kernel(const float* __restrict__ part_sum, con
 
 // ------------------------------------------------------------------------------------ SVD (one-sided Jacobi, fp64)
 constexpr int SV_LP = 8;                        // lanes that share a column pair: four pairs per warp
+constexpr int SV_PAD = 8;                       // doubles of padding per column (64 bytes)
 constexpr int SV_THREADS = 64 * SV_LP;          // 64 pairs per round at head_dim 128
 constexpr int SV_MAX_SWEEPS = 60;
 
@@ -288,8 +289,9 @@ learn_svd_kernel(const float* __restrict__ omega_pos, const float* __restrict__ 
                  float* __restrict__ U_pos, float* __restrict__ U_neg, float* __restrict__ S_pos, float* __restrict__ S_neg,
                  int* __restrict__ k_pos, int* __restrict__ k_neg, int* __restrict__ sweeps_out) {
     extern __shared__ double sv_sm[];
-    double* G = sv_sm;                      // [d][d], column j at G + j * d
-    double* sig = G + (size_t)d * d;        // [d]
+    const int ldg = d + SV_PAD;             // column stride: the pad staggers neighbouring columns over the banks
+    double* G = sv_sm;                      // [d][ldg], column j at G + j * ldg
+    double* sig = G + (size_t)d * ldg;      // [d]
     int* order = reinterpret_cast<int*>(sig + d);   // [d]: position of column j in the sorted output
     __shared__ int rotated;
     __shared__ double pr[64], scl[128], iscl[128], scale;
@@ -299,13 +301,13 @@ learn_svd_kernel(const float* __restrict__ omega_pos, const float* __restrict__ 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, n_warps = SV_THREADS / 32;
     for (int idx = tid; idx < d * d; idx += SV_THREADS) {
         const int i = idx / d, j = idx - i * d;     // Omega[i][j], coalesced read
-        G[(size_t)j * d + i] = (double)om[idx];
+        G[(size_t)j * ldg + i] = (double)om[idx];
     }
     __syncthreads();
     // scale the matrix to unit largest entry (squares of column norms stay far from under- and overflow)
     {
         double mx = 0.0;
-        for (int idx = tid; idx < d * d; idx += SV_THREADS) mx = fmax(mx, fabs(G[idx]));
+        for (int idx = tid; idx < d * d; idx += SV_THREADS) mx = fmax(mx, fabs(G[(size_t)(idx / d) * ldg + idx % d]));
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) mx = fmax(mx, __shfl_xor_sync(0xffffffffu, mx, o));
         if (lane == 0) pr[warp] = mx;
@@ -317,7 +319,7 @@ learn_svd_kernel(const float* __restrict__ omega_pos, const float* __restrict__ 
         }
         __syncthreads();
         const double inv = scale > 0.0 ? 1.0 / scale : 0.0;
-        for (int idx = tid; idx < d * d; idx += SV_THREADS) G[idx] *= inv;
+        for (int idx = tid; idx < d * d; idx += SV_THREADS) G[(size_t)(idx / d) * ldg + idx % d] *= inv;
         __syncthreads();
     }
     constexpr int RPL = 128 / SV_LP;                // rows per lane at d = 128 (d = 64 uses the first half)
@@ -355,8 +357,8 @@ learn_svd_kernel(const float* __restrict__ omega_pos, const float* __restrict__ 
             const double sj = scl[j];
             double ss = 0.0;
             for (int i = lane; i < d; i += 32) {
-                const double v = G[(size_t)j * d + i] * sj;
-                G[(size_t)j * d + i] = v;
+                const double v = G[(size_t)j * ldg + i] * sj;
+                G[(size_t)j * ldg + i] = v;
                 ss = fma(v, v, ss);
             }
 #pragma unroll
@@ -373,7 +375,7 @@ learn_svd_kernel(const float* __restrict__ omega_pos, const float* __restrict__ 
             double sa = 1.0, isa = 1.0;
             float aa = 0.f, saf = 1.f;
             if (active) {
-                const double* ga = G + (size_t)ca * d;
+                const double* ga = G + (size_t)ca * ldg;
 #pragma unroll
                 for (int e = 0; e < RPL; ++e)
                     if (e < per_lane) x[e] = ga[lg + SV_LP * e];
@@ -384,7 +386,7 @@ learn_svd_kernel(const float* __restrict__ omega_pos, const float* __restrict__ 
                     int ib = idx + r;
                     if (ib >= m) ib -= m;
                     const int cb = blk * 2 * m + m + ib;
-                    double* gb = G + (size_t)cb * d;
+                    double* gb = G + (size_t)cb * ldg;
                     double y[RPL];
                     double dsum[4] = {0.0, 0.0, 0.0, 0.0};      // four chains: dependent fp64 operations are slow
 #pragma unroll
@@ -439,7 +441,7 @@ learn_svd_kernel(const float* __restrict__ omega_pos, const float* __restrict__ 
             }
             // the level ends: the resident columns go back
             if (active) {
-                double* ga = G + (size_t)ca * d;
+                double* ga = G + (size_t)ca * ldg;
 #pragma unroll
                 for (int e = 0; e < RPL; ++e)
                     if (e < per_lane) ga[lg + SV_LP * e] = x[e];
@@ -453,13 +455,13 @@ learn_svd_kernel(const float* __restrict__ omega_pos, const float* __restrict__ 
     // fold the scales of the last sweep
     for (int j = warp; j < d; j += n_warps) {
         const double sj = scl[j];
-        for (int i = lane; i < d; i += 32) G[(size_t)j * d + i] *= sj;
+        for (int i = lane; i < d; i += 32) G[(size_t)j * ldg + i] *= sj;
     }
     __syncthreads();
     // singular values = column norms
     for (int j = warp; j < d; j += n_warps) {
         double ss = 0.0;
-        for (int i = lane; i < d; i += 32) ss = fma(G[(size_t)j * d + i], G[(size_t)j * d + i], ss);
+        for (int i = lane; i < d; i += 32) ss = fma(G[(size_t)j * ldg + i], G[(size_t)j * ldg + i], ss);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
         if (lane == 0) sig[j] = sqrt(ss);           // of the scaled matrix; the scale goes back on at the output
@@ -477,7 +479,7 @@ learn_svd_kernel(const float* __restrict__ omega_pos, const float* __restrict__ 
     for (int idx = tid; idx < d * d; idx += SV_THREADS) {
         const int i = idx / d, j = idx - i * d;     // component i of column j
         const double s = sig[j];
-        Uo[(size_t)i * d + order[j]] = s > 0.0 ? (float)(G[(size_t)j * d + i] / s) : 0.f;
+        Uo[(size_t)i * d + order[j]] = s > 0.0 ? (float)(G[(size_t)j * ldg + i] / s) : 0.f;
     }
     for (int j = tid; j < d; j += SV_THREADS) So[order[j]] = (float)(sig[j] * scale);
     __syncthreads();
@@ -574,7 +576,7 @@ extern "C" seka_status seka_learn_projections(const seka_learn_shape* shape, con
             cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm <= 0) return SEKA_ERR_CUDA;
         if (cudaFuncSetAttribute(learn_cov_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LC_DYN_BYTES) != cudaSuccess ||
             cudaFuncSetAttribute(learn_svd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)(sizeof(double) * (128 * 128 + 128) + sizeof(int) * 128)) != cudaSuccess)
+                                 (int)(sizeof(double) * (128 * (128 + SV_PAD) + 128) + sizeof(int) * 128)) != cudaSuccess)
             return SEKA_ERR_CUDA;
         configured = true;
     }
@@ -606,7 +608,7 @@ extern "C" seka_status seka_learn_projections(const seka_learn_shape* shape, con
     ++g_launches;
 
     // SVD of every Omega, rank rule
-    const size_t sv_smem = sizeof(double) * ((size_t)d * d + d) + sizeof(int) * d;
+    const size_t sv_smem = sizeof(double) * ((size_t)d * (d + SV_PAD) + d) + sizeof(int) * d;
     learn_svd_kernel<<<2 * slots, SV_THREADS, sv_smem, st>>>(omega_pos, omega_neg, slots, d, shape->gamma, U_pos, U_neg,
                                                            S_pos, S_neg, k_pos, k_neg, reinterpret_cast<int*>(ws + pl.sweeps_off));
     ++g_launches;
