@@ -12,7 +12,8 @@
 //   learn_reduce_kernel   sums the per-chunk partials in chunk order, scales by 1 / n.
 //   learn_dist_kernel     D = mean over the answer tokens of ||h+ - h-||_2, per slot (fixed summation order).
 //   learn_svd_kernel      one CTA per matrix: one-sided Jacobi (Hestenes) in fp64 on the columns of Omega held in
-//                         shared memory, round-robin pair ordering, one warp per column pair; on convergence the
+//                         shared memory; every pair of columns meets once per sweep (ordering by recursive halving,
+//                         four lanes per pair, one column of each pair resident in registers); on convergence the
 //                         column norms are the singular values and the normalised columns the left singular
 //                         vectors; sorted descending; the rank of Eq. 3 from the sorted values.
 #include <math.h>
@@ -276,8 +277,9 @@ __global__ void learn_dist_reduce_kernel(const float* __restrict__ part_sum, con
 }
 
 // ------------------------------------------------------------------------------------ SVD (one-sided Jacobi, fp64)
-constexpr int SV_LP = 8;                        // lanes that share a column pair: four pairs per warp
-constexpr int SV_PAD = 8;                       // doubles of padding per column (64 bytes)
+constexpr int SV_LP = 4;                        // lanes that share a column pair: eight pairs per warp
+constexpr int SV_PAD = 4;                       // doubles of padding per column (32 bytes: the eight 32-byte pieces a warp
+                                                // touches in neighbouring columns fall on different banks)
 constexpr int SV_THREADS = 64 * SV_LP;          // 64 pairs per round at head_dim 128
 constexpr int SV_MAX_SWEEPS = 60;
 
