@@ -206,8 +206,8 @@ __global__ void learn_reduce_kernel(const float* __restrict__ part, float* __res
 }
 
 // ------------------------------------------------------------------------------------ head-selection distance
-// Block b takes a range of tokens; warp w owns the slots w, w + 8, ... (so that the eight warps read neighbouring
-// rows) and keeps their running sums in shared memory: one writer per slot, fixed order.
+// Block b takes a range of tokens; every slot has one owner (a fixed group of lanes of one warp), which keeps the
+// slot's running sum in shared memory: one writer per slot, fixed order.
 constexpr int LD_THREADS = 256;
 __global__ void learn_dist_kernel(const __nv_bfloat16* __restrict__ hp, const __nv_bfloat16* __restrict__ hn,
                                   const uint8_t* __restrict__ answer, int n, int slots, int d, int tokens_per_block,
@@ -221,33 +221,47 @@ __global__ void learn_dist_kernel(const __nv_bfloat16* __restrict__ hp, const __
     for (int t = t0; t < t1; ++t) {
         if (answer != nullptr && answer[t] == 0) continue;
         ++count;
-        // four slots of the warp at a time: their loads and reductions are independent
-        for (int s0 = warp; s0 < slots; s0 += 4 * (LD_THREADS / 32)) {
+        // A row (one token of one slot) is d / 8 lanes of 16 bytes, so one warp load covers 2 (d = 128) or 4 (d = 64)
+        // neighbouring slots: 512 contiguous bytes.  Four such loads per tensor are in flight before the sums.
+        const int lpr = d / 8, rpw = 32 / lpr;              // lanes per row, rows per warp load
+        const int sub = lane / lpr;
+        const int n_q = (slots + rpw - 1) / rpw;
+        for (int q0 = warp; q0 < n_q; q0 += 4 * (LD_THREADS / 32)) {
             float ss[4];
+            uint4 a4[4], b4[4];
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-                const int s = s0 + u * (LD_THREADS / 32);
-                ss[u] = 0.f;
-                if (s < slots) {
-                    const size_t base = ((size_t)t * slots + s) * d;
-                    for (int i = 2 * lane; i < d; i += 64) {
-                        const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(hp + base + i));
-                        const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(hn + base + i));
-                        const float dx = a.x - b.x, dy = a.y - b.y;
-                        ss[u] = fmaf(dx, dx, fmaf(dy, dy, ss[u]));
-                    }
+                const int sl = (q0 + u * (LD_THREADS / 32)) * rpw + sub;
+                a4[u] = make_uint4(0u, 0u, 0u, 0u); b4[u] = a4[u];
+                if (q0 + u * (LD_THREADS / 32) < n_q && sl < slots) {
+                    const size_t off = ((size_t)t * slots + sl) * d + (size_t)(lane % lpr) * 8;
+                    a4[u] = *reinterpret_cast<const uint4*>(hp + off);
+                    b4[u] = *reinterpret_cast<const uint4*>(hn + off);
                 }
             }
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
+            for (int u = 0; u < 4; ++u) {
+                const uint32_t* aw = reinterpret_cast<const uint32_t*>(&a4[u]);
+                const uint32_t* bw = reinterpret_cast<const uint32_t*>(&b4[u]);
+                float acc2 = 0.f;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&aw[e]));
+                    const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&bw[e]));
+                    const float dx = a.x - b.x, dy = a.y - b.y;
+                    acc2 = fmaf(dx, dx, fmaf(dy, dy, acc2));
+                }
+                ss[u] = acc2;
+            }
+            for (int o = lpr / 2; o > 0; o >>= 1) {
 #pragma unroll
                 for (int u = 0; u < 4; ++u) ss[u] += __shfl_xor_sync(0xffffffffu, ss[u], o);
             }
-            if (lane == 0) {
+            if (lane % lpr == 0) {
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    const int s = s0 + u * (LD_THREADS / 32);
-                    if (s < slots) acc[s] += sqrtf(ss[u]);
+                    const int sl = (q0 + u * (LD_THREADS / 32)) * rpw + sub;
+                    if (q0 + u * (LD_THREADS / 32) < n_q && sl < slots) acc[sl] += sqrtf(ss[u]);
                 }
             }
         }
