@@ -308,16 +308,22 @@ struct DecodePlan {
     size_t ml_off, ml_bytes, o_off, o_bytes, total;
 };
 
-// Chunks of cached tokens: enough CTAs for several waves over the SMs, but at least 256 tokens each so that the
-// partials stay a few per cent of the cache traffic.
+// Chunks of cached tokens.  A CTA has a fixed cost (query fragments, the merge of its warps, its partial), so chunks
+// are long: about three waves of CTAs over the SMs, at least 1024 tokens each.  Where that would leave SMs without
+// work (few sequences), the chunks shrink until one wave is full, down to 256 tokens.
 DecodePlan decode_plan(const seka_shape* s) {
     DecodePlan d;
     const int G = s->n_q_heads / s->n_kv_heads;
     const long long pairs = (long long)s->batch * s->n_kv_heads;
     const int slots = DEC_SM_COUNT * (s->head_dim == 128 ? DecSmem<128>::CTAS_PER_SM : DecSmem<64>::CTAS_PER_SM);
-    const long long want = pairs > 0 ? (8LL * slots + pairs - 1) / pairs : 1;   // splits that would give 8 waves
-    long long chunk = want > 0 ? (s->max_seqlen + want - 1) / want : s->max_seqlen;
-    if (chunk < 256) chunk = 256;
+    const long long want = pairs > 0 ? (3LL * slots + pairs - 1) / pairs : 1;    // splits that would give 3 waves
+    const long long fill = pairs > 0 ? (slots + pairs - 1) / pairs : 1;          // splits that fill one wave
+    long long chunk = (s->max_seqlen + want - 1) / want;
+    if (chunk < 1024) {
+        chunk = (s->max_seqlen + fill - 1) / fill;
+        if (chunk > 1024) chunk = 1024;
+        if (chunk < 256) chunk = 256;
+    }
     chunk = (chunk + DEC_STAGE_KEYS - 1) / DEC_STAGE_KEYS * DEC_STAGE_KEYS;
     d.chunk = (int)chunk;
     d.n_splits = s->max_seqlen > 0 ? (s->max_seqlen + d.chunk - 1) / d.chunk : 1;
