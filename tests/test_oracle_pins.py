@@ -427,6 +427,34 @@ def test_learner_hand_case():
     np.testing.assert_allclose(oracle.learn_projections(h, hp, hn, 0.6, answer_tokens=[0, 1])["D"][0], 1.0, atol=1e-15)
 
 
+def test_learner_orientation_of_the_cross_covariance():
+    # Section 3.1: Omega+ = h^T h+ / n and U+ = its LEFT singular vectors.  One token, h = e1, h+ = 2 e2, h- = 3 e3:
+    # Omega+ = e1 (2 e2)^T has its only non-zero entry at (row 1, column 2), so the leading left vector is e1 (the
+    # neutral direction) and the leading right vector e2.  The transposed product h+^T h / n would put the entry at
+    # (2, 1) and return e2: this case tells the two apart (diagonal or symmetric Omega cannot).
+    h = np.array([1.0, 0.0, 0.0]).reshape(1, 1, 3)
+    hp = np.array([0.0, 2.0, 0.0]).reshape(1, 1, 3)
+    hn = np.array([0.0, 0.0, 3.0]).reshape(1, 1, 3)
+    r = oracle.learn_projections(h, hp, hn, gamma=0.5)
+    expect_pos = np.zeros((3, 3)); expect_pos[0, 1] = 2.0
+    expect_neg = np.zeros((3, 3)); expect_neg[0, 2] = 3.0
+    np.testing.assert_allclose(r["omega_pos"][0], expect_pos, atol=1e-15)
+    np.testing.assert_allclose(r["omega_neg"][0], expect_neg, atol=1e-15)
+    np.testing.assert_allclose(r["S_pos"][0], [2.0, 0.0, 0.0], atol=1e-15)
+    np.testing.assert_allclose(r["S_neg"][0], [3.0, 0.0, 0.0], atol=1e-15)
+    np.testing.assert_allclose(np.abs(r["U_pos"][0][:, 0]), [1.0, 0.0, 0.0], atol=1e-15)
+    np.testing.assert_allclose(np.abs(r["U_neg"][0][:, 0]), [1.0, 0.0, 0.0], atol=1e-15)
+    assert r["k_pos"][0] == 1 and r["k_neg"][0] == 1
+    # a second token makes the picture generic: h = (e1, e2), h+ = (2 e2, 5 e3): Omega+ = (e1 (2 e2)^T + e2 (5 e3)^T) / 2,
+    # left vectors in order e2 (value 2.5), e1 (value 1); the transposed product would give e3, e2
+    h2 = np.array([[1.0, 0, 0], [0, 1.0, 0]]).reshape(2, 1, 3)
+    hp2 = np.array([[0, 2.0, 0], [0, 0, 5.0]]).reshape(2, 1, 3)
+    r2 = oracle.learn_projections(h2, hp2, hp2, gamma=0.9)
+    np.testing.assert_allclose(r2["S_pos"][0], [2.5, 1.0, 0.0], atol=1e-15)
+    np.testing.assert_allclose(np.abs(r2["U_pos"][0][:, :2]), [[0, 1], [1, 0], [0, 0]], atol=1e-15)
+    assert r2["k_pos"][0] == 2          # 2.5 / 3.5 < 0.9
+
+
 def test_learner_recovers_a_planted_subspace_exactly():
     # neutral keys with h^T h / n = I exactly, positive keys h (I + a B B^T), negative keys h (I - b B B^T):
     # Omega+ = I + a B B^T and Omega- = I - b B B^T, whose spectra and subspaces are known in closed form
