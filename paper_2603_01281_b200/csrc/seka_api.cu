@@ -5,7 +5,7 @@
 
 namespace seka {
 
-unsigned long long g_launches = 0;
+std::atomic<unsigned long long> g_launches{0};
 
 seka_status validate_shape(const seka_shape* s) {
     if (s == nullptr) return SEKA_ERR_INVALID_ARG;
@@ -59,4 +59,4 @@ extern "C" const char* seka_status_string(seka_status status) {
     return "unknown status";
 }
 
-extern "C" uint64_t seka_launch_count(void) { return seka::g_launches; }
+extern "C" uint64_t seka_launch_count(void) { return seka::g_launches.load(); }

@@ -1,28 +1,32 @@
 // Fused SEKA / AdaSEKA steered causal GQA attention forward for sm_100a.
 //
-// One CTA (16 warps) owns two tiles of 128 queries that share a KV head ("A" and "B": two query heads of
-// one group at the same rows, or two consecutive row tiles of one head when the group size is odd) and
-// walks the key tiles 0 .. diagonal.  Warp roles:
-//   warp 0        TMA producer: Q tiles and the edit operator W once, then K and V tiles (128-byte swizzle)
-//                 through two shared-memory rings, throttled by "empty" mbarriers the tensor core signals;
-//   warp 1        MMA issuer: S_x = Q_x K'^T and O_x += P_x V on tcgen05 with all accumulators in tensor
-//                 memory (S_A, S_B, O_A, O_B = 512 columns); P_x is read from tensor memory.  For a staged
-//                 K tile that holds highlighted tokens of a steered head it first issues dK = K W into the
-//                 score columns of the tile that will use K first (they are idle just then);
-//   warps 12-15   key editors: read dK from tensor memory and add it, for highlighted rows only, to the
-//                 staged tile in place: k' = k + g * sum_m alpha_m U_m U_m^T k (Section 2 / Section 3.3, hook
-//                 of Algorithm 1/2) with W = g * sum_m alpha_m U_m U_m^T prepared per (sequence, KV head);
-//   warps 4-7 / 8-11  softmax of tile A / B, one query row per thread: causal mask on the diagonal
-//                 tile, online softmax in base 2 with a lazily updated running maximum, P written
-//                 back as bf16 over the consumed score columns, O rescaled in tensor memory only when
-//                 the maximum moved by more than 2^8; final normalisation and store.
-// While one tile's softmax runs, the tensor core works on the other tile.  Neither K' nor the score
-// matrix ever reaches global memory; K and V are read only.  Every wait is bounded: a wait that runs
+// The edited logit of Eq. 5 is q.k' = q.k + q.(g P k).  A small preparation launch leaves the edited keys k' of every
+// key tile that holds a highlighted token in a side buffer as a high and a low bf16 part (see SteerPlan); this kernel
+// stages such a tile from the high parts instead of from K and, where the gain is large enough for the rounding of k'
+// to matter, extends the score product S = Q K'^T on the tensor core, in the same tensor-memory accumulator, by the
+// contraction with the low parts, so that the logits are those of the fp32 k'.  The score matrix never reaches memory;
+// K and V are read only.
+//
+// One CTA (16 warps) owns two tiles of 128 queries that share a KV head ("A" and "B": two query heads of one group at
+// the same rows, or two consecutive row tiles of one head when the group size is odd) and walks the key tiles
+// 0 .. diagonal.  Warp roles:
+//   warp 0        TMA producer: Q tiles, then K (or edited-key) and V tiles (128-byte swizzle) through two
+//                 shared-memory rings, throttled by "free" mbarriers the tensor core signals, and the low parts of
+//                 edited tiles through a ring of their own;
+//   warp 1        MMA issuer: S_x = Q_x K^T (+ the low-part steps) and O_x += P_x V on tcgen05 with all accumulators
+//                 in tensor memory (S_A, S_B, O_A, O_B = 512 columns); P_x is read from tensor memory;
+//   warp 2        operand relay: tells the issuer when the operands have landed, so that it waits on one barrier per
+//                 hand-off;
+//   warps 4-7 / 8-11  softmax of tile A / B, one query row per thread: causal mask on the diagonal tile, online
+//                 softmax in base 2 with a lazily updated running maximum, P written back as bf16 over the consumed
+//                 score columns, O rescaled in tensor memory only when the maximum moved by more than 2^8; final
+//                 normalisation and store.
+// (Warps 3 and 12-15 only give their registers to the softmax warps.)
+// While one tile's softmax runs, the tensor core works on the other tile.  Every wait is bounded: a wait that runs
 // out raises the CTA's abort flag, every role leaves its loop, and the status word reports it.
-// The edit runs on tcgen05 like everything else: warp-level mma.sync is starved by a busy tcgen05 pipe
-// (it gets roughly one slot per UMMA), and its unrolled code evicts the other roles' loops from the
-// instruction cache.
 #include <math.h>
+
+#include <mutex>
 
 #include "seka_kernels.h"
 
@@ -35,18 +39,15 @@ namespace seka {
 struct AttnParams {
     void* O;
     float* lse;
-    const uint8_t* mask;
-    const float* gain;
-    const uint8_t* head_enable;
-    const int* cu_seqlens;
+    const uint8_t* bh_info;       // [B, Hkv]: bit 0 the keys of this (sequence, KV head) are edited, bit 1 with the low parts
     const uint8_t* tile_hot;      // [B, n_qt]: key tile holds a highlighted token
+    const int* first_hot;         // [B]: first such tile of the sequence
     int* status;
-    int B, L, Hq, Hkv, n_qt;
-    const ItemRecord* items;   // item table (built by the preparation kernel), heaviest first
-    const int* n_items;        // its length (device word)
-    long long n_items_max;
+    const ItemRecord* items;      // item table (packed batches), heaviest first
+    const int* n_items;           // its length (device word)
+    Sched sched;
+    SteerPlan plan;
     int steer;
-    int pair_heads;       // 1: the two tiles of an item are two query heads of one KV group; 0: two consecutive row tiles
     float scale_log2;
 };
 
@@ -55,36 +56,37 @@ constexpr int NTHREADS = 512;
 constexpr uint32_t BLK_BYTES = 128 * 128;   // one [128 x 64] bf16 block
 constexpr float LAZY_RESCALE_LOG2 = 8.0f;   // the running maximum is only raised when it moved by more than this
 // registers per thread after the roles split (the CTA owns the whole register file: 4 x 128 x (80+184+184+64) = 64 Ki)
-constexpr int REGS_CTRL = 80, REGS_SOFTMAX = 184, REGS_EDIT = 64;
+constexpr int REGS_CTRL = 80, REGS_SOFTMAX = 184, REGS_PROJ = 64;   // PROJ: the idle fourth warpgroup
 // which of the 16 element pairs of every 32-key chunk take the polynomial exp2 instead of the special-function unit
 constexpr uint32_t POLY_PAIR_MASK = SEKA_POLY_PAIR_MASK;
+constexpr uint32_t SMEM_LIMIT = 227 * 1024;
 
+// Shared memory of one CTA.  Tiles first (each a multiple of 1024 bytes), then barriers and per-warp item slots.
 template <int D>
-struct SmemLayout {
-    // K and V ring depth: head_dim 128 leaves room for two stages beside the 32 KB edit operator, head_dim 64 for three
-    static constexpr int NK = D == 128 ? 2 : 3;
-    static constexpr uint32_t TILE = (D / 64) * BLK_BYTES;
-    static constexpr uint32_t WBLK = D * 128;              // one [D x 64] block of W
-    static constexpr uint32_t Q = 0;                       // 2 tiles
-    static constexpr uint32_t K = Q + 2 * TILE;            // NK stages
-    static constexpr uint32_t V = K + NK * TILE;           // NK stages
-    static constexpr uint32_t W = V + NK * TILE;           // D x D bf16
-    static constexpr uint32_t BARS = W + (D / 64) * WBLK;  // mbarriers
-    static constexpr uint32_t NBARS = 3 + 2 * NK + 8 + 3;
-    static constexpr uint32_t MISC = BARS + NBARS * 8;     // tmem holder, abort flag
-    static constexpr uint32_t ITEMS = MISC + 16;           // one 32-byte item record per warp
-    static constexpr uint32_t TOTAL = ITEMS + 16 * 32;
-    static constexpr uint32_t DYN_BYTES = TOTAL + 1024;    // slack for the 1024-byte alignment
+struct Geo {
+    static constexpr int NK = D == 128 ? 2 : 3;                    // K and V ring depth
+    static constexpr uint32_t TILE = (D / 64) * BLK_BYTES;         // a [128 x D] tile
+    static constexpr int NXMAX = 3;                                // most stages of the key-side operand
+    static constexpr uint32_t NBARS = 14 + 2 * NK + NXMAX;
 };
 
-// One 128-row query tile of a CTA: query head, tile index within the sequence, number of key tiles it attends
-// to (the last of them is the diagonal tile); n == 0 means the tile lies beyond the sequence.
-struct TileWork { int hq, qt, n; };
+struct SmemPlan {
+    uint32_t k, v, x, xb, bars, misc, items, total;
+};
 
-// all lanes of a warp wait on the same barrier and then agree on the outcome
-__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status, int where) {
-    const bool ok = mbar_wait(bar, parity, abort_flag, status, where);
-    return __all_sync(0xffffffffu, ok);
+template <int D>
+__host__ __device__ inline SmemPlan smem_plan(const SteerPlan& sp) {
+    using G = Geo<D>;
+    SmemPlan s;
+    s.k = 2 * G::TILE;
+    s.v = s.k + G::NK * G::TILE;
+    s.x = s.v + G::NK * G::TILE;
+    s.xb = sp.mode ? G::TILE : 0u;                                  // one stage of low parts: [128 x D]
+    s.bars = s.x + (uint32_t)sp.nx * s.xb;
+    s.misc = s.bars + ((G::NBARS * 8 + 15) & ~15u);                 // 16-byte aligned: the item slots are filled by 16-byte async copies
+    s.items = s.misc + 32;
+    s.total = s.items + 16 * 32;
+    return s;
 }
 
 // true in exactly one lane of a fully active warp
@@ -140,93 +142,65 @@ template <> __device__ __forceinline__ void store_chunk32<float>(float* dst, con
                             __uint_as_float(v[4 * c + 2]) * inv, __uint_as_float(v[4 * c + 3]) * inv);
 }
 
-// Adds dK (fp32, tensor memory, one key row per lane) to this thread's row of a staged K tile for the 32-column
-// chunks [c0, c1); rows whose flag is clear are left alone.  The tensor-memory loads are warp-wide: every lane
-// takes part in them whatever its flag.  The four 16-byte units of a chunk are read before any is written back
-// (a store followed by a load of the same array would keep the updates strictly in sequence).
-__device__ __forceinline__ void drain_edit(uint32_t tE, uint8_t* sK, int row, bool hl, int c0, int c1) {
-#pragma unroll 1
-    for (int c = c0; c < c1; ++c) {
-        uint32_t dk[32];
-        tmem_ld32(tE + c * 32, dk);
-        tmem_wait_ld_on(dk);
-        if (hl) {
-            uint4* ptr[4];
-            uint4 kv[4];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {      // 8 elements = one 16-byte unit of the swizzled row
-                const int col = c * 32 + q * 8;
-                ptr[q] = reinterpret_cast<uint4*>(sK + (col >> 6) * (128 * 128) + sw128_offset(row, col & 63));
-                kv[q] = *ptr[q];
-            }
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                uint32_t* w = reinterpret_cast<uint32_t*>(&kv[q]);
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const float2 k2 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&w[e]));
-                    const float2 s2 = __fadd2_rn(k2, make_float2(__uint_as_float(dk[q * 8 + 2 * e]), __uint_as_float(dk[q * 8 + 2 * e + 1])));
-                    w[e] = pack_bf16(s2.x, s2.y);
-                }
-            }
-#pragma unroll
-            for (int q = 0; q < 4; ++q) *ptr[q] = kv[q];
-        }
-        __syncwarp();      // all lanes together again before the next warp-wide load
-    }
-}
-
 // One unit of work of a CTA: two 128-row query tiles that share a KV head of one sequence.
 struct Item {
     int b, hkv, seq0, Lb;
     int hqA, hqB, qtA, qtB;     // query head and row-tile index of tile A / B
     int nA, nB, n_kv;           // key tiles of A / B (0: the tile lies beyond the sequence) and of the item
-    bool steer;
+    bool steer;                 // the keys of this (sequence, KV head) are edited
+    bool hot_any;               // ... and one of the item's key tiles holds a highlighted token
+    bool need_lo;               // ... and the low parts of the edited keys are multiplied too
 };
 
 template <int D, typename OutT, bool TABLE>
 __global__ void __launch_bounds__(NTHREADS, 1)
 seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                     const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmW,
-                     const AttnParams p) {
-    using SL = SmemLayout<D>;
-    constexpr int NK = SL::NK;
+                     const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmX,
+                     const __grid_constant__ AttnParams p) {
+    using G = Geo<D>;
+    constexpr int NK = G::NK;
     constexpr int NBLK = D / 64;
     constexpr uint32_t TMEM_COLS = 512;
     constexpr uint32_t COL_S = 0, COL_O = 256;     // S_x at COL_S + 128 x, O_x at COL_O + D x
-    // head_dim 64 leaves 128 columns unused: dK of a highlighted key tile gets columns of its own there and is
-    // formed while the previous step's P V runs; head_dim 128 has to borrow the idle score columns of a tile
-    constexpr bool EDIT_OWN_COLS = (D == 64);
-    constexpr uint32_t COL_E = 384;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SL::BARS);
-    uint64_t* q_full = bars;                 // [2]   TMA bytes landed
+    const SmemPlan sl = smem_plan<D>(p.plan);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sl.bars);
+    uint64_t* q_full = bars;                 // [2]   Q tile landed
     uint64_t* k0_full = q_full + 2;          // [1]   first key tile of the item landed
     uint64_t* kv_full = k0_full + 1;         // [NK]  V(t) and K(t+1) landed (they are loaded as a pair)
     uint64_t* kv_free = kv_full + NK;        // [NK]  one event per step: the tensor core is done with K(j+1) and V(j)
-    uint64_t* s_full = kv_free + NK;         // [2]   scores of tile x are in tensor memory
-    uint64_t* p_full = s_full + 2;           // [2]   4 softmax-warp arrivals (O_x rescaled, keys 0-95 of P_x written) + 1 from the operand relay
+    uint64_t* x_full = kv_free + NK;         // [3]   low parts of an edited tile landed
+    uint64_t* s_full = x_full + G::NXMAX;    // [2]   scores of tile x are in tensor memory
+    uint64_t* p_full = s_full + 2;           // [2]   4 softmax-warp arrivals (O_x rescaled, keys 0-95 of P_x written) + 1 from the relay
     uint64_t* p_last = p_full + 2;           // [2]   4 softmax-warp arrivals: keys 96-127 of P_x written
     uint64_t* o_full = p_last + 2;           // [2]   last P V of tile x finished
-    uint64_t* w_full = o_full + 2;           // [1]   edit operator landed
-    uint64_t* e_full = w_full + 1;           // [1]   dK = K W of the current highlighted tile is in tensor memory
-    uint64_t* k_edited = e_full + 1;         // [1]   4 editor-warp + 4 softmax-warp arrivals: the staged tile now holds K'
-    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + SL::MISC);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + SL::MISC + 4);
+    uint64_t* o_drained = o_full + 2;        // [2]   4 softmax-warp arrivals: O_x of the item has been read
+    uint64_t* start_full = o_drained + 2;    // [1]   relay: Q tiles and first key tile of the item landed
+    uint64_t* drain = start_full + 1;        // [1]   every product issued has finished
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + sl.misc);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + sl.misc + 4);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    // an earlier launch (or CTA) gave up on this workspace: all threads agree on leaving
-    if (__syncthreads_or(*reinterpret_cast<volatile int*>(p.status) != 0)) return;
+    // an earlier launch (or CTA) gave up on this workspace: nothing is started (every role finds `ok` false)
+    const bool dead = __syncthreads_or(*reinterpret_cast<volatile int*>(p.status) != 0);
+    const int hook_skip = p.status[4];
+    const uint64_t limit_ns = p.status[5] > 0 ? (uint64_t)p.status[5] * 1000ull : kWaitLimitNs;
+
+    // all lanes of a warp wait on the same barrier and then agree on the outcome
+    auto warp_wait = [&](uint64_t* bar, uint32_t parity, int where) -> bool {
+        const bool ok = mbar_wait_limit(bar, parity, abort_flag, p.status, where, limit_ns);
+        return __all_sync(0xffffffffu, ok);
+    };
 
     // The CTA is persistent: it walks its share of the items (heaviest first; odd rounds run the CTAs in
     // reverse so that the shares come out even).  Every role goes through the same sequence of items by itself.
     // Fixed-length batches decode the item from its index; packed variable-length batches, where many index
     // slots are empty (row tiles beyond a short sequence), read a table from which those were dropped.
-    const int n_items = TABLE ? *p.n_items : (int)p.n_items_max;
+    const int n_items = TABLE ? *p.n_items : (int)p.sched.n_items_max;
     auto item_index = [&](int round) -> int {
-        const int G = (int)gridDim.x;
-        const long long idx = (long long)round * G + ((round & 1) ? (G - 1 - (int)blockIdx.x) : (int)blockIdx.x);
+        const int NG = (int)gridDim.x;
+        const long long idx = (long long)round * NG + ((round & 1) ? (NG - 1 - (int)blockIdx.x) : (int)blockIdx.x);
         return idx < n_items ? (int)idx : -1;
     };
     // (table) the record of the next item is copied into a per-warp slot of shared memory while the current item
@@ -234,7 +208,7 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     int round = 0, idx_next = TABLE ? item_index(0) : 0;
     auto prefetch = [&]() {
         if (TABLE && idx_next >= 0 && lane == 0) {
-            const uint32_t dst = smem_u32(smem + SL::ITEMS + warp * 32);
+            const uint32_t dst = smem_u32(smem + sl.items + warp * 32);
             const ItemRecord* rec = p.items + idx_next;
             asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(rec) : "memory");
             asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(dst + 16), "l"(reinterpret_cast<const char*>(rec) + 16) : "memory");
@@ -243,58 +217,49 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     };
     prefetch();
     auto next_item = [&](Item& it) -> bool {
+        ItemRecord rec;
         if (TABLE) {
             if (idx_next < 0) return false;
-            const uint8_t* slot = smem + SL::ITEMS + warp * 32;
+            const uint8_t* slot = smem + sl.items + warp * 32;
             if (lane == 0) asm volatile("cp.async.wait_group 0;" ::: "memory");
             __syncwarp();
             const int4 raw0 = *reinterpret_cast<const int4*>(slot), raw1 = *reinterpret_cast<const int4*>(slot + 16);
-            it.seq0 = raw0.x; it.Lb = raw0.y; it.b = raw0.z; it.hkv = raw0.w;
-            it.hqA = raw1.x & 0xffff; it.hqB = raw1.x >> 16;
-            it.qtA = raw1.y & 0xffff; it.qtB = raw1.y >> 16;
-            it.nA = raw1.z & 0xffff; it.nB = raw1.z >> 16;
-            it.steer = raw1.w != 0;
+            rec.seq0 = raw0.x; rec.Lb = raw0.y; rec.bh = raw0.z; rec.hq = raw0.w;
+            rec.qt = raw1.x; rec.n = raw1.y; rec.steer = raw1.z;
             __syncwarp();            // every lane has read the slot before it is refilled
             idx_next = item_index(++round);
             prefetch();
         } else {
             const int idx = item_index(round++);
             if (idx < 0) return false;
-            if (p.pair_heads) {
-                const int per_qt = p.B * (p.Hq >> 1);
-                const int qt = p.n_qt - 1 - (int)((unsigned)idx / (unsigned)per_qt);
-                const int rem = (int)((unsigned)idx % (unsigned)per_qt);
-                it.b = rem / (p.Hq >> 1);
-                const int hp = rem % (p.Hq >> 1);
-                it.hqA = 2 * hp; it.hqB = 2 * hp + 1;
-                it.qtA = it.qtB = qt;
-            } else {
-                const int per_qt = p.B * p.Hq;
-                const int qt2 = ((p.n_qt + 1) >> 1) - 1 - (int)((unsigned)idx / (unsigned)per_qt);
-                const int rem = (int)((unsigned)idx % (unsigned)per_qt);
-                it.b = rem / p.Hq;
-                it.hqA = it.hqB = rem % p.Hq;
-                it.qtA = 2 * qt2; it.qtB = 2 * qt2 + 1;
-            }
-            it.hkv = it.hqA / (p.Hq / p.Hkv);
-            it.seq0 = it.b * p.L;       // fixed length: every slot holds work (tile B of the last odd pair may not)
-            it.Lb = p.L;
-            it.nA = it.qtA * BM < it.Lb ? it.qtA + 1 : 0;
-            it.nB = it.qtB * BM < it.Lb ? it.qtB + 1 : 0;
-            it.steer = p.steer && p.gain[it.b] != 0.f && (p.head_enable == nullptr || p.head_enable[it.hkv] != 0);
+            decode_item(p.sched, idx, nullptr, rec);
+            const int b = rec.bh & 0xffff, hkv = rec.bh >> 16;
+            rec.steer = p.steer ? (int)__ldg(p.bh_info + b * p.sched.Hkv + hkv) : 0;      // one cache line for a whole batch
         }
+        it.seq0 = rec.seq0; it.Lb = rec.Lb; it.b = rec.bh & 0xffff; it.hkv = rec.bh >> 16;
+        it.hqA = rec.hq & 0xffff; it.hqB = rec.hq >> 16;
+        it.qtA = rec.qt & 0xffff; it.qtB = rec.qt >> 16;
+        it.nA = rec.n & 0xffff; it.nB = rec.n >> 16;
         it.n_kv = max(it.nA, it.nB);
+        it.steer = (rec.steer & 1) != 0 && p.plan.mode != 0;
+        it.hot_any = it.steer && p.first_hot[it.b] < it.n_kv;
+        it.need_lo = it.hot_any && (rec.steer & 2) != 0;
         return true;
     };
 
     if (tid == 0) {
         mbar_init(q_full + 0, 1); mbar_init(q_full + 1, 1); mbar_init(k0_full, 1);
         for (int i = 0; i < NK; ++i) { mbar_init(kv_full + i, 1); mbar_init(kv_free + i, 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(s_full + i, 1); mbar_init(p_full + i, 5); mbar_init(p_last + i, 4); mbar_init(o_full + i, 1); }
-        mbar_init(w_full, 1); mbar_init(e_full, 1); mbar_init(k_edited, 8);
-        *abort_flag = 0;
+        for (int i = 0; i < G::NXMAX; ++i) mbar_init(x_full + i, 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(s_full + i, 1); mbar_init(p_full + i, 5); mbar_init(p_last + i, 4); mbar_init(o_full + i, 1);
+            mbar_init(o_drained + i, 4);
+        }
+        mbar_init(start_full, 1); mbar_init(drain, 1);
+        *abort_flag = dead ? 1 : 0;
         mbar_fence_init();
         tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
+        if (p.plan.mode) tma_prefetch_desc(&tmX);
     }
     __syncwarp();
     if (warp == 0) { tmem_alloc(tmem_holder, TMEM_COLS); tmem_relinquish(); }
@@ -304,9 +269,14 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     const uint32_t tmem_base = *tmem_holder;
 
     // Running counts shared by all roles (each keeps its own copy; they advance identically):
-    //   ev   kv_free events so far (n_kv + 1 per item: after the first score products, then after every step)
-    //   pr   V/K pairs so far (n_kv per item); pair t of an item uses V stage (pr + t) % NK and K stage (pr + t + 1) % NK
-    //   cA/cB  steps of tile A / B so far (phases of s_full, p_full, p_last)
+    //   n_it   items so far (phases of start_full, q_full[0], k0_full)
+    //   n_o[x] items that had a tile x so far (phases of o_full, o_drained)
+    //   n_qb   items with a tile B so far (phase of q_full[1])
+    //   n_hot  edited key tiles whose low parts were loaded / used so far, over all items (stage and phase of x_full)
+    //   ev     kv_free events so far (n_kv + 1 per item: after the first score products, then after every step);
+    //          event j of an item covers the score products of its key tile j
+    //   pr     V/K pairs so far (n_kv per item); pair t of an item uses V stage (pr + t) % NK and K stage (pr + t + 1) % NK
+    //   cx[x]  steps of tile x so far (phases of s_full, p_full, p_last)
     Item it;
 
     if (warp < 4) {
@@ -316,43 +286,75 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         const bool leader = elect_one();
         if (warp == 0) {
             // ------------------------------------------------------------ TMA producer
-            uint32_t ev = 0, pr = 0, n_it = 0, n_qb = 0;
-            int prev_n = 0;
-            bool ok = true;
+            const int nx = p.plan.nx;
+            const bool staged = p.plan.mode != 0;       // key tiles with highlighted tokens come from the side buffer
+            uint32_t ev = 0, pr = 0, n_it = 0, n_qb = 0, n_hot = 0;
+            uint32_t ev_seen = 0;            // events [0, ev_seen) are known to have completed
+            uint32_t ev_hot[G::NXMAX] = {0, 0, 0};      // per stage of the key-side operand: event that releases it, + 1
+            // parity + 1 of the last load armed on each barrier (0: none), for the teardown after an abort
+            uint32_t armed_q[2] = {0, 0}, armed_k0 = 0, armed_kv[NK], armed_x[G::NXMAX] = {0, 0, 0};
+#pragma unroll
+            for (int i = 0; i < NK; ++i) armed_kv[i] = 0;
+            bool ok = !dead;
+            auto see_event = [&](uint32_t e, int where) {        // events complete in order
+                if (e < ev_seen) return;
+                ok = warp_wait(kv_free + e % NK, (e / NK) & 1, where);
+                ev_seen = e + 1;
+            };
+            // low parts of the edited key tile j of the item (event `e` covers its score products) into the next stage
+            auto load_x = [&](int j, uint32_t e) {
+                uint32_t st = 0, prev = 0;
+#pragma unroll
+                for (int i = 0; i < G::NXMAX; ++i)
+                    if ((int)(n_hot % (uint32_t)nx) == i) { st = i; prev = ev_hot[i]; ev_hot[i] = e + 1; }
+                if (prev) see_event(prev - 1, 14);       // the tile that used this stage before is through the tensor core
+                if (!ok) return;
+                if (leader) {
+                    mbar_expect_tx(x_full + st, sl.xb);
+#pragma unroll
+                    for (int c = 0; c < NBLK; ++c)
+                        tma_load_3d(smem + sl.x + st * sl.xb + c * BLK_BYTES, &tmX, x_full + st, D + c * 64, it.hkv, it.seq0 + j * BN);
+                }
+                __syncwarp();
+#pragma unroll
+                for (int i = 0; i < G::NXMAX; ++i)
+                    if ((int)st == i) armed_x[i] = ((n_hot / (uint32_t)nx) & 1) + 1;
+                ++n_hot;
+            };
             while (ok && next_item(it)) {
-                // Q, W and the first K of an item may land once the last score product of the previous item is
+                const uint8_t* hot_g = p.tile_hot + (size_t)it.b * p.sched.n_qt;
+                // Q and the first K of an item may land once the last score product of the previous item is
                 // done (event n_kv - 1 of that item), its V/K pairs once its last step is done (event n_kv)
                 if (n_it > 0) {
-                    const uint32_t e = ev - 2;
-                    ok = warp_wait(kv_free + e % NK, (e / NK) & 1, abort_flag, p.status, 12);
+                    see_event(ev - 2, 12);
                     if (!ok) break;
                 }
                 if (leader) {
-                    mbar_expect_tx(q_full + 0, SL::TILE);
+                    mbar_expect_tx(q_full + 0, G::TILE);
 #pragma unroll
                     for (int c = 0; c < NBLK; ++c)
-                        tma_load_3d(smem + SL::Q + c * BLK_BYTES, &tmQ, q_full + 0, c * 64, it.hqA, it.seq0 + it.qtA * BM);
+                        tma_load_3d(smem + c * BLK_BYTES, &tmQ, q_full + 0, c * 64, it.hqA, it.seq0 + it.qtA * BM);
                     if (it.nB > 0) {
-                        mbar_expect_tx(q_full + 1, SL::TILE);
+                        mbar_expect_tx(q_full + 1, G::TILE);
 #pragma unroll
                         for (int c = 0; c < NBLK; ++c)
-                            tma_load_3d(smem + SL::Q + SL::TILE + c * BLK_BYTES, &tmQ, q_full + 1, c * 64, it.hqB, it.seq0 + it.qtB * BM);
+                            tma_load_3d(smem + G::TILE + c * BLK_BYTES, &tmQ, q_full + 1, c * 64, it.hqB, it.seq0 + it.qtB * BM);
                     }
-                    mbar_expect_tx(k0_full, SL::TILE);
+                    mbar_expect_tx(k0_full, G::TILE);
+                    const CUtensorMap* km0 = (staged && it.hot_any && hot_g[0] != 0) ? &tmX : &tmK;
 #pragma unroll
                     for (int c = 0; c < NBLK; ++c)
-                        tma_load_3d(smem + SL::K + (pr % NK) * SL::TILE + c * BLK_BYTES, &tmK, k0_full, c * 64, it.hkv, it.seq0);
-                    if (it.steer) {
-                        mbar_expect_tx(w_full, NBLK * SL::WBLK);
-#pragma unroll
-                        for (int c = 0; c < NBLK; ++c)
-                            tma_load_3d(smem + SL::W + c * SL::WBLK, &tmW, w_full, c * 64, 0, (it.b * p.Hkv + it.hkv) * D);
-                    }
+                        tma_load_3d(smem + sl.k + (pr % NK) * G::TILE + c * BLK_BYTES, km0, k0_full, c * 64, it.hkv, it.seq0);
                 }
                 __syncwarp();
+                armed_q[0] = (n_it & 1) + 1; armed_k0 = (n_it & 1) + 1;
+                if (it.nB > 0) { armed_q[1] = (n_qb & 1) + 1; ++n_qb; }
+                if (it.need_lo && hot_g[0] != 0) {
+                    load_x(0, ev);
+                    if (!ok) break;
+                }
                 if (n_it > 0) {
-                    const uint32_t e = ev - 1;
-                    ok = warp_wait(kv_free + e % NK, (e / NK) & 1, abort_flag, p.status, 13);
+                    see_event(ev - 1, 13);
                     if (!ok) break;
                 }
                 // V(t) and K(t+1) travel as a pair: both of their stages are released by the same event, the end
@@ -360,79 +362,82 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 #pragma unroll 1
                 for (int t = 0; t < it.n_kv; ++t) {
                     if (t >= NK - 1) {
-                        const uint32_t e = ev + (uint32_t)(t - NK + 1);
-                        ok = warp_wait(kv_free + e % NK, (e / NK) & 1, abort_flag, p.status, 10);
+                        see_event(ev + (uint32_t)(t - NK + 1), 10);
                         if (!ok) break;
                     }
-                    if (leader) {
-                        const bool more = t + 1 < it.n_kv;
-                        uint64_t* bar = kv_full + (pr + t) % NK;
-                        mbar_expect_tx(bar, more ? 2 * SL::TILE : SL::TILE);
+                    const bool more = t + 1 < it.n_kv;
+                    const bool hot_n = more && it.hot_any && hot_g[t + 1] != 0;
+                    const uint32_t g = pr + (uint32_t)t;
+                    // (test hook: one pair of the first item of CTA 0 is left out altogether, so that its wait runs out)
+                    const bool skip = hook_skip > 0 && n_it == 0 && blockIdx.x == 0 && t + 1 == hook_skip;
+                    if (leader && !skip) {
+                        uint64_t* bar = kv_full + g % NK;
+                        mbar_expect_tx(bar, more ? 2 * G::TILE : G::TILE);
 #pragma unroll
                         for (int c = 0; c < NBLK; ++c)
-                            tma_load_3d(smem + SL::V + ((pr + t) % NK) * SL::TILE + c * BLK_BYTES, &tmV, bar, c * 64, it.hkv, it.seq0 + t * BN);
+                            tma_load_3d(smem + sl.v + (g % NK) * G::TILE + c * BLK_BYTES, &tmV, bar, c * 64, it.hkv, it.seq0 + t * BN);
                         if (more) {
+                            const CUtensorMap* km = (staged && hot_n) ? &tmX : &tmK;
 #pragma unroll
                             for (int c = 0; c < NBLK; ++c)
-                                tma_load_3d(smem + SL::K + ((pr + t + 1) % NK) * SL::TILE + c * BLK_BYTES, &tmK, bar, c * 64, it.hkv,
+                                tma_load_3d(smem + sl.k + ((g + 1) % NK) * G::TILE + c * BLK_BYTES, km, bar, c * 64, it.hkv,
                                             it.seq0 + (t + 1) * BN);
                         }
                     }
                     __syncwarp();
+                    if (!skip) {
+#pragma unroll
+                        for (int i = 0; i < NK; ++i)
+                            if ((int)(g % NK) == i) armed_kv[i] = ((g / NK) & 1) + 1;
+                    }
+                    if (hot_n && it.need_lo) {
+                        load_x(t + 1, ev + (uint32_t)(t + 1));
+                        if (!ok) break;
+                    }
                 }
-                ev += it.n_kv + 1; pr += it.n_kv; ++n_it; prev_n = it.n_kv;
-                if (it.nB > 0) ++n_qb;
+                ev += it.n_kv + 1; pr += it.n_kv; ++n_it;
             }
-            (void)prev_n; (void)n_qb;
+            if (*abort_flag) {
+                // loads that were armed may still be in flight: let them land before the shared memory is released
+                auto settle = [&](uint64_t* bar, uint32_t armed) {
+                    if (armed) mbar_wait_limit(bar, armed - 1, nullptr, nullptr, 0, limit_ns);
+                };
+                settle(q_full + 0, armed_q[0]); settle(q_full + 1, armed_q[1]); settle(k0_full, armed_k0);
+#pragma unroll
+                for (int i = 0; i < NK; ++i) settle(kv_full + i, armed_kv[i]);
+#pragma unroll
+                for (int i = 0; i < G::NXMAX; ++i) settle(x_full + i, armed_x[i]);
+            }
         } else if (warp == 1) {
             // ------------------------------------------------------------ MMA issuer
             constexpr uint32_t IDESC_S = umma_idesc_bf16(BN, false);
             constexpr uint32_t IDESC_PV = umma_idesc_bf16(D, true);
-            constexpr uint32_t IDESC_E = umma_idesc_bf16(D, false);
             constexpr uint32_t DESC_HI = umma_desc_hi_sw128(1024);
-            const uint32_t dQ = umma_desc_lo(smem_u32(smem + SL::Q), 16), dK = umma_desc_lo(smem_u32(smem + SL::K), 16);
-            const uint32_t dV = umma_desc_lo(smem_u32(smem + SL::V), BLK_BYTES);
-            const uint32_t dW = umma_desc_lo(smem_u32(smem + SL::W), 16);
-            uint32_t ev = 0, pr = 0, n_it = 0, n_qb = 0, n_w = 0, n_ob[2] = {0, 0};
+            const uint32_t dQ = umma_desc_lo(smem_u32(smem), 16), dK = umma_desc_lo(smem_u32(smem + sl.k), 16);
+            const uint32_t dX = umma_desc_lo(smem_u32(smem + sl.x), 16);
+            const uint32_t dV = umma_desc_lo(smem_u32(smem + sl.v), BLK_BYTES);
+            const uint32_t nx = p.plan.nx > 0 ? (uint32_t)p.plan.nx : 1u;
+            uint32_t ev = 0, pr = 0, n_it = 0, n_hot = 0;
             uint32_t cx[2] = {0, 0};      // steps of tile A / B so far
-            uint32_t n_hot = 0;           // highlighted tiles edited so far (phase of e_full / k_edited)
-            bool ok = true;
+            uint32_t n_o[2] = {0, 0};     // items that had a tile A / B so far
+            bool ok = !dead;
             auto commit = [&](uint64_t* bar) {
                 if (leader) umma_commit(bar);
                 __syncwarp();
             };
             while (ok && next_item(it)) {
-                const uint8_t* hot_g = p.tile_hot + (size_t)it.b * p.n_qt;
-                bool w_seen = false;
-                // Before the first score product of key tile j (by tile x): if the tile holds highlighted tokens,
-                // dK = K W goes into the score columns of tile x (idle between P_x V and the next S_x), the editors
-                // add it to the staged tile, and only then may the tile be multiplied.
-                auto edit_K = [&](int x, int j, bool is_hot) {
-                    if (!is_hot) return;
-                    if (!w_seen) { ok = warp_wait(w_full, n_w & 1, abort_flag, p.status, 31); w_seen = true; }
-                    if (!ok) return;
-                    const uint32_t kd = dK + ((pr + (uint32_t)j) % NK) * (SL::TILE >> 4);
-                    const uint32_t dst = tmem_base + (EDIT_OWN_COLS ? COL_E : COL_S + 128 * x);
-                    tc_fence_after();
-                    if (leader) {
-#pragma unroll
-                        for (int ks = 0; ks < D / 16; ++ks) {
-                            const uint32_t offk = ((uint32_t)(ks >> 2) * BLK_BYTES + (uint32_t)(ks & 3) * 32) >> 4;
-                            const uint32_t offw = ((uint32_t)(ks >> 2) * SL::WBLK + (uint32_t)(ks & 3) * 32) >> 4;
-                            umma_ss(dst, kd + offk, DESC_HI, dW + offw, DESC_HI, IDESC_E, ks > 0 ? 1u : 0u);
-                        }
-                        umma_commit(e_full);
-                    }
-                    __syncwarp();
-                };
-                // ... and the wait for the rows to be updated, kept apart: with columns of its own the product can be
-                // issued a good while before the edited tile is needed
-                auto edit_done = [&]() {
-                    ok = warp_wait(k_edited, n_hot & 1, abort_flag, p.status, 32);
+                const uint8_t* hot_g = p.tile_hot + (size_t)it.b * p.sched.n_qt;
+                const int nA = it.nA, nB = it.nB, n_kv = it.n_kv;
+                uint32_t x_stage = 0;      // stage that holds the low parts of the key tile being multiplied
+                // the low parts of the next edited key tile have landed (once per tile, before its first use)
+                auto see_x = [&]() {
+                    x_stage = n_hot % nx;
+                    ok = warp_wait(x_full + x_stage, (n_hot / nx) & 1, 32);
                     ++n_hot;
                 };
-                auto issue_S = [&](int x, int j) {
-                    const uint32_t kd = dK + ((pr + (uint32_t)j) % NK) * (SL::TILE >> 4), qd = dQ + (uint32_t)x * (SL::TILE >> 4);
+                // scores of tile x against key tile j; `hot`: the tile is an edited one whose low parts are multiplied too
+                auto issue_S = [&](int x, int j, bool hot) {
+                    const uint32_t kd = dK + ((pr + (uint32_t)j) % NK) * (G::TILE >> 4), qd = dQ + (uint32_t)x * (G::TILE >> 4);
                     const uint32_t dst = tmem_base + COL_S + 128 * x;
                     tc_fence_after();
                     if (leader) {
@@ -442,13 +447,21 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                             const uint32_t off = ((uint32_t)(ks >> 2) * BLK_BYTES + (uint32_t)(ks & 3) * 32) >> 4;
                             umma_ss(dst, qd + off, DESC_HI, kd + off, DESC_HI, IDESC_S, ks > 0 ? 1u : 0u);
                         }
+                        if (hot) {        // ... + Q (k'_lo)^T
+                            const uint32_t xd = dX + x_stage * (sl.xb >> 4);
+#pragma unroll
+                            for (int ks = 0; ks < D / 16; ++ks) {
+                                const uint32_t off = ((uint32_t)(ks >> 2) * BLK_BYTES + (uint32_t)(ks & 3) * 32) >> 4;
+                                umma_ss(dst, qd + off, DESC_HI, xd + off, DESC_HI, IDESC_S, 1u);
+                            }
+                        }
                         umma_commit(s_full + x);
                     }
                     __syncwarp();
                 };
                 // P V of tile x and key tile j, key blocks [ks0, ks1) of 16 keys (2048 bytes of the V tile, 8 columns of P)
                 auto issue_PV = [&](int x, int j, int ks0, int ks1, bool last) {
-                    const uint32_t vd = dV + ((pr + (uint32_t)j) % NK) * (SL::TILE >> 4);
+                    const uint32_t vd = dV + ((pr + (uint32_t)j) % NK) * (G::TILE >> 4);
                     const uint32_t dst = tmem_base + COL_O + D * x, src = tmem_base + COL_S + 128 * x;
                     tc_fence_after();
                     if (leader) {
@@ -461,86 +474,84 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     }
                     __syncwarp();
                 };
-                const int nA = it.nA, nB = it.nB, n_kv = it.n_kv;
-                // highlight flags of key tiles 0 and 1 (later ones are fetched one step ahead of their use)
-                bool hot_cur = it.steer && hot_g[0] != 0;
-                bool hot_nxt = it.steer && n_kv > 1 && hot_g[1] != 0;
+                // The O_x of the last item that had a tile x has been read.  Its phases count those items only, and each is
+                // seen, in order, by the next item that has the tile: a warp that could arrive for items in which it has
+                // nothing to do would run ahead, and a parity wait cannot tell a phase from the one two later.
+                auto see_drained = [&]() {
+                    if (n_o[0] > 0) ok = warp_wait(o_drained + 0, (n_o[0] - 1) & 1, 46);
+                    if (ok && nB > 0 && n_o[1] > 0) ok = warp_wait(o_drained + 1, (n_o[1] - 1) & 1, 47);
+                };
+                // do key tiles 0 and 1 take the low-part steps? (later ones are looked up one step ahead of their use)
+                const bool hot_cur = it.need_lo && hot_g[0] != 0;
+                bool hot_nxt = it.need_lo && n_kv > 1 && hot_g[1] != 0;
                 // One thread issues for both tiles, in a fixed order (A then B in every step): the in-order tensor
                 // pipe then keeps the two tiles half a period apart (softmax of one tile under the MMAs of the other).
-                ok = warp_wait(q_full + 0, n_it & 1, abort_flag, p.status, 20);
-                if (ok && nB > 0) ok = warp_wait(q_full + 1, n_qb & 1, abort_flag, p.status, 21);
-                if (ok) ok = warp_wait(k0_full, n_it & 1, abort_flag, p.status, 22);
-                if (ok && hot_cur) { edit_K(0, 0, true); if (ok) edit_done(); }
-                if (ok) {
-                    issue_S(0, 0);
-                    if (nB > 0) issue_S(1, 0);
-                    // The edit operator of this item is seen here at the latest, before the event that lets the
-                    // producer load the next item's: a barrier that ran two phases ahead of its waiter would
-                    // never look complete to it.
-                    if (it.steer && !w_seen) { ok = warp_wait(w_full, n_w & 1, abort_flag, p.status, 35); w_seen = true; }
-                    commit(kv_free + ev % NK);
-                    ++ev;
-                }
+                ok = warp_wait(start_full, n_it & 1, 20);
+                if (!ok) break;
+                if (hot_cur) { see_x(); if (!ok) break; }
+                issue_S(0, 0, hot_cur);
+                if (nB > 0) issue_S(1, 0, hot_cur);
+                commit(kv_free + ev % NK);
+                ++ev;
+                see_drained();          // before the item's first P V writes O_x again
+                if (!ok) break;
 #pragma unroll 1
                 for (int j = 0; j < n_kv && ok; ++j) {
                     const int j1 = j + 1;
-                    const bool hot_j1 = hot_nxt;
-                    hot_nxt = it.steer && j + 2 < n_kv && hot_g[j + 2] != 0;
+                    const bool hot_j1 = hot_nxt && j1 < n_kv;
+                    hot_nxt = it.need_lo && j + 2 < n_kv && hot_g[j + 2] != 0;
+                    bool x_seen = false;
                     // V of this step and K of the next have landed once p_full completes: the relay warp vouches
                     // for them there, so this warp has no waits of its own for operands (every wait here is a
                     // bubble in the tensor pipe: its queue is only a couple of MMAs deep)
                     if (j < nA) {
-                        ok = warp_wait(p_full + 0, (cx[0] + j) & 1, abort_flag, p.status, 24);
-                        if (!ok) break;
-                        if (EDIT_OWN_COLS && hot_j1 && j1 < nA) edit_K(0, j1, true);      // K(j1) has landed (the relay vouches), P_A V hides the drain
+                        ok = warp_wait(p_full + 0, (cx[0] + j) & 1, 24);
                         if (!ok) break;
                         issue_PV(0, j, 0, 6, false);
-                        ok = warp_wait(p_last + 0, (cx[0] + j) & 1, abort_flag, p.status, 28);
+                        ok = warp_wait(p_last + 0, (cx[0] + j) & 1, 28);
                         if (!ok) break;
                         issue_PV(0, j, 6, 8, j == nA - 1);
                         if (j1 < nA) {
-                            if (hot_j1) {
-                                if (!EDIT_OWN_COLS) edit_K(0, j1, true);
-                                if (ok) edit_done();
-                            }
-                            if (!ok) break;
-                            issue_S(0, j1);
+                            if (hot_j1) { see_x(); x_seen = true; if (!ok) break; }
+                            issue_S(0, j1, hot_j1);
                         }
                     }
                     if (j < nB) {
-                        ok = warp_wait(p_full + 1, (cx[1] + j) & 1, abort_flag, p.status, 26);
+                        ok = warp_wait(p_full + 1, (cx[1] + j) & 1, 26);
                         if (!ok) break;
                         issue_PV(1, j, 0, 6, false);
-                        ok = warp_wait(p_last + 1, (cx[1] + j) & 1, abort_flag, p.status, 29);
+                        ok = warp_wait(p_last + 1, (cx[1] + j) & 1, 29);
                         if (!ok) break;
                         issue_PV(1, j, 6, 8, j == nB - 1);
                     }
                     if (j1 < nB) {
-                        if (j1 >= nA && hot_j1) {      // tile A does not use this key tile: B is its first user
-                            edit_K(1, j1, true);
-                            if (ok) edit_done();
-                        }
-                        if (!ok) break;
-                        issue_S(1, j1);
+                        if (hot_j1 && !x_seen) { see_x(); if (!ok) break; }      // tile A does not use this key tile
+                        issue_S(1, j1, hot_j1);
                     }
                     commit(kv_free + ev % NK);      // K(j+1) and V(j) may be overwritten
                     ++ev;
                 }
                 pr += n_kv; cx[0] += nA; cx[1] += nB; ++n_it;
-                if (nB > 0) ++n_qb;
-                if (it.steer) ++n_w;
+                ++n_o[0];
+                if (nB > 0) ++n_o[1];
             }
-            (void)n_ob;
         } else if (warp == 2) {
-            // ------------------------------------------------------------ operand relay: "V(j) and K(j+1) have landed" as a
-            // fifth arrival on p_full of step j, so that the MMA issuer waits on one barrier per hand-off
-            uint32_t pr = 0, cx[2] = {0, 0};
-            bool ok = true;
+            // ------------------------------------------------------------ operand relay: "the operands have landed", once per
+            // item for Q and the first K, and per step "V(j) and K(j+1) landed" as a fifth arrival on the
+            // P hand-off barrier, so that the MMA issuer waits on one barrier per hand-off
+            uint32_t pr = 0, n_it = 0, n_qb = 0, cx[2] = {0, 0};
+            bool ok = !dead;
             while (ok && next_item(it)) {
+                ok = warp_wait(q_full + 0, n_it & 1, 21);
+                if (ok && it.nB > 0) { ok = warp_wait(q_full + 1, n_qb & 1, 22); ++n_qb; }
+                if (ok) ok = warp_wait(k0_full, n_it & 1, 23);
+                if (!ok) break;
+                if (lane == 0) mbar_arrive(start_full);
+                __syncwarp();
 #pragma unroll 1
                 for (int j = 0; j < it.n_kv; ++j) {
                     const uint32_t g = pr + j;
-                    ok = warp_wait(kv_full + g % NK, (g / NK) & 1, abort_flag, p.status, 23);
+                    ok = warp_wait(kv_full + g % NK, (g / NK) & 1, 25);
                     if (!ok) break;
                     if (lane == 0) {
                         if (j < it.nA) mbar_arrive(p_full + 0);
@@ -548,43 +559,16 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     }
                     __syncwarp();
                     // stay within the phase: the next arrival may only come after this phase has completed
-                    if (j < it.nA) ok = warp_wait(p_full + 0, (cx[0] + j) & 1, abort_flag, p.status, 33);
-                    if (ok && j < it.nB) ok = warp_wait(p_full + 1, (cx[1] + j) & 1, abort_flag, p.status, 34);
+                    if (j < it.nA) ok = warp_wait(p_full + 0, (cx[0] + j) & 1, 33);
+                    if (ok && j < it.nB) ok = warp_wait(p_full + 1, (cx[1] + j) & 1, 34);
                     if (!ok) break;
                 }
-                pr += it.n_kv; cx[0] += it.nA; cx[1] += it.nB;
+                pr += it.n_kv; cx[0] += it.nA; cx[1] += it.nB; ++n_it;
             }
         }
     } else if (warp >= 12) {
-        // ------------------------------------------------------------ key editors: one key row of the staged tile per thread
-        reg_dec<REGS_EDIT>();
-        const int row = (warp - 12) * 32 + lane;
-        const uint32_t t_lane = tmem_base + ((uint32_t)((warp - 12) * 32) << 16);
-        uint32_t pr = 0, n_hot = 0;
-        bool ok = true;
-        while (ok && next_item(it)) {
-            if (it.steer) {
-                const uint8_t* hot_g = p.tile_hot + (size_t)it.b * p.n_qt;
-#pragma unroll 1
-                for (int j = 0; j < it.n_kv; ++j) {
-                    if (hot_g[j] == 0) continue;
-                    const int kpos = j * BN + row;
-                    const bool hl = kpos < it.Lb && p.mask[it.seq0 + kpos] != 0;
-                    ok = warp_wait(e_full, n_hot & 1, abort_flag, p.status, 30);
-                    if (!ok) break;
-                    ++n_hot;
-                    tc_fence_after();
-                    const uint32_t tE = t_lane + (EDIT_OWN_COLS ? COL_E : COL_S + 128 * (j < it.nA ? 0 : 1));
-                    uint8_t* sK = smem + SL::K + ((pr + (uint32_t)j) % NK) * SL::TILE;
-                    drain_edit(tE, sK, row, hl, 0, D / 64);      // the other half of the columns is taken by the idle softmax warps
-                    fence_proxy_async();       // the rewritten rows are read next by the tensor core
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(k_edited);
-                }
-            }
-            pr += it.n_kv;
-        }
+        // (these warps only hand their registers to the softmax warps)
+        reg_dec<REGS_PROJ>();
     } else {
         // ------------------------------------------------------------ softmax of tile x, one query row per thread
         reg_inc<REGS_SOFTMAX>();
@@ -594,51 +578,14 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         const uint32_t tS = t_lane + COL_S + 128 * x, tO = t_lane + COL_O + D * x;
         const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
         uint32_t cX = 0, n_o = 0;       // steps and items of this tile so far
-        uint32_t pr = 0, n_hot = 0;     // V/K pairs and highlighted key tiles so far (all items)
-        bool ok = true;
+        bool ok = !dead;
         while (ok && next_item(it)) {
             const int nX = x ? it.nB : it.nA;
             const int hqX = x ? it.hqB : it.hqA, qtX = x ? it.qtB : it.qtA;
-            const uint8_t* hot_g = p.tile_hot + (size_t)it.b * p.n_qt;
-            // Every softmax warp waits for dK of EVERY highlighted key tile, in order, whether or not it helps to drain
-            // it: a warp that skipped a phase of e_full could find its next phase "complete" while the skipped one is
-            // still running (a parity wait only tells the current phase from the one before).  The waits cost nothing:
-            // the scores a warp needs next are issued after the edit anyway.
-            auto see_edit = [&](int j0, int j1) {
-                for (int j = j0; j < j1 && ok; ++j) {
-                    if (hot_g[j] == 0) continue;
-                    ok = warp_wait(e_full, n_hot & 1, abort_flag, p.status, 38);
-                    ++n_hot;
-                }
-            };
-            if (nX == 0) {      // tile B lies beyond the sequence: only the counts move
-                if (it.steer) see_edit(0, it.n_kv);
-                pr += it.n_kv;
-                if (!ok) break;
-                continue;
-            }
             float m_run = -INFINITY, l_run = 0.f;
 #pragma unroll 1
             for (int j = 0; j < nX; ++j) {
-                // Key tile j holds highlighted tokens and this tile is the first to use it: while waiting for its
-                // scores anyway, these warps add the upper half of the columns of dK to the staged K tile (the
-                // key editors take the lower half).  Every softmax warp counts the highlighted tiles.
-                if (it.steer && hot_g[j] != 0) {
-                    ok = warp_wait(e_full, n_hot & 1, abort_flag, p.status, 36 + x);
-                    if (!ok) break;
-                    if ((j < it.nA ? 0 : 1) == x) {
-                        const int kpos = j * BN + row;
-                        const bool hl = kpos < it.Lb && p.mask[it.seq0 + kpos] != 0;
-                        tc_fence_after();
-                        drain_edit(EDIT_OWN_COLS ? t_lane + COL_E : tS, smem + SL::K + ((pr + (uint32_t)j) % NK) * SL::TILE, row, hl, D / 64, D / 32);
-                        fence_proxy_async();
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(k_edited);
-                    }
-                    ++n_hot;
-                }
-                ok = warp_wait(s_full + x, (cX + j) & 1, abort_flag, p.status, 40 + x);
+                ok = warp_wait(s_full + x, (cX + j) & 1, 40 + x);
                 if (!ok) break;
                 tc_fence_after();
                 // the whole score row of this thread: 128 fp32 values in registers
@@ -709,16 +656,17 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                 const float2 s2 = __fadd2_rn(sum[0], sum[1]);
                 l_run = l_run * factor + (s2.x + s2.y);
             }
-            cX += nX; pr += it.n_kv;
-            if (ok) ok = warp_wait(o_full + x, n_o & 1, abort_flag, p.status, 44 + x);
-            ++n_o;
-            if (ok) {
-                // final normalisation and store; the next item's first P_x (hence its first P_x V into these
-                // columns) comes from these same threads, after they are done reading here
+            if (!ok) break;
+            cX += nX;
+            if (nX > 0) {
+                ok = warp_wait(o_full + x, n_o & 1, 44 + x);
+                ++n_o;
+                if (!ok) break;
+                // final normalisation and store
                 tc_fence_after();
                 const int qpos = qtX * BM + row;
                 const bool valid = qpos < it.Lb;
-                const size_t orow = (size_t)(it.seq0 + (valid ? qpos : 0)) * p.Hq + hqX;
+                const size_t orow = (size_t)(it.seq0 + (valid ? qpos : 0)) * p.sched.Hq + hqX;
                 const float inv = 1.f / l_run;
                 uint32_t o[32];
 #pragma unroll 1
@@ -729,23 +677,24 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                 }
                 if (valid && p.lse != nullptr) p.lse[orow] = (m_run + log2f(l_run)) * 0.6931471805599453f;
                 tc_fence_before();
+                // O_x may be written again (the next item's first P V)
+                __syncwarp();
+                if (lane == 0) mbar_arrive(o_drained + x);
             }
-            // highlighted tiles that only the other tile uses are seen too (after the output is on its way)
-            if (it.steer && ok) see_edit(nX, it.n_kv);
         }
     }
 
+    // ---------------------------------------------------------------- teardown (also after an abort)
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) {
-        if (*abort_flag && lane == 0) {
-            // let tile loads that may still be in flight land before the shared memory is released
-            int dummy = 0;
-            for (int i = 0; i < NK; ++i) { mbar_wait(kv_full + i, 0, &dummy, nullptr, 0); }
-        }
+    if (warp == 1) {
+        // every product issued has finished before tensor and shared memory are released
+        if (elect_one()) umma_commit(drain);
         __syncwarp();
-        tmem_dealloc(tmem_base, TMEM_COLS);
+        mbar_wait_limit(drain, 0, nullptr, p.status, 90, limit_ns);
     }
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem_base, TMEM_COLS);
 }
 
 // ---------------------------------------------------------------- host side
@@ -755,6 +704,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 static EncodeTiledFn encode_tiled_fn() {
     static EncodeTiledFn fn = nullptr;
+    static std::mutex mu;
+    std::lock_guard<std::mutex> lock(mu);
     if (fn == nullptr) {
         void* sym = nullptr;
         cudaDriverEntryPointQueryResult qres;
@@ -778,34 +729,47 @@ bool make_tile_map(CUtensorMap* m, const void* base, int d, int H, long long T, 
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Per-device facts, looked up once per device (a process may drive several GPUs from several threads).
+bool device_info(int* n_sm) {
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static int sm_of[kMaxDevices] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return false;
+    std::lock_guard<std::mutex> lock(mu);
+    if (sm_of[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return false;
+        sm_of[dev] = n;
+    }
+    *n_sm = sm_of[dev];
+    return true;
+}
+
+struct TileMaps { CUtensorMap q, k, v, x; };
+
 template <int D, typename OutT, bool TABLE>
-static seka_status launch_attn_t(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                                 const CUtensorMap& tw, const AttnParams& p, cudaStream_t st) {
-    using SL = SmemLayout<D>;
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(seka_attn_fwd_kernel<D, OutT, TABLE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)SL::DYN_BYTES) != cudaSuccess) return SEKA_ERR_CUDA;
-        configured = true;
-    }
-    static int n_sm = 0;
-    if (n_sm == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm <= 0) { n_sm = 0; return SEKA_ERR_CUDA; }
-    }
+static seka_status launch_attn_t(const TileMaps& tm, const AttnParams& p, cudaStream_t st) {
+    const SmemPlan sl = smem_plan<D>(p.plan);
+    const uint32_t dyn = sl.total + 1024;      // slack for the 1024-byte alignment
+    if (dyn > SMEM_LIMIT) return SEKA_ERR_UNSUPPORTED;
+    auto kern = seka_attn_fwd_kernel<D, OutT, TABLE>;
+    // the attribute belongs to the function on the current device: set on every call (a cheap driver call), so that a
+    // process that drives several devices, or calls from several threads, needs no bookkeeping here
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT) != cudaSuccess) return SEKA_ERR_CUDA;
+    int n_sm = 0;
+    if (!device_info(&n_sm)) return SEKA_ERR_CUDA;
     // persistent CTAs, one per SM (the kernel needs the whole SM: all of tensor memory and most of shared memory)
-    const unsigned grid = (unsigned)(p.n_items_max < (long long)n_sm ? p.n_items_max : (long long)n_sm);
-    seka_attn_fwd_kernel<D, OutT, TABLE><<<grid, NTHREADS, SL::DYN_BYTES, st>>>(tq, tk, tv, tw, p);
-    ++g_launches;
+    const unsigned grid = (unsigned)(p.sched.n_items_max < (long long)n_sm ? p.sched.n_items_max : (long long)n_sm);
+    if (grid == 0) return SEKA_OK;
+    kern<<<grid, NTHREADS, dyn, st>>>(tm.q, tm.k, tm.v, tm.x, p);
+    g_launches.fetch_add(1);
     return cudaGetLastError() == cudaSuccess ? SEKA_OK : SEKA_ERR_CUDA;
 }
 
 template <int D, typename OutT>
-static seka_status launch_attn(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv,
-                               const CUtensorMap& tw, const AttnParams& p, cudaStream_t st) {
-    return p.cu_seqlens != nullptr ? launch_attn_t<D, OutT, true>(tq, tk, tv, tw, p, st)
-                                   : launch_attn_t<D, OutT, false>(tq, tk, tv, tw, p, st);
+static seka_status launch_attn(const TileMaps& tm, const AttnParams& p, bool table, cudaStream_t st) {
+    return table ? launch_attn_t<D, OutT, true>(tm, p, st) : launch_attn_t<D, OutT, false>(tm, p, st);
 }
 
 // The fused forward behind both entry points: coefficients either given (`alpha`, may be null) or, with `sigma`
@@ -824,11 +788,12 @@ static seka_status attention_fwd_impl(const seka_shape* shape, const void* Q, co
     const bool steer = mask != nullptr && U != nullptr;
     if (steer && !gain) return SEKA_ERR_INVALID_ARG;
     const WorkspaceLayout w = workspace_layout(shape);
-    if (w.n_tiles > 32767 || shape->n_q_heads > 32767 || w.n_items_max > 0x7fffffffLL) return SEKA_ERR_UNSUPPORTED;   // item records pack 15-bit fields
+    const int D = shape->head_dim, Hq = shape->n_q_heads, Hkv = shape->n_kv_heads;
+    const Sched sched = make_sched(shape);
+    if (w.n_tiles > 32767 || Hq > 32767 || shape->batch > 65535 || sched.n_items_max > 0x7fffffffLL) return SEKA_ERR_UNSUPPORTED;   // item records pack 15/16-bit fields
     if (!workspace || workspace_bytes < w.total || ((uintptr_t)workspace & 255)) return SEKA_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     char* ws = static_cast<char*>(workspace);
-    const int D = shape->head_dim, Hq = shape->n_q_heads, Hkv = shape->n_kv_heads;
 
     const void *q16 = Q, *k16 = K, *v16 = V;
     if (shape->dtype == SEKA_F32) {
@@ -841,34 +806,43 @@ static seka_status attention_fwd_impl(const seka_shape* shape, const void* Q, co
         launch_convert_bf16(static_cast<const float*>(V), cv, nk, st);
         q16 = cq; k16 = ck; v16 = cv;
     }
-    void* W = ws + w.w_off;
-    uint8_t* tile_hot = reinterpret_cast<uint8_t*>(ws + w.hot_off);
-    if (steer) launch_prep_steering(shape, U, alpha, gain, head_enable, mask, W, tile_hot, w.n_tiles, st, Q, sigma, k_route, alpha_out);
-
-    CUtensorMap tq, tk, tv, tw;
-    if (!make_tile_map(&tq, q16, D, Hq, T) || !make_tile_map(&tk, k16, D, Hkv, T) || !make_tile_map(&tv, v16, D, Hkv, T) ||
-        !make_tile_map(&tw, W, D, 1, (long long)shape->batch * Hkv * D, D))
-        return SEKA_ERR_CUDA;
-
     AttnParams p;
-    p.O = O; p.lse = lse; p.mask = mask; p.gain = gain; p.head_enable = head_enable;
-    p.cu_seqlens = shape->cu_seqlens; p.tile_hot = tile_hot; p.status = reinterpret_cast<int*>(ws);
-    p.B = shape->batch; p.L = shape->max_seqlen; p.Hq = Hq; p.Hkv = Hkv;
-    p.n_qt = w.n_tiles; p.steer = steer ? 1 : 0;
+    p.plan = make_steer_plan(shape, steer);
+    p.sched = sched;
+    void* X = ws + w.x_off;
+    uint8_t* tile_hot = reinterpret_cast<uint8_t*>(ws + w.hot_off);
+    int* first_hot = reinterpret_cast<int*>(ws + w.first_off);
+    uint8_t* bh_info = reinterpret_cast<uint8_t*>(ws + w.info_off);
+    if (steer) {
+        stc = launch_prep_steering(shape, p.plan, k16, U, alpha, gain, head_enable, mask, X, tile_hot, first_hot, bh_info,
+                                   reinterpret_cast<int*>(ws),
+                                   w.n_tiles, st, Q, sigma, k_route, alpha_out);
+        if (stc != SEKA_OK) return stc;
+    }
+
+    TileMaps tm;
+    if (!make_tile_map(&tm.q, q16, D, Hq, T, 128) || !make_tile_map(&tm.k, k16, D, Hkv, T, 128) ||
+        !make_tile_map(&tm.v, v16, D, Hkv, T, 128))
+        return SEKA_ERR_CUDA;
+    tm.x = tm.k;      // never dereferenced without steering
+    if (p.plan.mode != 0 && !make_tile_map(&tm.x, X, p.plan.xcols, Hkv, T, 128)) return SEKA_ERR_CUDA;
+
+    p.O = O; p.lse = lse;
+    p.tile_hot = tile_hot; p.first_hot = first_hot; p.bh_info = bh_info; p.status = reinterpret_cast<int*>(ws);
+    p.steer = steer ? 1 : 0;
     ItemRecord* items = reinterpret_cast<ItemRecord*>(ws + w.item_off);
-    if (shape->cu_seqlens != nullptr)
-        launch_build_items(shape, w, steer, gain, head_enable, items, reinterpret_cast<int*>(ws) + 3, st);
-    p.pair_heads = w.pair_heads;
-    p.items = items; p.n_items = reinterpret_cast<int*>(ws) + 3; p.n_items_max = w.n_items_max;
+    const bool table = shape->cu_seqlens != nullptr;
+    if (table) launch_build_items(sched, shape->cu_seqlens, steer ? bh_info : nullptr, items, reinterpret_cast<int*>(ws) + 3, st);
+    p.items = items; p.n_items = reinterpret_cast<int*>(ws) + 3;
     const float scale = shape->softmax_scale > 0.f ? shape->softmax_scale : 1.f / sqrtf((float)D);
     p.scale_log2 = scale * 1.4426950408889634f;
 
     if (D == 128) {
-        return shape->dtype == SEKA_F32 ? launch_attn<128, float>(tq, tk, tv, tw, p, st)
-                                        : launch_attn<128, __nv_bfloat16>(tq, tk, tv, tw, p, st);
+        return shape->dtype == SEKA_F32 ? launch_attn<128, float>(tm, p, table, st)
+                                        : launch_attn<128, __nv_bfloat16>(tm, p, table, st);
     }
-    return shape->dtype == SEKA_F32 ? launch_attn<64, float>(tq, tk, tv, tw, p, st)
-                                    : launch_attn<64, __nv_bfloat16>(tq, tk, tv, tw, p, st);
+    return shape->dtype == SEKA_F32 ? launch_attn<64, float>(tm, p, table, st)
+                                    : launch_attn<64, __nv_bfloat16>(tm, p, table, st);
 }
 
 }  // namespace seka

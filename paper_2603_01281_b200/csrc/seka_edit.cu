@@ -599,7 +599,7 @@ extern "C" seka_status seka_edit_keys(const seka_shape* shape, const void* K_in,
     if (!K_in || !K_out || !mask || !U || !gain) return SEKA_ERR_INVALID_ARG;
     if (((uintptr_t)K_in | (uintptr_t)K_out) & 15) return SEKA_ERR_INVALID_ARG;
     const WorkspaceLayout w = workspace_layout(shape);
-    if (!workspace || workspace_bytes < w.total) return SEKA_ERR_WORKSPACE;
+    if (!workspace || workspace_bytes < w.edit_total) return SEKA_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     char* ws = static_cast<char*>(workspace);
     int* status = reinterpret_cast<int*>(ws);

@@ -8,14 +8,17 @@
 
 namespace seka {
 
-// With `sigma` set, the routing coefficients of Eq. 6 are computed inside the launch from Q_route (the caller's Q
-// in its own dtype) instead of being read from `alpha`, and written to `alpha_out` if that is not null.
-void launch_prep_steering(const seka_shape* s, const float* U, const float* alpha, const float* gain,
-                          const uint8_t* head_enable, const uint8_t* mask, void* W, uint8_t* tile_hot, int n_tiles,
-                          cudaStream_t st, const void* Q_route = nullptr, const float* sigma = nullptr, int k_route = 0,
-                          float* alpha_out = nullptr);
-void launch_build_items(const seka_shape* s, const WorkspaceLayout& w, bool steer, const float* gain,
-                        const uint8_t* head_enable, ItemRecord* items, int* count, cudaStream_t st);
+// Operand preparation of the fused kernel (tile flags, edited keys of the tiles with highlighted tokens; see seka_prep.cu).  With
+// `sigma` set, the routing coefficients of Eq. 6 are computed inside the launch from Q_route (the caller's Q in its own
+// dtype) instead of being read from `alpha`, and written to `alpha_out` if that is not null.
+seka_status launch_prep_steering(const seka_shape* s, const SteerPlan& plan, const void* K16, const float* U,
+                                 const float* alpha, const float* gain, const uint8_t* head_enable, const uint8_t* mask,
+                                 void* X, uint8_t* tile_hot, int* first_hot, uint8_t* bh_info, int* status, int n_tiles, cudaStream_t st,
+                                 const void* Q_route = nullptr, const float* sigma = nullptr, int k_route = 0,
+                                 float* alpha_out = nullptr);
+// `bh_info` (null: no steering) is the per-(sequence, KV head) byte the preparation launch wrote
+void launch_build_items(const Sched& sc, const int* cu, const uint8_t* bh_info, ItemRecord* items, int* count,
+                        cudaStream_t st);
 void launch_compact_mask(const uint8_t* mask, int T, int* list, int* count, cudaStream_t st);
 void launch_convert_bf16(const float* in, void* out, size_t n, cudaStream_t st);
 
@@ -26,5 +29,8 @@ void launch_prep_edit(const seka_shape* s, const float* U, const uint8_t* mask, 
 bool make_tile_map(CUtensorMap* m, const void* base, int d, int H, long long T, int box_rows = 128);
 
 seka_status validate_shape(const seka_shape* s);
+
+// Number of SMs of the current device (looked up once per device, thread-safe).
+bool device_info(int* n_sm);
 
 }  // namespace seka

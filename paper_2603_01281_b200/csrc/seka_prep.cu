@@ -5,81 +5,399 @@
 
 namespace seka {
 
-// Operand preparation of the fused kernel, one launch:
-//   blocks [0, n_w):   a 32 x 32 tile of W[b][h] = gain_b * sum_m alpha_{b,h,m} U_m[h] U_m[h]^T  (bf16 [D x D]; the
-//                      dynamic projector of Section 3.3 times the gain, or g U U^T for plain SEKA), so that the
-//                      edit of a key tile is one product  K' = K + K W  (W is symmetric).  Pairs (b, h) that are
-//                      not steered (zero gain, head switched off) are skipped: the fused kernel never reads them.
-//   blocks [n_w, ...): one warp per (sequence, 128-key tile): does the tile hold a highlighted token?
-// With `route.sigma` set the routing coefficients of Eq. 6 are computed here as well (each block of a (b, h) pair
-// repeats the few thousand multiply-adds, from the last token's query), so that AdaSEKA needs no launch of its own
-// before the forward; the coefficients are also written to `route.alpha_out` if that is set.
+// Operand preparation of the fused kernel, one launch.  The fused kernel stages every key tile that holds a highlighted
+// token from a side buffer of edited keys (Eq. 5: the edited logit is q.k' with k' = k + g P k); this launch writes it:
+//   blocks [0, n_flag):        one block per sequence: a flag per 128-key tile (does it hold a highlighted token?), the
+//                              sequence's first such tile, and per KV head whether it is steered and whether the fused
+//                              kernel multiplies the low parts too (see lo_needed);
+//   blocks [n_flag, +n_a):     (only with `route.alpha_out`) one block per (sequence, KV head): the routing coefficients
+//                              of Eq. 6, from the last token's query, for the caller;
+//   the remaining n_x blocks:  a KV head each (n_x is a multiple of Hkv); together the warps of a head's blocks walk the
+//                              tokens of every (sequence, key tile) pair that holds a highlighted token, a warp per token:
+//                                  k' = k + g_b sum_m alpha_{b,h,m} U_m[h] (U_m[h]^T k)   (highlighted tokens; k otherwise)
+//                              in fp32 (the contraction order of Algorithm 1's hook: first U^T k, then back through U),
+//                              written as a high and a low bf16 part into one row of `X` [T, Hkv, 2 d]: high parts at
+//                              columns [0, d), low parts at [d, 2 d) (only where the fused kernel reads them).  With
+//                              `route.sigma` set these blocks compute the coefficients of Eq. 6 themselves, so that
+//                              AdaSEKA needs no launch of its own before the forward.
+// Plain fp32 multiply-adds on purpose: warp-level mma.sync gets little from this GPU's tensor cores (measured: about
+// ten cycles per m16n8k16 and SM), the two bf16 parts it needs for fp32 accuracy triple the products, and it cannot
+// skip the tokens that are not highlighted.
 struct RouteArgs {
     const void* Q; int q_is_f32; const float* sigma; int k_route; int Hq; float* alpha_out;
 };
 
-__global__ void prep_steering_kernel(const float* __restrict__ U, const float* __restrict__ alpha,
-                                     const float* __restrict__ gain, const uint8_t* __restrict__ head_enable,
-                                     const uint8_t* __restrict__ mask, const int* __restrict__ cu_seqlens,
-                                     __nv_bfloat16* __restrict__ W, uint8_t* __restrict__ tile_hot,
-                                     int B, int L, int Hkv, int D, int r, int M, int n_tiles, int n_w,
-                                     const RouteArgs route) {
-    const int tid = threadIdx.x;
-    extern __shared__ double route_sm[];
-    if ((int)blockIdx.x < n_w) {
-        const int tiles = D / 32;
-        const int bh = blockIdx.x / (tiles * tiles), t = blockIdx.x % (tiles * tiles);
-        const int b = bh / Hkv, h = bh % Hkv;
-        const float g = gain[b];
-        const double* routed = nullptr;
-        if (route.sigma != nullptr) {
-            routed = route_group(route.Q, route.q_is_f32, U, route.sigma, cu_seqlens, L, route.Hq, Hkv, D, r, M,
-                                 route.k_route, b, h, route_sm);
-            if (t == 0 && route.alpha_out != nullptr)
-                for (int m = tid; m < M; m += blockDim.x) route.alpha_out[(size_t)bh * M + m] = (float)routed[m];
+constexpr int PREP_THREADS = 256;
+constexpr int HOT_CAP = 2048;  // (sequence, tile) pairs looked at per round of the edited-key blocks
+constexpr int ALPHA_CAP = 2048; // routed coefficients a block can hold (sequences x experts)
+__device__ __forceinline__ size_t align_up_dev(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// two fp32 values -> their high bf16 parts and their low bf16 parts, packed in pairs
+__device__ __forceinline__ void split_pair(float x, float y, uint32_t& hi, uint32_t& lo) {
+    const __nv_bfloat16 xh = __float2bfloat16_rn(x), yh = __float2bfloat16_rn(y);
+    hi = (uint32_t)__bfloat16_as_ushort(xh) | ((uint32_t)__bfloat16_as_ushort(yh) << 16);
+    lo = pack_bf16(x - __bfloat162float(xh), y - __bfloat162float(yh));
+}
+
+template <int D>
+__global__ void __launch_bounds__(PREP_THREADS, 2)
+prep_steering_kernel(const __grid_constant__ CUtensorMap tmK, int* status, const float* __restrict__ U, const float* __restrict__ alpha,
+                     const float* __restrict__ gain, const uint8_t* __restrict__ head_enable,
+                     const uint8_t* __restrict__ mask, const int* __restrict__ cu_seqlens,
+                     __nv_bfloat16* __restrict__ X, uint8_t* __restrict__ tile_hot, int* __restrict__ first_hot,
+                     uint8_t* __restrict__ bh_info, int B, int L, int Hkv, int r, int M, int n_tiles, int n_flag,
+                     int n_a, int n_x, const RouteArgs route) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    extern __shared__ __align__(16) unsigned char prep_sm[];
+    if ((int)blockIdx.x < n_flag) {
+        // ------------------------------------------------------------ flags of one sequence
+        const int b = blockIdx.x;
+        const int seq0 = cu_seqlens ? cu_seqlens[b] : b * L;
+        const int Lb = (cu_seqlens ? cu_seqlens[b + 1] : (b + 1) * L) - seq0;
+        __shared__ int first_s;
+        if (tid == 0) first_s = 0x7fffffff;
+        __syncthreads();
+        int first = 0x7fffffff;
+        for (int t = warp; t < n_tiles; t += PREP_THREADS / 32) {
+            bool any = false;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int pos = t * 128 + q * 32 + lane;
+                any = any || (pos < Lb && mask[seq0 + pos] != 0);
+            }
+            any = __any_sync(0xffffffffu, any);
+            if (lane == 0) tile_hot[(size_t)b * n_tiles + t] = any ? 1 : 0;
+            if (any && t < first) first = t;
         }
-        if (g == 0.f || (head_enable != nullptr && head_enable[h] == 0)) return;
-        const int i0 = (t / tiles) * 32, j0 = (t % tiles) * 32;
-        __shared__ float ui[32][33], uj[32][33];
-        const int tx = tid & 31, ty = tid >> 5;          // 256 threads: 8 rows of 32
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        if (lane == 0 && first != 0x7fffffff) atomicMin(&first_s, first);
+        const float g = gain[b];
+        for (int h = tid; h < Hkv; h += PREP_THREADS) {
+            const bool on = g != 0.f && (head_enable == nullptr || head_enable[h] != 0);
+            const float amax = route.sigma != nullptr ? 1.f : alpha_max_of(alpha, (size_t)b * Hkv + h, M);
+            bh_info[(size_t)b * Hkv + h] = (on ? 1 : 0) | ((on && lo_needed(g, amax)) ? 2 : 0);
+        }
+        __syncthreads();
+        if (tid == 0) first_hot[b] = first_s;
+        return;
+    }
+    if ((int)blockIdx.x < n_flag + n_a) {
+        // ------------------------------------------------------------ routing coefficients for the caller
+        const int bh = blockIdx.x - n_flag, b = bh / Hkv, h = bh % Hkv;
+        const double* a = route_group(route.Q, route.q_is_f32, U, route.sigma, cu_seqlens, L, route.Hq, Hkv, D, r, M,
+                                      route.k_route, b, h, reinterpret_cast<double*>(prep_sm));
+        for (int m = tid; m < M; m += PREP_THREADS) route.alpha_out[(size_t)bh * M + m] = (float)a[m];
+        return;
+    }
+    // ---------------------------------------------------------------- edited keys of one KV head, on tcgen05
+    // The block keeps the edit operator of its head in shared memory as the B operand of a tensor-core product, as a
+    // high and a low bf16 part (so that K W is fp32-accurate):  one expert: W = U U^T, and g_b alpha_{b,h} is applied to
+    // the product per token;  several experts: W = g_b sum_m alpha_{b,h,m} U_m U_m^T, rebuilt when the sequence changes.
+    // It walks a contiguous share of the head's (sequence, tile) pairs that hold a highlighted token: TMA stages the key
+    // tile (two stages: the next tile lands while this one is worked on), one thread issues K W into tensor memory, the
+    // eight warps add it to the highlighted rows (half a row per thread), split k' into its two bf16 parts (the high
+    // parts in place in the staged tile, the low parts straight to global memory) and write the high parts of all
+    // rows out, 16 bytes per lane with the lanes of a row adjacent.
+    const int kb = blockIdx.x - n_flag - n_a;
+    const int h = kb % Hkv, slot = kb / Hkv, n_slots = n_x / Hkv;
+    if (head_enable != nullptr && head_enable[h] == 0) return;
+    constexpr int NS = 2;
+    constexpr uint32_t TILE = (D / 64) * 128 * 128, PBLK = D * 128, PMAT = (D / 64) * PBLK;
+    constexpr uint32_t TMEM_COLS = 2 * D;
+    const int Rt = r * M;
+    const bool routed = route.sigma != nullptr;
+    // dynamic shared memory (1024-byte aligned): key stages | W high, low | a chunk of U^T | routing scratch and coefficients
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(prep_sm) + 1023) & ~uintptr_t(1023));
+    uint8_t* sW = smem + NS * TILE;
+    float* ut = reinterpret_cast<float*>(sW + 2 * PMAT);        // staged chunk of U^T: [32][D + 4]
+    unsigned char* tail = sW + 2 * PMAT + 32 * (D + 4) * 4;
+    float* alpha_s = reinterpret_cast<float*>(tail + (routed ? align_up_dev(route_smem_bytes(D, M, route.k_route), 16) : 0));
+    __shared__ __align__(8) uint64_t bars[NS + 2];
+    __shared__ uint32_t tmem_holder;
+    __shared__ int abort_s;
+    __shared__ unsigned char row_hl[NS][128];
+    uint64_t* full = bars;            // [NS] key tile landed
+    uint64_t* done = bars + NS;       // [2]  K W of a tile is in column set c
+    volatile int* abort_flag = &abort_s;
+    if (tid == 0) {
+        for (int i = 0; i < NS; ++i) mbar_init(full + i, 1);
+        mbar_init(done + 0, 1); mbar_init(done + 1, 1);
+        abort_s = 0;
+        mbar_fence_init();
+        tma_prefetch_desc(&tmK);
+    }
+    __syncwarp();
+    if (warp == 0) { tmem_alloc(&tmem_holder, TMEM_COLS); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_holder;
+    const uint32_t t_lane = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+    constexpr uint32_t IDESC = umma_idesc_bf16(D, false);
+    constexpr uint32_t DESC_HI = umma_desc_hi_sw128(1024);
+    const uint32_t dKd = umma_desc_lo(smem_u32(smem), 16), dWd = umma_desc_lo(smem_u32(sW), 16);
+
+    if (routed) {
+        // Eq. 6 for every sequence (the whole block works on one at a time)
+        for (int b = 0; b < B; ++b) {
+            const double* a = route_group(route.Q, route.q_is_f32, U, route.sigma, cu_seqlens, L, route.Hq, Hkv, D, r, M,
+                                          route.k_route, b, h, reinterpret_cast<double*>(tail));
+            for (int m = tid; m < M; m += PREP_THREADS) alpha_s[b * M + m] = (float)a[m];
+            __syncthreads();
+        }
+    }
+    auto coef = [&](int b, int m) -> float {
+        return routed ? alpha_s[b * M + m] : (alpha != nullptr ? alpha[((size_t)b * Hkv + h) * M + m] : 1.f);
+    };
+    // W (both parts) into shared memory in the operand layout: [D x 64] blocks of 128-byte rows, 128-byte swizzle.
+    // U is staged 32 columns at a time, transposed (ut[kk][i] = U_m[i][kk0 + kk]: read coalesced, then every read
+    // below is a row of ut); a thread forms PR rows x 16 columns of  W[n][k] = sum_j a_j U[n][j] U[k][j],  j = m r + kk,
+    // its 16 columns being two groups of 8 (one 16-byte unit of the operand each), 64 apart.
+    constexpr int UTP = D + 4;            // row pitch (floats) of ut: rows stay 16-byte aligned, transposed writes spread over banks
+    auto build_W = [&](int b_for) {       // b_for < 0: plain U U^T (one expert)
+        constexpr int PR = D * D / (PREP_THREADS * 16);
+        constexpr int CG = D / 16;                       // column groups: thread g takes columns 8 g .. and D/2 + 8 g ..
+        const int n0 = (tid / CG) * PR, kA = (tid % CG) * 8, kB = D / 2 + kA;
+        float acc[PR][16];
+#pragma unroll
+        for (int p = 0; p < PR; ++p)
+#pragma unroll
+            for (int q = 0; q < 16; ++q) acc[p][q] = 0.f;
+        const float gb = b_for >= 0 ? gain[b_for] : 1.f;
         for (int m = 0; m < M; ++m) {
-            const float a = g * (routed != nullptr ? (float)routed[m]
-                                                   : (alpha != nullptr ? alpha[((size_t)b * Hkv + h) * M + m] : 1.f));
+            const float am = b_for >= 0 ? gb * coef(b_for, m) : 1.f;
             const float* Um = U + ((size_t)m * Hkv + h) * D * r;
-            for (int k0 = 0; k0 < r; k0 += 32) {
+            for (int kk0 = 0; kk0 < r; kk0 += 32) {
+                const int kn = min(32, r - kk0);
                 __syncthreads();
-                for (int q = ty; q < 32; q += 8) {
-                    const bool in = k0 + tx < r;
-                    ui[q][tx] = in ? a * Um[(size_t)(i0 + q) * r + k0 + tx] : 0.f;
-                    uj[q][tx] = in ? Um[(size_t)(j0 + q) * r + k0 + tx] : 0.f;
+                {   // 32 D values, D / 8 per thread: all loads first, so that their latencies overlap
+                    constexpr int NL = 32 * D / PREP_THREADS;
+                    float v[NL];
+                    const int kk = tid & 31;
+#pragma unroll
+                    for (int q = 0; q < NL; ++q) {
+                        const int i = (tid >> 5) + q * (PREP_THREADS / 32);
+                        v[q] = kk < kn ? __ldg(Um + (size_t)i * r + kk0 + kk) : 0.f;
+                    }
+#pragma unroll
+                    for (int q = 0; q < NL; ++q) ut[kk * UTP + (tid >> 5) + q * (PREP_THREADS / 32)] = v[q];
                 }
                 __syncthreads();
+#pragma unroll 2
+                for (int kk = 0; kk < kn; ++kk) {
+                    const float* row = ut + kk * UTP;
+                    float un[PR], uk[16];
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const int i = ty + 8 * q;
-#pragma unroll 8
-                    for (int k = 0; k < 32; ++k) acc[q] = fmaf(ui[i][k], uj[tx][k], acc[q]);
+                    for (int p = 0; p < PR; ++p) un[p] = am * row[n0 + p];
+#pragma unroll
+                    for (int q4 = 0; q4 < 2; ++q4) {
+                        const float4 a4 = *reinterpret_cast<const float4*>(row + kA + 4 * q4);
+                        const float4 b4 = *reinterpret_cast<const float4*>(row + kB + 4 * q4);
+                        uk[4 * q4] = a4.x; uk[4 * q4 + 1] = a4.y; uk[4 * q4 + 2] = a4.z; uk[4 * q4 + 3] = a4.w;
+                        uk[8 + 4 * q4] = b4.x; uk[8 + 4 * q4 + 1] = b4.y; uk[8 + 4 * q4 + 2] = b4.z; uk[8 + 4 * q4 + 3] = b4.w;
+                    }
+#pragma unroll
+                    for (int p = 0; p < PR; ++p)
+#pragma unroll
+                        for (int q = 0; q < 16; ++q) acc[p][q] = fmaf(un[p], uk[q], acc[p][q]);
                 }
             }
         }
-        __nv_bfloat16* Wbh = W + (size_t)bh * D * D;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) Wbh[(size_t)(i0 + ty + 8 * q) * D + j0 + tx] = __float2bfloat16_rn(acc[q]);
-    } else {
-        const int item = ((int)blockIdx.x - n_w) * 8 + (tid >> 5), lane = tid & 31;
-        if (item >= B * n_tiles) return;
-        const int b = item / n_tiles, t = item % n_tiles;
-        const int seq0 = cu_seqlens ? cu_seqlens[b] : b * L;
-        const int Lb = (cu_seqlens ? cu_seqlens[b + 1] : (b + 1) * L) - seq0;
-        bool any = false;
-        for (int q = 0; q < 4; ++q) {
-            const int pos = t * 128 + q * 32 + lane;
-            any = any || (pos < Lb && mask[seq0 + pos] != 0);
+        for (int p = 0; p < PR; ++p) {
+            uint32_t hi[8], lo[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) split_pair(acc[p][2 * q], acc[p][2 * q + 1], hi[q], lo[q]);
+#pragma unroll
+            for (int u8 = 0; u8 < 2; ++u8) {
+                const int k0 = u8 ? kB : kA;
+                uint8_t* dst = sW + (k0 >> 6) * PBLK + sw128_offset(n0 + p, k0 & 63);
+                *reinterpret_cast<uint4*>(dst) = make_uint4(hi[4 * u8], hi[4 * u8 + 1], hi[4 * u8 + 2], hi[4 * u8 + 3]);
+                *reinterpret_cast<uint4*>(dst + PMAT) = make_uint4(lo[4 * u8], lo[4 * u8 + 1], lo[4 * u8 + 2], lo[4 * u8 + 3]);
+            }
         }
-        any = __any_sync(0xffffffffu, any);
-        if (lane == 0) tile_hot[item] = any ? 1 : 0;
+        fence_proxy_async();           // read next by the tensor core
+    };
+
+    // The (sequence, tile) pairs that hold a highlighted token, HOT_CAP candidates at a time: every block finds them for
+    // itself (eight lanes per pair, 16 mask bytes each), so that the walk below only meets tiles with work.
+    __shared__ int hot_list[HOT_CAP];
+    __shared__ unsigned char hot_flag[HOT_CAP];
+    __shared__ int warp_cnt[PREP_THREADS / 32];
+    const int n_pairs = B * n_tiles;
+    uint32_t n_load = 0, n_mma = 0;       // tiles loaded / multiplied so far (stage, column set and phases)
+    int built_for = -2;                   // sequence W was built for (-1: plain U U^T, -2: nothing yet)
+    bool ok = true;
+    for (int p0 = 0; p0 < n_pairs && ok; p0 += HOT_CAP) {
+        __syncthreads();
+        const int p1 = min(n_pairs, p0 + HOT_CAP);
+        for (int i = tid; i < HOT_CAP; i += PREP_THREADS) hot_flag[i] = 0;
+        __syncthreads();
+        for (int pp0 = p0; pp0 < p1; pp0 += PREP_THREADS / 8) {
+            const int pp = pp0 + (tid >> 3), part = tid & 7;
+            bool any = false;
+            if (pp < p1) {
+                const int b = pp / n_tiles, t = pp - b * n_tiles;
+                const int seq0 = cu_seqlens ? cu_seqlens[b] : b * L;
+                const int Lb = (cu_seqlens ? cu_seqlens[b + 1] : (b + 1) * L) - seq0;
+                const int pos0 = t * 128 + part * 16;
+                if (gain[b] != 0.f && pos0 < Lb) {
+                    const uint8_t* mp = mask + seq0 + pos0;
+                    if (pos0 + 16 <= Lb && (reinterpret_cast<uintptr_t>(mp) & 15) == 0) {
+                        const uint4 w = *reinterpret_cast<const uint4*>(mp);
+                        any = (w.x | w.y | w.z | w.w) != 0;
+                    } else {
+                        for (int q = 0; q < 16; ++q) any = any || (pos0 + q < Lb && mp[q] != 0);
+                    }
+                }
+            }
+            any = __any_sync(0xffu << (lane & 24), any);
+            if (part == 0 && pp < p1) hot_flag[pp - p0] = any ? 1 : 0;
+        }
+        __syncthreads();
+        // the pairs in order (the same list in every block: the blocks of a head share it out by position)
+        constexpr int PER = HOT_CAP / PREP_THREADS;
+        int cnt = 0;
+#pragma unroll
+        for (int q = 0; q < PER; ++q) cnt += hot_flag[tid * PER + q];
+        int incl = cnt;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int o = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += o;
+        }
+        if (lane == 31) warp_cnt[warp] = incl;
+        __syncthreads();
+        int base = incl - cnt, n_hot = 0;
+#pragma unroll
+        for (int w = 0; w < PREP_THREADS / 32; ++w) { if (w < warp) base += warp_cnt[w]; n_hot += warp_cnt[w]; }
+#pragma unroll
+        for (int q = 0; q < PER; ++q)
+            if (hot_flag[tid * PER + q]) {
+                const int pp = p0 + tid * PER + q, b = pp / n_tiles, t = pp - b * n_tiles;
+                hot_list[base++] = b | (t << 16);
+            }
+        __syncthreads();
+
+        // this block's contiguous share of the list
+        const int i0 = (int)((long long)slot * n_hot / n_slots), i1 = (int)((long long)(slot + 1) * n_hot / n_slots);
+        auto load_tile = [&](int i) {      // thread 0: key tile of list entry i into the next stage
+            const int e = hot_list[i], b = e & 0xffff, t = e >> 16;
+            const int seq0 = cu_seqlens ? cu_seqlens[b] : b * L;
+            const uint32_t st = n_load % NS;
+            mbar_expect_tx(full + st, TILE);
+#pragma unroll
+            for (int c = 0; c < D / 64; ++c) tma_load_3d(smem + st * TILE + c * (128 * 128), &tmK, full + st, c * 64, h, seq0 + t * 128);
+        };
+        if (i0 < i1 && tid == 0) load_tile(i0);
+        if (i0 < i1) ++n_load;
+        for (int i = i0; i < i1 && ok; ++i) {
+            const int e = hot_list[i], b = e & 0xffff, t = e >> 16;
+            const int seq0 = cu_seqlens ? cu_seqlens[b] : b * L;
+            const int Lb = (cu_seqlens ? cu_seqlens[b + 1] : (b + 1) * L) - seq0;
+            const float g = gain[b];
+            const uint32_t st = n_mma % NS, cs = n_mma & 1;
+            // the operator for this tile (the previous tile is through: every iteration ends with a barrier)
+            const int want = M == 1 ? -1 : b;
+            if (built_for != want) { build_W(want); built_for = want; }
+            // highlight flags of the tile's rows; the next tile starts to land meanwhile
+            if (tid < 128) {
+                const int kpos = t * 128 + tid;
+                row_hl[st][tid] = (kpos < Lb && mask[seq0 + kpos] != 0) ? 1 : 0;
+            }
+            if (i + 1 < i1) {
+                if (tid == 0) load_tile(i + 1);
+                ++n_load;
+            }
+            __syncthreads();               // W and the flags are in place
+            ok = mbar_wait(full + st, ((n_mma / NS) & 1), abort_flag, status, 70);
+            if (ok && tid == 0) {
+                tc_fence_after();
+                const uint32_t kd = dKd + st * (TILE >> 4);
+#pragma unroll
+                for (int part = 0; part < 2; ++part)
+#pragma unroll
+                    for (int ks = 0; ks < D / 16; ++ks) {
+                        const uint32_t offk = ((uint32_t)(ks >> 2) * (128 * 128) + (uint32_t)(ks & 3) * 32) >> 4;
+                        const uint32_t offw = ((uint32_t)part * PMAT + (uint32_t)(ks >> 2) * PBLK + (uint32_t)(ks & 3) * 32) >> 4;
+                        umma_ss(tmem_base + cs * D, kd + offk, DESC_HI, dWd + offw, DESC_HI, IDESC, (ks > 0 || part) ? 1u : 0u);
+                    }
+                umma_commit(done + cs);
+            }
+            if (ok) ok = mbar_wait(done + cs, (n_mma >> 1) & 1, abort_flag, status, 71);
+            ok = __syncthreads_and(ok);
+            if (!ok) break;
+            tc_fence_after();
+            ++n_mma;
+            // k' = k + c (K W)[row] for highlighted rows; high parts in place, low parts to global memory
+            const float amax = routed ? 1.f : alpha_max_of(alpha, (size_t)b * Hkv + h, M);
+            const bool with_lo = lo_needed(g, amax);
+            const float c = M == 1 ? g * coef(b, 0) : 1.f;
+            const int row = tid & 127, half = tid >> 7;
+            const bool hl = row_hl[st][row] != 0;
+            const int kpos = t * 128 + row;
+            const bool valid = kpos < Lb;
+            uint8_t* sK = smem + st * TILE;
+            __nv_bfloat16* xlo = X + ((size_t)(seq0 + (valid ? kpos : 0)) * Hkv + h) * (2 * D) + D;
+            const bool warp_hl = __any_sync(0xffffffffu, hl);
+#pragma unroll 1
+            for (int cb = half * (D / 64); cb < (half + 1) * (D / 64); ++cb) {
+                uint32_t v[32];
+                if (warp_hl) { tmem_ld32(t_lane + cs * D + cb * 32, v); tmem_wait_ld_on(v); }      // warp-wide: every lane takes part
+                uint4 lo4[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) lo4[q] = make_uint4(0u, 0u, 0u, 0u);
+                if (hl) {
+                    uint4* ptr[4];
+                    uint4 kv[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {      // 8 elements = one 16-byte unit of the swizzled row; reads before writes
+                        const int col = cb * 32 + q * 8;
+                        ptr[q] = reinterpret_cast<uint4*>(sK + (col >> 6) * (128 * 128) + sw128_offset(row, col & 63));
+                        kv[q] = *ptr[q];
+                    }
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        uint32_t* w = reinterpret_cast<uint32_t*>(&kv[q]);
+                        uint32_t* l = reinterpret_cast<uint32_t*>(&lo4[q]);
+#pragma unroll
+                        for (int e2 = 0; e2 < 4; ++e2) {
+                            const float2 k2 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&w[e2]));
+                            split_pair(fmaf(c, __uint_as_float(v[q * 8 + 2 * e2]), k2.x), fmaf(c, __uint_as_float(v[q * 8 + 2 * e2 + 1]), k2.y), w[e2], l[e2]);
+                        }
+                    }
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) *ptr[q] = kv[q];
+                }
+                if (with_lo && valid) {
+                    uint4* dst = reinterpret_cast<uint4*>(xlo + cb * 32);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) dst[q] = lo4[q];
+                }
+                __syncwarp();      // all lanes together again before the next warp-wide load
+            }
+            tc_fence_before();
+            __syncthreads();
+            // the high parts of all rows of the sequence go out: D / 8 lanes per row, 16 bytes each; 16 rows per warp
+            constexpr int LPR = D / 8, RPI = 32 / LPR;
+#pragma unroll 1
+            for (int q = 0; q < 16 / RPI; ++q) {
+                const int rr = warp * 16 + q * RPI + lane / LPR, col = (lane % LPR) * 8;
+                if (t * 128 + rr < Lb) {
+                    const uint4 val = *reinterpret_cast<const uint4*>(sK + (col >> 6) * (128 * 128) + sw128_offset(rr, col & 63));
+                    *reinterpret_cast<uint4*>(X + ((size_t)(seq0 + t * 128 + rr) * Hkv + h) * (2 * D) + col) = val;
+                }
+            }
+            __syncthreads();        // the stage, the flags and the columns are reused
+        }
     }
+    // a load that was armed may still be in flight after an abort: let it land before the shared memory is released
+    if (!ok && tid == 0 && n_load > n_mma) {
+        int dummy = 0;
+        mbar_wait(full + n_mma % NS, (n_mma / NS) & 1, &dummy, nullptr, 0);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem_base, TMEM_COLS);
 }
 
 // Operand preparation of the stand-alone edit, one launch:
@@ -144,62 +462,25 @@ __global__ void prep_edit_kernel(const float* __restrict__ U, const uint8_t* __r
     }
 }
 
-// Item table of the fused kernel: slot idx (heaviest row tiles first; the items of one (sequence, KV head)
-// next to each other) decoded into an ItemRecord.  Returns false for a slot whose tiles lie beyond the
-// sequence.
-__device__ __forceinline__ bool decode_item(long long idx, int B, int L, int Hq, int Hkv, int n_qt, int pair_heads,
-                                            const int* __restrict__ cu, int steer_call, const float* __restrict__ gain,
-                                            const uint8_t* __restrict__ head_enable, ItemRecord& r) {
-    int hqA, hqB, qtA, qtB;
-    if (pair_heads) {
-        const int per_qt = B * (Hq >> 1);
-        const int qt = n_qt - 1 - (int)(idx / per_qt);
-        const int rem = (int)(idx % per_qt);
-        r.b = rem / (Hq >> 1);
-        const int hp = rem % (Hq >> 1);
-        hqA = 2 * hp; hqB = 2 * hp + 1; qtA = qtB = qt;
-    } else {
-        const int per_qt = B * Hq;
-        const int qt2 = ((n_qt + 1) >> 1) - 1 - (int)(idx / per_qt);
-        const int rem = (int)(idx % per_qt);
-        r.b = rem / Hq;
-        hqA = hqB = rem % Hq; qtA = 2 * qt2; qtB = 2 * qt2 + 1;
-    }
-    r.hkv = hqA / (Hq / Hkv);
-    r.seq0 = cu ? cu[r.b] : r.b * L;
-    r.Lb = (cu ? cu[r.b + 1] : (r.b + 1) * L) - r.seq0;
-    const int nA = qtA * 128 < r.Lb ? qtA + 1 : 0, nB = qtB * 128 < r.Lb ? qtB + 1 : 0;
-    r.hq = hqA | (hqB << 16); r.qt = qtA | (qtB << 16); r.n = nA | (nB << 16);
-    r.steer = (steer_call && gain[r.b] != 0.f && (head_enable == nullptr || head_enable[r.hkv] != 0)) ? 1 : 0;
-    return nA > 0;
-}
-
-// Fixed-length batches have no empty slots: one thread per item.
-__global__ void build_items_kernel(long long n, int B, int L, int Hq, int Hkv, int n_qt, int pair_heads, int steer_call,
-                                   const float* __restrict__ gain, const uint8_t* __restrict__ head_enable,
-                                   ItemRecord* __restrict__ items, int* __restrict__ count) {
-    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx == 0) *count = (int)n;
-    if (idx >= n) return;
-    ItemRecord r;
-    decode_item(idx, B, L, Hq, Hkv, n_qt, pair_heads, nullptr, steer_call, gain, head_enable, r);
-    items[idx] = r;
-}
-
-// Packed variable-length batches: slots beyond a short sequence are dropped, order kept (one CTA scans).
-__global__ void build_items_varlen_kernel(long long n, int B, int L, int Hq, int Hkv, int n_qt, int pair_heads,
-                                          const int* __restrict__ cu, int steer_call, const float* __restrict__ gain,
-                                          const uint8_t* __restrict__ head_enable, ItemRecord* __restrict__ items,
-                                          int* __restrict__ count) {
+// Item table of the fused kernel for packed variable-length batches: items (see decode_item) whose tiles lie beyond
+// their sequence are dropped, order kept (one CTA scans).
+__global__ void build_items_varlen_kernel(const Sched sc, const int* __restrict__ cu, const uint8_t* __restrict__ bh_info,
+                                          ItemRecord* __restrict__ items, int* __restrict__ count) {
     __shared__ int warp_tot[32];
     __shared__ int base_s;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nw = blockDim.x >> 5;
     if (tid == 0) base_s = 0;
     __syncthreads();
+    const long long n = sc.n_items_max;
     for (long long start = 0; start < n; start += blockDim.x) {
         const long long idx = start + tid;
         ItemRecord r;
-        const bool keep = idx < n && decode_item(idx, B, L, Hq, Hkv, n_qt, pair_heads, cu, steer_call, gain, head_enable, r);
+        bool keep = false;
+        if (idx < n) {
+            keep = decode_item(sc, idx, cu, r);
+            const int b = r.bh & 0xffff, hkv = r.bh >> 16;
+            r.steer = bh_info != nullptr ? (int)bh_info[b * sc.Hkv + hkv] : 0;
+        }
         const unsigned bal = __ballot_sync(0xffffffffu, keep);
         if (lane == 0) warp_tot[wid] = __popc(bal);
         __syncthreads();
@@ -238,20 +519,52 @@ __global__ void convert_f32_bf16_kernel(const float4* __restrict__ in, uint2* __
     out[i] = make_uint2(pack_bf16(v.x, v.y), pack_bf16(v.z, v.w));
 }
 
-void launch_prep_steering(const seka_shape* sh, const float* U, const float* alpha, const float* gain,
-                          const uint8_t* head_enable, const uint8_t* mask, void* W, uint8_t* tile_hot, int n_tiles,
-                          cudaStream_t st, const void* Q_route, const float* sigma, int k_route, float* alpha_out) {
-    const int D = sh->head_dim, tiles = D / 32;
-    const int n_w = sh->batch * sh->n_kv_heads * tiles * tiles;
-    const int n_flag = (sh->batch * n_tiles + 7) / 8;
+static size_t route_bytes_aligned(int D, int M, int k_route) { return align_up(route_smem_bytes(D, M, k_route), 16); }
+
+// dynamic shared memory of prep_steering_kernel: the routing scratch (blocks that route), then the staged chunk of U
+// in both layouts (blocks that form edited keys)
+size_t prep_steering_smem(const seka_shape* sh, bool routed, int k_route) {
+    const int D = sh->head_dim;
+    const size_t tile = (size_t)(D / 64) * 128 * 128, pmat = (size_t)D * D * 2;
+    const size_t route = routed ? route_bytes_aligned(D, sh->n_experts, k_route) + (size_t)ALPHA_CAP * 4 : 0;
+    return 1024 + 2 * tile + 2 * pmat + (size_t)32 * (D + 4) * 4 + route;
+}
+
+seka_status launch_prep_steering(const seka_shape* sh, const SteerPlan& plan, const void* K16, const float* U,
+                                 const float* alpha, const float* gain, const uint8_t* head_enable, const uint8_t* mask,
+                                 void* X, uint8_t* tile_hot, int* first_hot, uint8_t* bh_info, int* status, int n_tiles,
+                                 cudaStream_t st, const void* Q_route, const float* sigma, int k_route, float* alpha_out) {
+    (void)plan;
+    const int D = sh->head_dim, Hkv = sh->n_kv_heads;
+    const bool routed = sigma != nullptr;
+    if (routed && (long long)sh->batch * sh->n_experts > ALPHA_CAP) return SEKA_ERR_UNSUPPORTED;
+    const int n_flag = sh->batch;
+    const int n_a = (routed && alpha_out != nullptr) ? sh->batch * Hkv : 0;
+    int n_sm = 0;
+    if (!device_info(&n_sm)) return SEKA_ERR_CUDA;
+    // blocks per KV head for the edited keys: about one wave of the device (shared and tensor memory decide how many
+    // blocks fit an SM), at most one per (sequence, tile)
+    const size_t smem = prep_steering_smem(sh, routed, k_route);
+    if (smem > 200 * 1024) return SEKA_ERR_UNSUPPORTED;
+    const int per_sm = D == 64 && smem <= 64 * 1024 ? 3 : 1;
+    // (one wave: a block that had to wait for a free SM would finish a whole block-time later)
+    long long per_head = ((long long)per_sm * n_sm - n_flag - n_a) / Hkv;
+    const long long pairs = (long long)sh->batch * n_tiles;
+    if (per_head > pairs) per_head = pairs;
+    if (per_head < 1) per_head = 1;
+    const long long n_x = per_head * Hkv;
+    if (n_flag + n_a + n_x > 0x7fffffffLL) return SEKA_ERR_UNSUPPORTED;
     RouteArgs route{Q_route, sh->dtype == SEKA_F32 ? 1 : 0, sigma, k_route, sh->n_q_heads, alpha_out};
-    const size_t smem = sigma != nullptr ? route_smem_bytes(D, sh->n_experts, k_route) : 0;
-    if (smem > 48 * 1024) cudaFuncSetAttribute(prep_steering_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    prep_steering_kernel<<<n_w + n_flag, 256, smem, st>>>(U, alpha, gain, head_enable, mask, sh->cu_seqlens,
-                                                         static_cast<__nv_bfloat16*>(W), tile_hot, sh->batch,
-                                                         sh->max_seqlen, sh->n_kv_heads, D, sh->rank, sh->n_experts,
-                                                         n_tiles, n_w, route);
+    CUtensorMap tk;
+    if (!make_tile_map(&tk, K16, D, Hkv, shape_total_tokens(sh), 128)) return SEKA_ERR_CUDA;
+    auto kern = D == 128 ? prep_steering_kernel<128> : prep_steering_kernel<64>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return SEKA_ERR_CUDA;
+    kern<<<(unsigned)(n_flag + n_a + n_x), PREP_THREADS, smem, st>>>(
+        tk, status, U, alpha, gain, head_enable, mask, sh->cu_seqlens,
+        static_cast<__nv_bfloat16*>(X), tile_hot, first_hot, bh_info, sh->batch, sh->max_seqlen,
+        Hkv, sh->rank, sh->n_experts, n_tiles, n_flag, n_a, (int)n_x, route);
     ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? SEKA_OK : SEKA_ERR_CUDA;
 }
 
 void launch_prep_edit(const seka_shape* sh, const float* U, const uint8_t* mask, void* P, uint8_t* tile_hot, int n_tiles,
@@ -266,16 +579,9 @@ void launch_prep_edit(const seka_shape* sh, const float* U, const uint8_t* mask,
     ++g_launches;
 }
 
-void launch_build_items(const seka_shape* sh, const WorkspaceLayout& w, bool steer, const float* gain,
-                        const uint8_t* head_enable, ItemRecord* items, int* count, cudaStream_t st) {
-    const long long n = w.n_items_max;
-    if (sh->cu_seqlens == nullptr)
-        build_items_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(n, sh->batch, sh->max_seqlen, sh->n_q_heads,
-                                                                       sh->n_kv_heads, w.n_tiles, w.pair_heads, steer ? 1 : 0,
-                                                                       gain, head_enable, items, count);
-    else
-        build_items_varlen_kernel<<<1, 1024, 0, st>>>(n, sh->batch, sh->max_seqlen, sh->n_q_heads, sh->n_kv_heads, w.n_tiles,
-                                                      w.pair_heads, sh->cu_seqlens, steer ? 1 : 0, gain, head_enable, items, count);
+void launch_build_items(const Sched& sc, const int* cu, const uint8_t* bh_info, ItemRecord* items, int* count,
+                        cudaStream_t st) {
+    build_items_varlen_kernel<<<1, 1024, 0, st>>>(sc, cu, bh_info, items, count);
     ++g_launches;
 }
 

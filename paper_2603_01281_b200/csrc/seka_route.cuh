@@ -16,6 +16,9 @@ static inline int route_chunks(int M, int k_route) {
     return pairs <= 512 ? 8 : (pairs <= 2048 ? 2 : 1);
 }
 // shared memory of route_group: the summed query, one term per (expert, piece, singular direction), the coefficients
+#ifdef __CUDACC__
+__host__ __device__
+#endif
 static inline size_t route_smem_bytes(int D, int M, int k_route) {
     return sizeof(double) * ((size_t)D + (size_t)M * k_route * route_chunks(M, k_route) + M + 1);
 }
