@@ -243,7 +243,7 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         it.n_kv = max(it.nA, it.nB);
         it.steer = (rec.steer & 1) != 0 && p.plan.mode != 0;
         it.hot_any = it.steer && p.first_hot[it.b] < it.n_kv;
-        it.need_lo = it.hot_any && (rec.steer & 2) != 0;
+        it.need_lo = it.hot_any && ((rec.steer & 2) != 0 || it.n_kv <= kLoTiles);
         return true;
     };
 

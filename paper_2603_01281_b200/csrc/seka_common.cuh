@@ -60,9 +60,16 @@ static inline SteerPlan make_steer_plan(const seka_shape* s, bool steer) {
     return p;
 }
 
-// Staged form: is the low part of k' worth a second product?  One bf16 rounding of k' perturbs a logit by about
-// 2^-9 |q| |k'| / sqrt(3 d) in scaled units; with |k'| <= (1 + |g| a) |k| (a = largest |alpha|) and unit-variance
-// inputs that stays several times below the rounding of P itself while |g| a <= 1.  Beyond that the low part is used.
+// Is the low part of k' worth a second product?  One bf16 rounding of k' perturbs a logit by about
+// eps = 2^-9 |q| |k'| / sqrt(3 d) in scaled units (1.2e-3 (1 + |g| a) for unit-variance inputs, a = largest |alpha|),
+// and the output by about eps |v - o| sqrt(sum_j p_j^2).  Two cases take the low parts:
+//   - |g| a > 1: the edited keys are far from unit variance and eps grows with them;
+//   - query rows that see at most kLoTiles key tiles (1024 keys): with few keys sqrt(sum p^2) is not small and the
+//     tail of that noise reaches the stated 1e-2 on single elements (seen on a 35-key row at g = 1); these work items
+//     are a few per cent of the steps of a long prompt.
+// Everywhere else (long rows, |g| a <= 1) the noise is averaged over thousands of keys and stays several times
+// below the rounding of P itself.
+constexpr int kLoTiles = 8;
 #if defined(__CUDACC__)
 __host__ __device__
 #endif

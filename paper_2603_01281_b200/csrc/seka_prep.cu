@@ -330,7 +330,7 @@ prep_steering_kernel(const __grid_constant__ CUtensorMap tmK, int* status, const
             ++n_mma;
             // k' = k + c (K W)[row] for highlighted rows; high parts in place, low parts to global memory
             const float amax = routed ? 1.f : alpha_max_of(alpha, (size_t)b * Hkv + h, M);
-            const bool with_lo = lo_needed(g, amax);
+            const bool with_lo = lo_needed(g, amax) || t < kLoTiles;     // what the fused kernel reads (see lo_needed)
             const float c = M == 1 ? g * coef(b, 0) : 1.f;
             const int row = tid & 127, half = tid >> 7;
             const bool hl = row_hl[st][row] != 0;

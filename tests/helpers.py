@@ -67,30 +67,17 @@ def oracle_rows(w, rows, alpha=None, head_enable=None):
                                  head_enable=head_enable, rows=rows)
 
 
-def key_magnification(w):
-    """RMS growth of an edited key relative to a unit-variance key: the edit multiplies the component
-    inside the steered subspace (dimension R = min(d, M r)) by (1+g) (Eq. 12) and the added term
-    itself has size |g|, so kappa = sqrt((R a^2 + d - R) / d) with a = max(|g|, |1+g|, 1) at the
-    largest gain of the batch; never below 1."""
-    d = w.head_dim
-    R = min(d, w.rank * w.n_experts)
-    g = w.gain.astype(np.float64)
-    a = float(max(1.0, np.max(np.abs(g)), np.max(np.abs(1.0 + g)))) if g.size else 1.0
-    return float(np.sqrt((R * a * a + d - R) / d))
-
-
-def check_attention(O_gpu, O_ref, label="", kappa=1.0):
+def check_attention(O_gpu, O_ref, label=""):
     """Stated tolerance for bf16 attention output on unit-variance inputs: max abs error 1e-2 and
     mean abs error 1e-3.  Where |o| > 1.28 the rounding of the bf16 output alone can reach 2^-8 |o|,
-    so the per-element bound is max(1e-2, 2^-7 |o|) (one bf16 ulp, relative).  ``kappa`` widens both
-    bounds for stress cases whose edited keys are far from unit variance (large |g| on a wide
-    subspace): the bf16 rounding of k' perturbs the logits in proportion to |k'|."""
+    so the per-element bound is max(1e-2, 2^-7 |o|) (one bf16 ulp, relative).  The bound is used as
+    stated for every gain: the edited keys enter the score product with fp32 accuracy."""
     err = np.abs(O_gpu - O_ref)
     assert np.isfinite(O_gpu).all(), label + ": non-finite output"
-    bound = kappa * np.maximum(1e-2, 2.0 ** -7 * np.abs(O_ref))
+    bound = np.maximum(1e-2, 2.0 ** -7 * np.abs(O_ref))
     worst = float((err / bound).max()) if err.size else 0.0
     assert worst <= 1.0, "%s: max abs err %.4g (ratio to bound %.3f)" % (label, err.max(), worst)
-    assert err.size == 0 or err.mean() <= 1e-3 * kappa, "%s: mean abs err %.4g" % (label, err.mean())
+    assert err.size == 0 or err.mean() <= 1e-3, "%s: mean abs err %.4g" % (label, err.mean())
     return float(err.max()) if err.size else 0.0, float(err.mean()) if err.size else 0.0
 
 
