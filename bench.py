@@ -31,9 +31,12 @@ if ROOT not in sys.path:
 
 METRIC = "SEKA fused attention TFLOP/s (% BF16 peak); overhead vs g=0, 8B shape"
 WORKLOAD = "C2: 8B-shaped prefill layer B=4 Hq=32 Hkv=8 d=128 L=4096 bf16, rank 32, ~10% highlighted spans, g=1"
-# DRAM bytes of one fused-kernel launch on this workload from the ncu capture summarised in
-# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture exists.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 437662720  # profiles/seka_attn_fwd_kernel_d128_C2.md (341.05 MB read + 96.61 MB written)
+# Counters of one fused-kernel launch on this workload, from the ncu capture of the current kernel (summary under
+# profiles/): dram__bytes_read.sum + dram__bytes_write.sum, and sm__pipe_tensor_cycles_active in per cent.
+# None means: no capture of the kernel as it stands.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+NCU_TENSOR_PIPE_ACTIVE_PCT = None
+NOMINAL_BF16_TFLOPS = 2250.0      # dense bf16, datasheet
 
 
 def measured_peaks():
@@ -117,7 +120,7 @@ def cpu_oracle_sample(w, budget_s: float, seed: int = 0):
 def edit_keys_bench(w, peaks, layers: int = 36, steps: int = 20):
     """Stand-alone key edit on a layer-stacked key cache [layers * B, L, Hkv, d] (bf16, in place): the hook of
     Algorithm 1 applied to the cached keys of every layer of an 8B-shaped model in one launch.  Returns achieved
-    GB/s on the algorithmic bytes (highlighted rows read and written once, the mask read once) at two densities."""
+    GB/s on the algorithmic bytes (highlighted rows read and written once, the mask read once) at three densities."""
     import torch
     from paper_2603_01281_b200 import binding
     out = {}
@@ -128,7 +131,9 @@ def edit_keys_bench(w, peaks, layers: int = 36, steps: int = 20):
     shp = binding.make_shape(batch=B, max_seqlen=L, n_q_heads=w.n_q_heads, n_kv_heads=Hkv, head_dim=d, rank=w.rank,
                              n_experts=1, dtype=torch.bfloat16)
     ws = binding.new_workspace(shp)
+    from paper_2603_01281_b200 import inputs as _inputs
     masks = {"10pct_spans": torch.from_numpy(np.tile(w.mask, layers)).cuda(),
+             "70pct_span": torch.from_numpy(np.tile(_inputs.make_workload("C2s70").mask, layers)).cuda(),
              "100pct": torch.ones(B * L, dtype=torch.uint8, device="cuda")}
     for name, mask in masks.items():
         n_h = int(mask.sum().item())
@@ -222,6 +227,139 @@ def learn_bench(peaks, n: int = 32768, slots: int = 288, d: int = 128, steps: in
             "k_pos_mean": float(res["k_pos"].float().mean().item())}
 
 
+def oracle_c1_single_thread():
+    """Whole C1 configuration (edit + attention, every row) through the oracle on one host thread, in a child process
+    (the thread count of the C routine is fixed when its runtime starts)."""
+    code = ("import time, sys; sys.path.insert(0, %r); import oracle; from paper_2603_01281_b200 import inputs; "
+            "w = inputs.make_workload('C1'); oracle.seka_attention(w.Q, w.K, w.V, w.mask, w.cu_seqlens, w.U, gain=w.gain); "
+            "t = time.perf_counter(); oracle.seka_attention(w.Q, w.K, w.V, w.mask, w.cu_seqlens, w.U, gain=w.gain); "
+            "print(time.perf_counter() - t, oracle.threads(), w.attention_flops())" % ROOT)
+    env = dict(os.environ, OMP_NUM_THREADS="1")
+    try:
+        out = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=120).stdout.split()
+        secs, thr, fl = float(out[-3]), int(out[-2]), float(out[-1])
+        return {"seconds": secs, "threads": thr, "TFLOP/s": fl / secs / 1e12}
+    except Exception as exc:      # the figure is context only: never fail the bench line for it
+        return {"error": str(exc)[:100]}
+
+
+class FusedRunner:
+    """One workload on the device with everything a fused call needs (and a scratch key tensor for the unfused arm)."""
+
+    def __init__(self, w):
+        import torch
+        from paper_2603_01281_b200 import binding
+        self.w, self.b, self.t = w, binding, torch
+        dt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+        self.Q, self.K, self.V = (torch.from_numpy(getattr(w, k)).cuda().to(dt) for k in "QKV")
+        self.mask = torch.from_numpy(w.mask).cuda(); self.U = torch.from_numpy(w.U).cuda()
+        self.gain = torch.from_numpy(w.gain).cuda(); self.cu = torch.from_numpy(w.cu_seqlens).cuda()
+        varlen = w.fixed_len is None
+        self.shp = binding.make_shape(batch=w.batch, max_seqlen=w.max_seqlen, n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads,
+                                      head_dim=w.head_dim, rank=w.rank, n_experts=w.n_experts, dtype=dt,
+                                      total_tokens=w.total_tokens if varlen else 0, cu_seqlens=self.cu if varlen else None)
+        self.ws = binding.new_workspace(self.shp)
+        self.O = torch.empty_like(self.Q)
+        self.sigma = None if w.sigma is None else torch.from_numpy(w.sigma).cuda()
+        self.alpha = None
+        if w.n_experts > 1:
+            self.alpha = torch.empty((w.batch, w.n_kv_heads, w.n_experts), device="cuda")
+            binding.adaseka_route(self.shp, self.Q, self.U, self.sigma, 0, self.alpha)
+        self.Kscratch = None
+
+    def fused(self):
+        self.b.seka_attention_fwd(self.shp, self.Q, self.K, self.V, self.O, None, self.mask, self.U, self.alpha, self.gain, None, self.ws)
+
+    def plain(self):
+        self.b.seka_attention_fwd(self.shp, self.Q, self.K, self.V, self.O, None, None, None, None, self.gain, None, self.ws)
+
+    def unfused(self):
+        """The hook as the paper runs it: edited keys written to a scratch tensor, then plain attention over it."""
+        if self.Kscratch is None:
+            self.Kscratch = self.t.empty_like(self.K)
+        self.b.seka_edit_keys(self.shp, self.K, self.Kscratch, self.mask, self.U, self.alpha, self.gain, None, self.ws)
+        self.b.seka_attention_fwd(self.shp, self.Q, self.Kscratch, self.V, self.O, None, None, None, None, self.gain, None, self.ws)
+
+    def routed(self):
+        a = self.t.empty_like(self.alpha)
+        self.b.seka_attention_fwd_routed(self.shp, self.Q, self.K, self.V, self.O, None, self.mask, self.U, self.sigma, 0, a,
+                                         self.gain, None, self.ws)
+
+    def two_call(self):
+        a = self.t.empty_like(self.alpha)
+        self.b.adaseka_route(self.shp, self.Q, self.U, self.sigma, 0, a)
+        self.b.seka_attention_fwd(self.shp, self.Q, self.K, self.V, self.O, None, self.mask, self.U, a, self.gain, None, self.ws)
+
+
+def interleaved_ms(fns, rounds: int, block: int = 1):
+    """Mean milliseconds per call of each function: `rounds` rounds, each running `block` calls of every function in
+    turn between its own pair of events (block = 1: single steps alternate; larger: homogeneous blocks, ABAB)."""
+    import torch
+    for f in fns:
+        for _ in range(2):
+            f()
+    torch.cuda.synchronize()
+    n = len(fns)
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(rounds * n + 1)]
+    evs[0].record()
+    for r in range(rounds):
+        for i, f in enumerate(fns):
+            for _ in range(block):
+                f()
+            evs[r * n + i + 1].record()
+    torch.cuda.synchronize()
+    return [sum(evs[r * n + i].elapsed_time(evs[r * n + i + 1]) for r in range(rounds)) / (rounds * block) for i in range(n)]
+
+
+def config_table(peaks, names=("C1", "C3", "C4", "C5", "C2s70", "C2s100"), oracle_rows: int = 6):
+    """The other configurations and the stress masks: time per step with steering, without (the same kernel, g = 0
+    path) and for the unfused route (stand-alone edit into a scratch tensor + plain attention), single steps
+    alternating and in homogeneous blocks of 20, plus the error of a handful of complete query rows against the oracle."""
+    import torch
+    import oracle
+    from paper_2603_01281_b200 import inputs
+    out = {}
+    for name in names:
+        w = inputs.make_workload(name)
+        r = FusedRunner(w)
+        flops = w.attention_flops()
+        big = flops > 2e12
+        rounds = 6 if big else 20
+        fns = [r.plain, r.fused, r.unfused] if w.dtype == "bf16" else [r.plain, r.fused]
+        alt = interleaved_ms(fns, rounds, 1)
+        blk = interleaved_ms(fns, 2 if big else 3, 5 if big else 20)
+        row = {"ms_g0": alt[0], "ms_steered": alt[1], "overhead_vs_g0": alt[1] / alt[0] - 1.0,
+               "overhead_vs_g0_blocks": blk[1] / blk[0] - 1.0,
+               "TFLOP/s": flops / (alt[1] * 1e-3) / 1e12, "TFLOP/s_g0": flops / (alt[0] * 1e-3) / 1e12,
+               "tokens_per_s": w.total_tokens / (alt[1] * 1e-3),
+               "frac_of_burst": flops / (alt[1] * 1e-3) / 1e12 / peaks["bf16_burst"]}
+        if len(fns) == 3:
+            row["ms_unfused"] = alt[2]; row["unfused_vs_g0"] = alt[2] / alt[0] - 1.0
+            row["unfused_vs_g0_blocks"] = blk[2] / blk[0] - 1.0
+        if name == "C3":
+            rt = interleaved_ms([r.routed, r.two_call, r.fused], rounds, 1)
+            row["routed"] = {"ms_one_call": rt[0], "ms_route_then_forward": rt[1], "ms_alpha_given": rt[2]}
+        # a handful of complete query rows per sequence (of at most four sequences) against the oracle
+        rng = np.random.default_rng(5)
+        rows = []
+        for b in range(w.batch):
+            Lb = int(w.cu_seqlens[b + 1] - w.cu_seqlens[b])
+            take = b < 4 and Lb > 0
+            rows.append(np.sort(rng.choice(Lb, size=min(oracle_rows, Lb), replace=False)).astype(np.int32) if take
+                        else np.zeros(0, dtype=np.int32))
+        r.fused(); torch.cuda.synchronize()
+        alpha = None if r.alpha is None else r.alpha.cpu().numpy().astype(np.float64)
+        Oref, _, idx = oracle.seka_attention(w.Q, w.K, w.V, w.mask, w.cu_seqlens, w.U, alpha=alpha, gain=w.gain, rows=rows)
+        err = np.abs(r.O.double().cpu().numpy()[idx] - Oref)
+        row["max_abs_err"] = float(err.max()); row["mean_abs_err"] = float(err.mean()); row["oracle_rows"] = int(len(idx))
+        st = r.b.seka_poll_status(r.ws)
+        row["status"] = r.b.status_string(st)
+        out[name] = row
+        del r
+        torch.cuda.empty_cache()
+    return out
+
+
 def run_reference(args, rank: int):
     """The reference arm: the CPU oracle on a bounded sample of the same workload, K timed steps."""
     if rank != 0:
@@ -260,6 +398,7 @@ def main():
     ap.add_argument("--learn-tokens", type=int, default=32768, help="tokens per embedding tensor in the learning measurement")
     ap.add_argument("--no-learn-bench", action="store_true", help="skip the offline spectral-learning measurement")
     ap.add_argument("--no-decode-bench", action="store_true", help="skip the decode-over-edited-cache measurement")
+    ap.add_argument("--no-config-table", action="store_true", help="skip the other configurations and stress masks")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -326,20 +465,19 @@ def main():
     if st != binding.SEKA_OK:
         raise SystemExit("device status: " + binding.status_string(st))
 
-    # the same kernel with steering off (g = 0 path): single steps of either kind alternate, each between its own
-    # pair of events, so that clock and temperature drift under the power cap falls on both alike
-    for _ in range(3):
-        step(False)
+    # The same kernel with steering off (g = 0 path), and the unfused route (stand-alone edit into a scratch key tensor,
+    # then the g = 0 kernel over it): single steps of the three kinds alternate, each between its own pair of events, so
+    # that clock and temperature drift under the power cap falls on all alike; then homogeneous blocks of 20, ABCABC.
+    Kscratch = torch.empty_like(dev["K"])
+
+    def step_unfused():
+        binding.seka_edit_keys(shp, dev["K"], Kscratch, mask, U, None, gain, None, ws)
+        binding.seka_attention_fwd(shp, dev["Q"], Kscratch, dev["V"], O, None, None, None, None, gain, None, ws)
     n_alt = max(10, min(args.steps, 100))
-    evs = [torch.cuda.Event(enable_timing=True) for _ in range(2 * n_alt + 1)]
     barrier()
-    evs[0].record()
-    for i in range(n_alt):
-        step(False); evs[2 * i + 1].record()
-        step(True); evs[2 * i + 2].record()
+    ms0, ms1, ms2 = interleaved_ms([lambda: step(False), lambda: step(True), step_unfused], n_alt, 1)
+    blk0, blk1, blk2 = interleaved_ms([lambda: step(False), lambda: step(True), step_unfused], 3, 20)
     barrier()
-    ms0 = sum(evs[2 * i].elapsed_time(evs[2 * i + 1]) for i in range(n_alt)) / n_alt * args.steps
-    ms1 = sum(evs[2 * i + 1].elapsed_time(evs[2 * i + 2]) for i in range(n_alt)) / n_alt * args.steps
 
     # end to end through the host-buffer entry point: H2D of Q, K, V, mask and D2H of O every step
     staging = torch.empty(binding.seka_host_staging_bytes(shp), dtype=torch.uint8, device="cuda")
@@ -368,6 +506,11 @@ def main():
     decode_res = None
     if rank == 0 and world == 1 and not args.no_decode_bench:
         decode_res = decode_bench(w, measured_peaks())
+    table_res = None
+    if rank == 0 and world == 1 and not args.no_config_table:
+        del Kscratch, staging
+        torch.cuda.empty_cache()
+        table_res = config_table(measured_peaks())
 
     if rank == 0:
         peaks = measured_peaks()
@@ -387,11 +530,19 @@ def main():
             "gpu_launches": int(launches),
             "roofline": {"bound": "tensor", "achieved": per_gpu, "peak": peaks["bf16_burst"], "unit": "TFLOP/s",
                          "frac": per_gpu / peaks["bf16_burst"], "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
-                         "peak_source": "of %s (cuBLAS bf16 burst); sustained %.1f -> %.3f, nominal 2250 -> %.3f" % (
-                             peaks["source"], peaks["bf16_sustained"], per_gpu / peaks["bf16_sustained"], per_gpu / 2250.0)},
+                         "tensor_pipe_active_pct": NCU_TENSOR_PIPE_ACTIVE_PCT,
+                         "frac_of_sustained": per_gpu / peaks["bf16_sustained"], "frac_of_nominal": per_gpu / NOMINAL_BF16_TFLOPS,
+                         "peak_source": "of %s (cuBLAS bf16 burst %.1f; sustained %.1f; nominal dense bf16 %.0f)" % (
+                             peaks["source"], peaks["bf16_burst"], peaks["bf16_sustained"], NOMINAL_BF16_TFLOPS)},
             "extra": {"tokens_per_s": world * tokens_step * args.steps / (ms * 1e-3),
-                      "ms_per_step_g0": ms0 / args.steps, "ms_per_step_steered": ms1 / args.steps,
-                      "overhead_vs_g0": ms1 / ms0 - 1.0, "flops_per_step": flops_step},
+                      "ms_per_step_g0": ms0, "ms_per_step_steered": ms1, "overhead_vs_g0": ms1 / ms0 - 1.0,
+                      "overhead_vs_g0_blocks": blk1 / blk0 - 1.0,
+                      "TFLOP/s_g0": flops_step / (ms0 * 1e-3) / 1e12,
+                      "frac_of_burst_g0": flops_step / (ms0 * 1e-3) / 1e12 / peaks["bf16_burst"],
+                      "unfused": {"what": "seka_edit_keys into a scratch key tensor, then the g = 0 kernel over it",
+                                  "ms_per_step": ms2, "vs_g0": ms2 / ms0 - 1.0, "vs_g0_blocks": blk2 / blk0 - 1.0,
+                                  "fused_over_unfused": ms1 / ms2},
+                      "flops_per_step": flops_step},
         }
         if edit_res is not None:
             line["extra"]["edit_keys"] = edit_res
@@ -399,11 +550,14 @@ def main():
             line["extra"]["decode"] = decode_res
         if learn_res is not None:
             line["extra"]["learn"] = learn_res
+        if table_res is not None:
+            line["extra"]["configs"] = table_res
         if world == 1 and not args.no_cpu_baseline:
             import oracle
             f, s, r = cpu_oracle_sample(w, args.cpu_budget)
             line["cpu_baseline"] = {"value": f / s / 1e12, "unit": "TFLOP/s", "cores": oracle.threads(), "kind": "oracle",
-                                    "sample": "%d random complete query rows (all 32 heads) of the same workload, %.1f s" % (r, s)}
+                                    "sample": "%d random complete query rows (all 32 heads) of the same workload, %.1f s" % (r, s),
+                                    "c1_single_thread": oracle_c1_single_thread()}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

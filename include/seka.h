@@ -11,7 +11,11 @@
  *
  * Conventions shared by every entry point
  *  - Pointers are DEVICE pointers unless the name starts with `h_`. The caller owns
- *    every buffer; the library keeps none and allocates none.
+ *    every buffer; the library keeps none and allocates no device memory.  Process state it
+ *    does keep: the launch counter of seka_launch_count (atomic), the SM count of each
+ *    device it has been called on, the driver entry point for tensor maps, and the
+ *    per-device address of the built-in scratch of seka_edit_keys_static (all behind
+ *    mutexes; calls may come from several host threads and for several devices).
  *  - Tensors are packed token-major: Q [T, Hq, d], K and V [T, Hkv, d], O [T, Hq, d],
  *    mask [T] (non-zero = highlighted), T = total_tokens, rows contiguous, base
  *    pointers 16-byte aligned.  Sequence b owns tokens cu_seqlens[b] .. cu_seqlens[b+1]-1;
@@ -96,7 +100,13 @@ seka_status adaseka_route(const seka_shape* shape, const void* Q, const float* U
 /*
  * Fused steered attention (Algorithm 1/2 hook + the attention it feeds, Eq. 4-5 in the
  * single-projector form): O = softmax_causal(Q K'^T * scale) V with K' the edited keys;
- * K' and the score matrix are never written to memory, K and V are not modified.
+ * the score matrix is never written to memory, K and V are not modified.  The edited
+ * keys of the 128-token key tiles that hold a highlighted token (and of no others) are
+ * formed once per call, in fp32, by a preparation launch into `workspace` as a high and
+ * a low bf16 part; the attention kernel stages those tiles from there instead of from K
+ * and adds the contraction with the low parts where it matters (gain x coefficient above
+ * 1 in magnitude, and every query row that sees at most 1024 keys), so the logits follow
+ * the fp32 edited keys there and one bf16 rounding of them elsewhere.
  * O has the dtype of the inputs.  With dtype SEKA_F32 the inputs are rounded to bf16
  * on the way in (the contraction runs on bf16 tensor cores, fp32 accumulation).
  * lse, if not NULL, receives log sum_j exp(score_ij) as fp32 [T, Hq].
@@ -126,9 +136,12 @@ seka_status seka_attention_fwd_routed(const seka_shape* shape, const void* Q, co
  * Same computation as seka_attention_fwd for callers whose tensors live in HOST memory
  * (pinned memory makes the copies asynchronous): h_Q, h_K, h_V, h_mask are copied to
  * `staging` (device, seka_host_staging_bytes(shape) bytes, 256-byte aligned), the
- * fused kernel runs, and O (and lse if h_lse != NULL) is copied back to h_O, all on
- * `cuda_stream`.  U, alpha, gain, head_enable stay device pointers (they are per-model
- * or per-prompt constants).
+ * fused kernel runs, and O (and lse if h_lse != NULL) is copied back to h_O.  The result
+ * is complete when the work queued on `cuda_stream` is.  A fixed-length batch is cut by
+ * sequence into up to eight parts that are copied in, computed and copied out as a
+ * pipeline (the call creates two more streams and a few events for its duration and
+ * releases them before it returns); a packed batch goes through in one piece.  U, alpha,
+ * gain, head_enable stay device pointers (they are per-model or per-prompt constants).
  */
 size_t seka_host_staging_bytes(const seka_shape* shape);
 seka_status seka_attention_fwd_host(const seka_shape* shape, const void* h_Q, const void* h_K,
@@ -147,13 +160,17 @@ seka_status seka_attention_fwd_host(const seka_shape* shape, const void* h_Q, co
  * start-up, a plug-in that runs inside another framework's stream callback, or code that has
  * already frozen its allocator.  seka_edit_keys needs a scratch buffer (the compacted list of
  * highlighted tokens) that such a caller has nowhere to get.  This variant keeps that scratch in
- * a fixed array inside the library's device image instead; it computes exactly what
- * seka_edit_keys computes and takes the same tensors, minus the workspace.
+ * a fixed array inside the library's device image instead; it takes the same tensors, minus
+ * the workspace, and computes the same edit: in fp32 arithmetic with one rounding to the
+ * tensor's type (for bf16 tensors seka_edit_keys uses a tensor-core kernel whose result can
+ * differ from this one in the last bf16 place).
  *
  *  - Limit: total tokens <= SEKA_STATIC_MAX_TOKENS.  A larger shape is refused with
  *    SEKA_ERR_UNSUPPORTED before anything is launched; use seka_edit_keys with a workspace there.
  *  - Cost: every GPU that loads the library holds the array (4 * SEKA_STATIC_MAX_TOKENS + 256
- *    bytes) until the process exits, whether or not this entry point is ever called.
+ *    bytes) until the process exits, whether or not this entry point is ever called.  The
+ *    kernel behind it (a warp per highlighted token, plain multiply-adds) is several times
+ *    slower on large caches than the pipelined kernel of seka_edit_keys.
  *  - The call itself performs no cudaMalloc / cudaFree and uses no allocating library routine.
  *    The first call on each device looks up the array's device address (once, with that device
  *    current); make that first call outside any stream capture.
@@ -218,7 +235,14 @@ seka_status seka_learn_projections(const seka_learn_shape* shape, const void* h,
                                    float* S_pos, float* S_neg, int32_t* k_pos, int32_t* k_neg, float* D,
                                    void* workspace, size_t workspace_bytes, void* cuda_stream);
 
-/* Clears the device status word (async on the stream); call once before first use of a workspace. */
+/*
+ * The first 256 bytes of a workspace are its status block (int32 words): word 0 the status, word 1 a code for the
+ * wait that gave up.  Two more words are read by the fused forward and are there for tests of the failure path:
+ * word 4 (non-zero n: CTA 0 leaves out the load of the n-th V/K pair of its first work item, so that a wait runs out)
+ * and word 5 (limit of every device-side wait of that launch in microseconds; 0 means 2 s).  A launch on a workspace
+ * whose status is not SEKA_OK does nothing.
+ * seka_reset_status clears the whole block (async on the stream); call it once before first use of a workspace.
+ */
 seka_status seka_reset_status(void* workspace, void* cuda_stream);
 /* Synchronises the stream and returns the device status word (SEKA_OK if no wait ran out). */
 seka_status seka_poll_status(const void* workspace, void* cuda_stream);

@@ -61,6 +61,7 @@ constexpr int REGS_CTRL = 80, REGS_SOFTMAX = 184, REGS_PROJ = 64;   // PROJ: the
 constexpr uint32_t POLY_PAIR_MASK = SEKA_POLY_PAIR_MASK;
 constexpr uint32_t SMEM_LIMIT = 227 * 1024;
 
+
 // Shared memory of one CTA.  Tiles first (each a multiple of 1024 bytes), then barriers and per-warp item slots.
 template <int D>
 struct Geo {
@@ -68,10 +69,14 @@ struct Geo {
     static constexpr uint32_t TILE = (D / 64) * BLK_BYTES;         // a [128 x D] tile
     static constexpr int NXMAX = 3;                                // most stages of the key-side operand
     static constexpr uint32_t NBARS = 14 + 2 * NK + NXMAX;
+    // shared-memory copy of the per-(sequence, KV head) steering bytes and the per-sequence first highlighted tile
+    // (what fits beside the tiles; larger batches look them up in global memory)
+    static constexpr int INFO_HEADS = D == 128 ? 768 : 4096, INFO_SEQS = D == 128 ? 64 : 512;
+    static constexpr uint32_t INFO_BYTES = INFO_HEADS + INFO_SEQS * 4;
 };
 
 struct SmemPlan {
-    uint32_t k, v, x, xb, bars, misc, items, total;
+    uint32_t k, v, x, xb, bars, misc, items, info, total;
 };
 
 template <int D>
@@ -85,7 +90,8 @@ __host__ __device__ inline SmemPlan smem_plan(const SteerPlan& sp) {
     s.bars = s.x + (uint32_t)sp.nx * s.xb;
     s.misc = s.bars + ((G::NBARS * 8 + 15) & ~15u);                 // 16-byte aligned: the item slots are filled by 16-byte async copies
     s.items = s.misc + 32;
-    s.total = s.items + 16 * 32;
+    s.info = s.items + 16 * 32;                                     // steering info of every (sequence, KV head), if it fits
+    s.total = s.info + (sp.mode ? G::INFO_BYTES : 0u);
     return s;
 }
 
@@ -186,6 +192,10 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     const bool dead = __syncthreads_or(*reinterpret_cast<volatile int*>(p.status) != 0);
     const int hook_skip = p.status[4];
     const uint64_t limit_ns = p.status[5] > 0 ? (uint64_t)p.status[5] * 1000ull : kWaitLimitNs;
+    // steering info is kept in shared memory when it fits (a look-up per work item then costs no trip to the caches)
+    const bool info_local = p.steer && p.sched.B * p.sched.Hkv <= G::INFO_HEADS && p.sched.B <= G::INFO_SEQS;
+    uint8_t* info_bh = smem + sl.info;
+    int* info_first = reinterpret_cast<int*>(smem + sl.info + G::INFO_HEADS);
 
     // all lanes of a warp wait on the same barrier and then agree on the outcome
     auto warp_wait = [&](uint64_t* bar, uint32_t parity, int where) -> bool {
@@ -216,7 +226,8 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         }
     };
     prefetch();
-    auto next_item = [&](Item& it) -> bool {
+    // `steering`: also look up whether the item's keys are edited (only the producer and the MMA issuer need to know)
+    auto next_item = [&](Item& it, bool steering = false) -> bool {
         ItemRecord rec;
         if (TABLE) {
             if (idx_next < 0) return false;
@@ -234,15 +245,15 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             if (idx < 0) return false;
             decode_item(p.sched, idx, nullptr, rec);
             const int b = rec.bh & 0xffff, hkv = rec.bh >> 16;
-            rec.steer = p.steer ? (int)__ldg(p.bh_info + b * p.sched.Hkv + hkv) : 0;      // one cache line for a whole batch
+            rec.steer = (steering && p.steer) ? (int)(info_local ? info_bh[b * p.sched.Hkv + hkv] : __ldg(p.bh_info + b * p.sched.Hkv + hkv)) : 0;
         }
         it.seq0 = rec.seq0; it.Lb = rec.Lb; it.b = rec.bh & 0xffff; it.hkv = rec.bh >> 16;
         it.hqA = rec.hq & 0xffff; it.hqB = rec.hq >> 16;
         it.qtA = rec.qt & 0xffff; it.qtB = rec.qt >> 16;
         it.nA = rec.n & 0xffff; it.nB = rec.n >> 16;
         it.n_kv = max(it.nA, it.nB);
-        it.steer = (rec.steer & 1) != 0 && p.plan.mode != 0;
-        it.hot_any = it.steer && p.first_hot[it.b] < it.n_kv;
+        it.steer = steering && (rec.steer & 1) != 0 && p.plan.mode != 0;
+        it.hot_any = it.steer && (info_local ? info_first[it.b] : __ldg(p.first_hot + it.b)) < it.n_kv;
         it.need_lo = it.hot_any && ((rec.steer & 2) != 0 || it.n_kv <= kLoTiles);
         return true;
     };
@@ -263,6 +274,11 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     }
     __syncwarp();
     if (warp == 0) { tmem_alloc(tmem_holder, TMEM_COLS); tmem_relinquish(); }
+    // steering info into shared memory
+    if (info_local) {
+        for (int i = tid; i < p.sched.B * p.sched.Hkv; i += NTHREADS) info_bh[i] = p.bh_info[i];
+        for (int i = tid; i < p.sched.B; i += NTHREADS) info_first[i] = p.first_hot[i];
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -321,7 +337,7 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     if ((int)st == i) armed_x[i] = ((n_hot / (uint32_t)nx) & 1) + 1;
                 ++n_hot;
             };
-            while (ok && next_item(it)) {
+            while (ok && next_item(it, true)) {
                 const uint8_t* hot_g = p.tile_hot + (size_t)it.b * p.sched.n_qt;
                 // Q and the first K of an item may land once the last score product of the previous item is
                 // done (event n_kv - 1 of that item), its V/K pairs once its last step is done (event n_kv)
@@ -425,7 +441,7 @@ seka_attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                 if (leader) umma_commit(bar);
                 __syncwarp();
             };
-            while (ok && next_item(it)) {
+            while (ok && next_item(it, true)) {
                 const uint8_t* hot_g = p.tile_hot + (size_t)it.b * p.sched.n_qt;
                 const int nA = it.nA, nB = it.nB, n_kv = it.n_kv;
                 uint32_t x_stage = 0;      // stage that holds the low parts of the key tile being multiplied
@@ -890,23 +906,73 @@ extern "C" seka_status seka_attention_fwd_host(const seka_shape* shape, const vo
     if (!staging || staging_bytes < seka_host_staging_bytes(shape) || ((uintptr_t)staging & 255)) return SEKA_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const size_t esz = shape->dtype == SEKA_F32 ? 4 : 2;
-    const size_t bq = T * shape->n_q_heads * shape->head_dim * esz, bk = T * shape->n_kv_heads * shape->head_dim * esz;
+    const size_t rq = (size_t)shape->n_q_heads * shape->head_dim * esz, rk = (size_t)shape->n_kv_heads * shape->head_dim * esz;
+    const size_t bq = T * rq, bk = T * rk;
     char* dq = static_cast<char*>(staging);
     char* dk = dq + align_up(bq, 256);
     char* dv = dk + align_up(bk, 256);
     char* dO = dv + align_up(bk, 256);
     char* dm = dO + align_up(bq, 256);
     char* dl = dm + align_up(T, 256);
-    bool okc = cudaMemcpyAsync(dq, h_Q, bq, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    okc = okc && cudaMemcpyAsync(dk, h_K, bk, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    okc = okc && cudaMemcpyAsync(dv, h_V, bk, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    if (h_mask) okc = okc && cudaMemcpyAsync(dm, h_mask, T, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    if (!okc) return SEKA_ERR_CUDA;
-    stc = seka_attention_fwd(shape, dq, dk, dv, dO, h_lse ? reinterpret_cast<float*>(dl) : nullptr,
-                             h_mask ? reinterpret_cast<const uint8_t*>(dm) : nullptr, U, alpha, gain, head_enable,
-                             workspace, workspace_bytes, cuda_stream);
+    // Sequences are independent, so a fixed-length batch is cut into parts (one sequence each, at most eight) that go
+    // through a three-stage pipeline: the inputs of part i + 1 are copied in (a second stream) while part i is computed
+    // (the caller's stream) and the output of part i - 1 is copied out (a third stream); the two copy directions share
+    // the link at full duplex.  A packed batch (cu_seqlens) runs as one part.
+    int parts = 1;
+    if (shape->cu_seqlens == nullptr && shape->batch > 1) {
+        parts = shape->batch < 8 ? shape->batch : 8;
+        while (shape->batch % parts) --parts;
+    }
+    const int seq_per = shape->batch / parts;
+    const size_t tok_per = (size_t)seq_per * shape->max_seqlen;
+    cudaStream_t s_in = nullptr, s_out = nullptr;
+    cudaEvent_t ev_start = nullptr, ev_in[8] = {}, ev_cmp[8] = {}, ev_out = nullptr;
+    bool okc = true;
+    auto make_event = [&](cudaEvent_t* e) { okc = okc && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess; };
+    if (parts > 1) {
+        okc = okc && cudaStreamCreateWithFlags(&s_in, cudaStreamNonBlocking) == cudaSuccess;
+        okc = okc && cudaStreamCreateWithFlags(&s_out, cudaStreamNonBlocking) == cudaSuccess;
+        make_event(&ev_start); make_event(&ev_out);
+        for (int i = 0; i < parts; ++i) { make_event(&ev_in[i]); make_event(&ev_cmp[i]); }
+        // the copies start after whatever the caller queued before this call
+        okc = okc && cudaEventRecord(ev_start, st) == cudaSuccess && cudaStreamWaitEvent(s_in, ev_start, 0) == cudaSuccess &&
+              cudaStreamWaitEvent(s_out, ev_start, 0) == cudaSuccess;
+    } else {
+        s_in = st; s_out = st;
+    }
+    seka_shape part = *shape;
+    part.batch = seq_per;
+    part.total_tokens = shape->cu_seqlens ? shape->total_tokens : 0;
+    for (int i = 0; i < parts && okc && stc == SEKA_OK; ++i) {
+        const size_t t0 = (size_t)i * tok_per, nt = parts > 1 ? tok_per : T;
+        okc = okc && cudaMemcpyAsync(dq + t0 * rq, static_cast<const char*>(h_Q) + t0 * rq, nt * rq, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
+        okc = okc && cudaMemcpyAsync(dk + t0 * rk, static_cast<const char*>(h_K) + t0 * rk, nt * rk, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
+        okc = okc && cudaMemcpyAsync(dv + t0 * rk, static_cast<const char*>(h_V) + t0 * rk, nt * rk, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
+        if (h_mask) okc = okc && cudaMemcpyAsync(dm + t0, h_mask + t0, nt, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
+        if (parts > 1) okc = okc && cudaEventRecord(ev_in[i], s_in) == cudaSuccess && cudaStreamWaitEvent(st, ev_in[i], 0) == cudaSuccess;
+        if (!okc) break;
+        stc = seka_attention_fwd(&part, dq + t0 * rq, dk + t0 * rk, dv + t0 * rk, dO + t0 * rq,
+                                 h_lse ? reinterpret_cast<float*>(dl) + t0 * shape->n_q_heads : nullptr,
+                                 h_mask ? reinterpret_cast<const uint8_t*>(dm) + t0 : nullptr, U,
+                                 alpha ? alpha + (size_t)i * seq_per * shape->n_kv_heads * shape->n_experts : nullptr,
+                                 gain ? gain + (size_t)i * seq_per : nullptr, head_enable, workspace, workspace_bytes, cuda_stream);
+        if (stc != SEKA_OK) break;
+        if (parts > 1) okc = okc && cudaEventRecord(ev_cmp[i], st) == cudaSuccess && cudaStreamWaitEvent(s_out, ev_cmp[i], 0) == cudaSuccess;
+        okc = okc && cudaMemcpyAsync(static_cast<char*>(h_O) + t0 * rq, dO + t0 * rq, nt * rq, cudaMemcpyDeviceToHost, s_out) == cudaSuccess;
+        if (h_lse) okc = okc && cudaMemcpyAsync(h_lse + t0 * shape->n_q_heads, reinterpret_cast<float*>(dl) + t0 * shape->n_q_heads,
+                                                nt * shape->n_q_heads * 4, cudaMemcpyDeviceToHost, s_out) == cudaSuccess;
+    }
+    if (parts > 1) {
+        // the caller's stream ends behind the last copy out (and behind the copies in, if the loop stopped early)
+        if (ev_out && s_out) { cudaEventRecord(ev_out, s_out); cudaStreamWaitEvent(st, ev_out, 0); }
+        if (ev_start && s_in) { cudaEventRecord(ev_start, s_in); cudaStreamWaitEvent(st, ev_start, 0); }
+        // queued work keeps what it needs: destroying a stream or an event only drops the handle
+        for (int i = 0; i < parts; ++i) { if (ev_in[i]) cudaEventDestroy(ev_in[i]); if (ev_cmp[i]) cudaEventDestroy(ev_cmp[i]); }
+        if (ev_start) cudaEventDestroy(ev_start);
+        if (ev_out) cudaEventDestroy(ev_out);
+        if (s_in) cudaStreamDestroy(s_in);
+        if (s_out) cudaStreamDestroy(s_out);
+    }
     if (stc != SEKA_OK) return stc;
-    okc = cudaMemcpyAsync(h_O, dO, bq, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-    if (h_lse) okc = okc && cudaMemcpyAsync(h_lse, dl, T * shape->n_q_heads * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
     return okc ? SEKA_OK : SEKA_ERR_CUDA;
 }

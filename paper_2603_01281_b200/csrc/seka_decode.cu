@@ -348,12 +348,10 @@ seka_status validate_decode(const seka_shape* s) {
 template <int D, bool HALF>
 seka_status launch_split(const CUtensorMap& tk, const CUtensorMap& tv, const DecodeParams& p, cudaStream_t st) {
     using SL = DecSmem<D>;
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(decode_split_kernel<D, HALF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)SL::DYN_BYTES) != cudaSuccess) return SEKA_ERR_CUDA;
-        configured = true;
-    }
+    // the attribute belongs to the function on the current device: set on every call (a cheap driver call), so that
+    // several devices or host threads need no bookkeeping here
+    if (cudaFuncSetAttribute(decode_split_kernel<D, HALF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)SL::DYN_BYTES) != cudaSuccess) return SEKA_ERR_CUDA;
     dim3 grid((unsigned)p.n_splits, (unsigned)p.Hkv, (unsigned)p.B);
     decode_split_kernel<D, HALF><<<grid, DEC_THREADS, SL::DYN_BYTES, st>>>(tk, tv, p);
     ++g_launches;

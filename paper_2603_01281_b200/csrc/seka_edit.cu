@@ -538,16 +538,11 @@ static seka_status launch_edit_tiles(const seka_shape* s, const WorkspaceLayout&
                                      const uint8_t* mask, const float* U, const float* alpha, const float* gain,
                                      const uint8_t* he, char* ws, cudaStream_t st) {
     using SL = EditSmem<D>;
-    static bool configured = false;
-    static int n_sm = 0;
-    if (!configured) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm <= 0) return SEKA_ERR_CUDA;
-        if (cudaFuncSetAttribute(edit_tiles_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SL::DYN_BYTES) != cudaSuccess)
-            return SEKA_ERR_CUDA;
-        configured = true;
-    }
+    // per-device facts: looked up per device; function attributes set on every call (they belong to the current device)
+    int n_sm = 0;
+    if (!device_info(&n_sm)) return SEKA_ERR_CUDA;
+    if (cudaFuncSetAttribute(edit_tiles_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SL::DYN_BYTES) != cudaSuccess)
+        return SEKA_ERR_CUDA;
     int* status = reinterpret_cast<int*>(ws);
     void* P = ws + w.w_off;
     uint8_t* tile_hot = reinterpret_cast<uint8_t*>(ws + w.hot_off);
@@ -558,12 +553,8 @@ static seka_status launch_edit_tiles(const seka_shape* s, const WorkspaceLayout&
     if (!make_tile_map(&tk, K_in, D, Hkv, T) || !make_tile_map(&tp, P, D, 1, (long long)2 * M * Hkv * D, D)) return SEKA_ERR_CUDA;
     if (M == 1) {
         using PL = EpSmem<D>;
-        static bool configured_p = false;
-        if (!configured_p) {
-            if (cudaFuncSetAttribute(edit_tiles_pipe_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PL::DYN_BYTES) != cudaSuccess)
-                return SEKA_ERR_CUDA;
-            configured_p = true;
-        }
+        if (cudaFuncSetAttribute(edit_tiles_pipe_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PL::DYN_BYTES) != cudaSuccess)
+            return SEKA_ERR_CUDA;
         const long long work = (long long)s->batch * w.n_tiles * Hkv;
         const unsigned gridp = (unsigned)(work < (long long)n_sm ? work : (long long)n_sm);
         edit_tiles_pipe_kernel<D><<<gridp, EP_THREADS, PL::DYN_BYTES, st>>>(tk, tp, static_cast<__nv_bfloat16*>(K_out), mask, alpha, gain, he,

@@ -584,18 +584,13 @@ extern "C" seka_status seka_learn_projections(const seka_learn_shape* shape, con
     char* ws = static_cast<char*>(workspace);
     const int d = shape->head_dim, slots = shape->n_slots, n = shape->n_tokens;
 
-    static bool configured = false;
-    static int n_sm = 0;
-    if (!configured) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm <= 0) return SEKA_ERR_CUDA;
-        if (cudaFuncSetAttribute(learn_cov_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LC_DYN_BYTES) != cudaSuccess ||
-            cudaFuncSetAttribute(learn_svd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)(sizeof(double) * (128 * (128 + SV_PAD) + 128) + sizeof(int) * 128)) != cudaSuccess)
-            return SEKA_ERR_CUDA;
-        configured = true;
-    }
+    // per-device facts: looked up per device; function attributes set on every call (they belong to the current device)
+    int n_sm = 0;
+    if (!device_info(&n_sm)) return SEKA_ERR_CUDA;
+    if (cudaFuncSetAttribute(learn_cov_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LC_DYN_BYTES) != cudaSuccess ||
+        cudaFuncSetAttribute(learn_svd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)(sizeof(double) * (128 * (128 + SV_PAD) + 128) + sizeof(int) * 128)) != cudaSuccess)
+        return SEKA_ERR_CUDA;
 
     // cross-covariances: columns in groups of 128 (one head of 128, or two neighbouring heads of 64)
     CUtensorMap tmH, tmP, tmN;
