@@ -100,27 +100,29 @@ prep_steering_kernel(const __grid_constant__ CUtensorMap tmK, int* status, const
     const int kb = blockIdx.x - n_flag - n_a;
     const int h = kb % Hkv, slot = kb / Hkv, n_slots = n_x / Hkv;
     if (head_enable != nullptr && head_enable[h] == 0) return;
-    constexpr int NS = 2;
+    constexpr int NS = 1;                 // one key stage: two blocks share an SM instead of a block prefetching
     constexpr uint32_t TILE = (D / 64) * 128 * 128, PBLK = D * 128, PMAT = (D / 64) * PBLK;
     constexpr uint32_t TMEM_COLS = 2 * D;
     const int Rt = r * M;
     const bool routed = route.sigma != nullptr;
+    const bool tc_build = D == 128 && M == 1 && r <= 64;      // U U^T on the tensor core (see build_W_tc)
     // dynamic shared memory (1024-byte aligned): key stages | W high, low | a chunk of U^T | routing scratch and coefficients
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(prep_sm) + 1023) & ~uintptr_t(1023));
     uint8_t* sW = smem + NS * TILE;
     float* ut = reinterpret_cast<float*>(sW + 2 * PMAT);        // staged chunk of U^T: [32][D + 4]
-    unsigned char* tail = sW + 2 * PMAT + 32 * (D + 4) * 4;
+    unsigned char* tail = sW + 2 * PMAT + (tc_build ? 0 : 32 * (D + 4) * 4);       // (no chunk of U^T with the tensor-core build)
     float* alpha_s = reinterpret_cast<float*>(tail + (routed ? align_up_dev(route_smem_bytes(D, M, route.k_route), 16) : 0));
-    __shared__ __align__(8) uint64_t bars[NS + 2];
+    __shared__ __align__(8) uint64_t bars[NS + 3];
     __shared__ uint32_t tmem_holder;
     __shared__ int abort_s;
     __shared__ unsigned char row_hl[NS][128];
     uint64_t* full = bars;            // [NS] key tile landed
     uint64_t* done = bars + NS;       // [2]  K W of a tile is in column set c
+    uint64_t* built = bars + NS + 2;  // [1]  U U^T is in tensor memory
     volatile int* abort_flag = &abort_s;
     if (tid == 0) {
         for (int i = 0; i < NS; ++i) mbar_init(full + i, 1);
-        mbar_init(done + 0, 1); mbar_init(done + 1, 1);
+        mbar_init(done + 0, 1); mbar_init(done + 1, 1); mbar_init(built, 1);
         abort_s = 0;
         mbar_fence_init();
         tma_prefetch_desc(&tmK);
@@ -218,6 +220,78 @@ prep_steering_kernel(const __grid_constant__ CUtensorMap tmK, int* status, const
         fence_proxy_async();           // read next by the tensor core
     };
 
+    // One expert, rank <= 64, head_dim 128: W = U U^T on the tensor core.  U (two bf16 parts) is written into the space
+    // of W's low part (overwritten only after the product has finished) as two K-major operand tiles [128 x 64],
+    // columns beyond the rank zero up to the next multiple of 16; hi.hi + hi.lo + lo.hi accumulate in tensor memory (column set 0); every thread then
+    // reads half a row of the product, splits it and writes it where build_W would.
+    uint32_t n_build = 0;
+    auto build_W_tc = [&]() -> bool {
+        const int r16 = (r + 15) / 16 * 16;
+        uint8_t* t_hi = sW + PMAT;                  // [128 x 64] bf16, 128-byte swizzle: where the low part of W goes afterwards
+        uint8_t* t_lo = sW + PMAT + 128 * 128;
+        const float* Uh = U + (size_t)h * D * r;
+        for (int e0 = 0; e0 < D * r16; e0 += PREP_THREADS * 8) {
+            float v[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const int e = e0 + q * PREP_THREADS + tid, i = e / r16, kk = e - i * r16;
+                v[q] = (e < D * r16 && kk < r) ? __ldg(Uh + (size_t)i * r + kk) : 0.f;
+            }
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const int e = e0 + q * PREP_THREADS + tid, i = e / r16, kk = e - i * r16;
+                if (e < D * r16) {
+                    const __nv_bfloat16 hi = __float2bfloat16_rn(v[q]);
+                    const __nv_bfloat16 lo = __float2bfloat16_rn(v[q] - __bfloat162float(hi));
+                    const uint32_t off = sw128_offset(i, kk & ~7) + (kk & 7) * 2;
+                    *reinterpret_cast<__nv_bfloat16*>(t_hi + off) = hi;
+                    *reinterpret_cast<__nv_bfloat16*>(t_lo + off) = lo;
+                }
+            }
+        }
+        fence_proxy_async();
+        __syncthreads();
+        if (tid == 0) {
+            tc_fence_after();
+            const uint32_t dhi = umma_desc_lo(smem_u32(t_hi), 16), dlo = umma_desc_lo(smem_u32(t_lo), 16);
+            uint32_t acc = 0;
+            for (int ks = 0; ks < r16 / 16; ++ks) {
+                const uint32_t off = (uint32_t)(ks * 32) >> 4;
+                umma_ss(tmem_base, dhi + off, DESC_HI, dhi + off, DESC_HI, IDESC, acc); acc = 1;
+                umma_ss(tmem_base, dhi + off, DESC_HI, dlo + off, DESC_HI, IDESC, 1u);
+                umma_ss(tmem_base, dlo + off, DESC_HI, dhi + off, DESC_HI, IDESC, 1u);
+            }
+            umma_commit(built);
+        }
+        bool good = mbar_wait(built, n_build & 1, abort_flag, status, 72);
+        ++n_build;
+        good = __syncthreads_and(good);
+        if (!good) return false;
+        tc_fence_after();
+        const int row = tid & 127, half = tid >> 7;
+#pragma unroll 1
+        for (int cb = half * (D / 64); cb < (half + 1) * (D / 64); ++cb) {
+            uint32_t v[32];
+            tmem_ld32(t_lane + cb * 32, v);
+            tmem_wait_ld_on(v);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                uint32_t hi[4], lo[4];
+#pragma unroll
+                for (int e2 = 0; e2 < 4; ++e2)
+                    split_pair(__uint_as_float(v[q * 8 + 2 * e2]), __uint_as_float(v[q * 8 + 2 * e2 + 1]), hi[e2], lo[e2]);
+                const int col = cb * 32 + q * 8;
+                uint8_t* dst = sW + (col >> 6) * PBLK + sw128_offset(row, col & 63);
+                *reinterpret_cast<uint4*>(dst) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                *reinterpret_cast<uint4*>(dst + PMAT) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+            }
+        }
+        tc_fence_before();
+        fence_proxy_async();           // read next by the tensor core
+        __syncthreads();
+        return true;
+    };
+
     // The (sequence, tile) pairs that hold a highlighted token, HOT_CAP candidates at a time: every block finds them for
     // itself (eight lanes per pair, 16 mask bytes each), so that the walk below only meets tiles with work.
     __shared__ int hot_list[HOT_CAP];
@@ -288,8 +362,6 @@ prep_steering_kernel(const __grid_constant__ CUtensorMap tmK, int* status, const
 #pragma unroll
             for (int c = 0; c < D / 64; ++c) tma_load_3d(smem + st * TILE + c * (128 * 128), &tmK, full + st, c * 64, h, seq0 + t * 128);
         };
-        if (i0 < i1 && tid == 0) load_tile(i0);
-        if (i0 < i1) ++n_load;
         for (int i = i0; i < i1 && ok; ++i) {
             const int e = hot_list[i], b = e & 0xffff, t = e >> 16;
             const int seq0 = cu_seqlens ? cu_seqlens[b] : b * L;
@@ -298,15 +370,17 @@ prep_steering_kernel(const __grid_constant__ CUtensorMap tmK, int* status, const
             const uint32_t st = n_mma % NS, cs = n_mma & 1;
             // the operator for this tile (the previous tile is through: every iteration ends with a barrier)
             const int want = M == 1 ? -1 : b;
-            if (built_for != want) { build_W(want); built_for = want; }
-            // highlight flags of the tile's rows; the next tile starts to land meanwhile
+            // the key tile starts to land (the stage is free: the previous tile is through)
+            if (tid == 0) load_tile(i);
+            ++n_load;
+            if (built_for != want) {
+                if (tc_build) { ok = build_W_tc(); if (!ok) break; } else build_W(want);
+                built_for = want;
+            }
+            // the highlight flags of the tile's rows
             if (tid < 128) {
                 const int kpos = t * 128 + tid;
                 row_hl[st][tid] = (kpos < Lb && mask[seq0 + kpos] != 0) ? 1 : 0;
-            }
-            if (i + 1 < i1) {
-                if (tid == 0) load_tile(i + 1);
-                ++n_load;
             }
             __syncthreads();               // W and the flags are in place
             ok = mbar_wait(full + st, ((n_mma / NS) & 1), abort_flag, status, 70);
@@ -526,8 +600,9 @@ static size_t route_bytes_aligned(int D, int M, int k_route) { return align_up(r
 size_t prep_steering_smem(const seka_shape* sh, bool routed, int k_route) {
     const int D = sh->head_dim;
     const size_t tile = (size_t)(D / 64) * 128 * 128, pmat = (size_t)D * D * 2;
+    const bool tc_build = D == 128 && sh->n_experts == 1 && sh->rank <= 64;      // as in the kernel: no staged chunk of U^T
     const size_t route = routed ? route_bytes_aligned(D, sh->n_experts, k_route) + (size_t)ALPHA_CAP * 4 : 0;
-    return 1024 + 2 * tile + 2 * pmat + (size_t)32 * (D + 4) * 4 + route;
+    return 1024 + tile + 2 * pmat + (tc_build ? 0 : (size_t)32 * (D + 4) * 4) + route;
 }
 
 seka_status launch_prep_steering(const seka_shape* sh, const SteerPlan& plan, const void* K16, const float* U,
@@ -542,11 +617,12 @@ seka_status launch_prep_steering(const seka_shape* sh, const SteerPlan& plan, co
     const int n_a = (routed && alpha_out != nullptr) ? sh->batch * Hkv : 0;
     int n_sm = 0;
     if (!device_info(&n_sm)) return SEKA_ERR_CUDA;
-    // blocks per KV head for the edited keys: about one wave of the device (shared and tensor memory decide how many
-    // blocks fit an SM), at most one per (sequence, tile)
+    // blocks per KV head for the edited keys: one wave of the device (shared and tensor memory decide how many blocks
+    // fit an SM), at most one per (sequence, tile)
     const size_t smem = prep_steering_smem(sh, routed, k_route);
     if (smem > 200 * 1024) return SEKA_ERR_UNSUPPORTED;
-    const int per_sm = D == 64 && smem <= 64 * 1024 ? 3 : 1;
+    // (about 10.5 KB of static shared memory per block on top; the register file holds two blocks)
+    const int per_sm = (227 * 1024) / (smem + 11 * 1024) >= 2 ? 2 : 1;
     // (one wave: a block that had to wait for a free SM would finish a whole block-time later)
     long long per_head = ((long long)per_sm * n_sm - n_flag - n_a) / Hkv;
     const long long pairs = (long long)sh->batch * n_tiles;
