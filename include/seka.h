@@ -105,7 +105,7 @@ seka_status adaseka_route(const seka_shape* shape, const void* Q, const float* U
  * formed once per call, in fp32, by a preparation launch into `workspace` as a high and
  * a low bf16 part; the attention kernel stages those tiles from there instead of from K
  * and adds the contraction with the low parts where it matters (gain x coefficient above
- * 1 in magnitude, and every query row that sees at most 1024 keys), so the logits follow
+ * 1 in magnitude, and every query row that sees at most 512 keys), so the logits follow
  * the fp32 edited keys there and one bf16 rounding of them elsewhere.
  * O has the dtype of the inputs.  With dtype SEKA_F32 the inputs are rounded to bf16
  * on the way in (the contraction runs on bf16 tensor cores, fp32 accumulation).

@@ -64,12 +64,12 @@ static inline SteerPlan make_steer_plan(const seka_shape* s, bool steer) {
 // eps = 2^-9 |q| |k'| / sqrt(3 d) in scaled units (1.2e-3 (1 + |g| a) for unit-variance inputs, a = largest |alpha|),
 // and the output by about eps |v - o| sqrt(sum_j p_j^2).  Two cases take the low parts:
 //   - |g| a > 1: the edited keys are far from unit variance and eps grows with them;
-//   - query rows that see at most kLoTiles key tiles (1024 keys): with few keys sqrt(sum p^2) is not small and the
+//   - query rows that see at most kLoTiles key tiles (512 keys): with few keys sqrt(sum p^2) is not small and the
 //     tail of that noise reaches the stated 1e-2 on single elements (seen on a 35-key row at g = 1); these work items
 //     are a few per cent of the steps of a long prompt.
 // Everywhere else (long rows, |g| a <= 1) the noise is averaged over thousands of keys and stays several times
 // below the rounding of P itself.
-constexpr int kLoTiles = 8;
+constexpr int kLoTiles = 4;
 #if defined(__CUDACC__)
 __host__ __device__
 #endif
