@@ -830,9 +830,13 @@ static seka_status attention_fwd_impl(const seka_shape* shape, const void* Q, co
     int* first_hot = reinterpret_cast<int*>(ws + w.first_off);
     uint8_t* bh_info = reinterpret_cast<uint8_t*>(ws + w.info_off);
     if (steer) {
-        stc = launch_prep_steering(shape, p.plan, k16, U, alpha, gain, head_enable, mask, X, tile_hot, first_hot, bh_info,
-                                   reinterpret_cast<int*>(ws),
-                                   w.n_tiles, st, Q, sigma, k_route, alpha_out);
+        // one expert with given coefficients: the pipelined tile kernel of the stand-alone edit writes the side buffer (two
+        // small launches); banks of experts and routed coefficients: the one-launch preparation kernel
+        if (shape->n_experts == 1 && sigma == nullptr)
+            stc = launch_stage_keys_pipe(shape, w, k16, X, mask, U, alpha, gain, head_enable, ws, st);
+        else
+            stc = launch_prep_steering(shape, p.plan, k16, U, alpha, gain, head_enable, mask, X, tile_hot, first_hot, bh_info,
+                                       reinterpret_cast<int*>(ws), w.n_tiles, st, Q, sigma, k_route, alpha_out);
         if (stc != SEKA_OK) return stc;
     }
 

@@ -296,7 +296,7 @@ edit_tiles_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
 constexpr int EP_NS = 4;                      // key tiles in flight per SM
 constexpr int EP_THREADS = 320;
 
-struct EpMeta { int tok0, h, valid, p_gen; float c; int pad[3]; };     // per stage: first token, head, end marker, projector generation, g * alpha
+struct EpMeta { int tok0, h, valid, p_gen; float c; int nvalid, with_lo, pad; };     // per stage: first token, head, end marker, projector generation, g * alpha, rows inside the sequence, low parts wanted (side mode)
 
 template <int D>
 struct EpSmem {
@@ -313,7 +313,10 @@ struct EpSmem {
     static constexpr uint32_t DYN_BYTES = MISC + 16 + 1024;
 };
 
-template <int D>
+// SIDE: instead of rewriting the highlighted rows of the key tensor, write k' of every row of the tile that lies inside
+// its sequence into the side buffer of the fused forward, rows of 2 D bf16: high parts [0, D), low parts [D, 2 D) (the low
+// parts only where the fused kernel reads them: see lo_needed; zero for rows that are not highlighted).
+template <int D, bool SIDE>
 __global__ void __launch_bounds__(EP_THREADS, 1)
 edit_tiles_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmP,
                        __nv_bfloat16* __restrict__ K_out, const uint8_t* __restrict__ mask, const float* __restrict__ alpha,
@@ -409,6 +412,8 @@ edit_tiles_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
             if (lane == 0) {
                 EpMeta* m = reinterpret_cast<EpMeta*>(smem + SL::META + s * 32);
                 m->tok0 = seq0 + t * 128; m->h = h; m->valid = last ? 0 : 1; m->p_gen = p_gen; m->c = c;
+                m->nvalid = Lb - t * 128 < 128 ? Lb - t * 128 : 128;
+                m->with_lo = (SIDE && !last && (lo_needed(gain[b], alpha != nullptr ? fabsf(alpha[(size_t)b * Hkv + h]) : 1.f) || t < kLoTiles)) ? 1 : 0;
                 if (!last) {
                     mbar_expect_tx(full + s, SL::TILE);
 #pragma unroll
@@ -476,12 +481,19 @@ edit_tiles_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
             if (!ok) break;
             tc_fence_after();
             // (the tensor-memory loads are warp-wide: every lane takes part, only the row update depends on the flag)
-            if (__any_sync(0xffffffffu, hl)) {
+            const bool side_lo = SIDE && m.with_lo != 0 && row < m.nvalid;
+            __nv_bfloat16* xlo = K_out + ((size_t)(m.tok0 + (row < m.nvalid ? row : 0)) * Hkv + m.h) * (2 * D) + D;
+            if (__any_sync(0xffffffffu, hl) || (SIDE && m.with_lo != 0)) {
+                const bool warp_hl = __any_sync(0xffffffffu, hl);
 #pragma unroll 1
                 for (int c = half * (D / 64); c < (half + 1) * (D / 64); ++c) {
                     uint32_t v[32];
-                    tmem_ld32(t_lane + cset * D + c * 32, v);
-                    tmem_wait_ld_on(v);
+                    if (warp_hl) { tmem_ld32(t_lane + cset * D + c * 32, v); tmem_wait_ld_on(v); }
+                    uint4 lo4[4];
+                    if (SIDE) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) lo4[q] = make_uint4(0u, 0u, 0u, 0u);
+                    }
                     if (hl) {
                         uint4* ptr[4];
                         uint4 kv[4];
@@ -494,14 +506,25 @@ edit_tiles_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
                             uint32_t* w = reinterpret_cast<uint32_t*>(&kv[q]);
+                            uint32_t* l = reinterpret_cast<uint32_t*>(&lo4[q]);
 #pragma unroll
                             for (int e = 0; e < 4; ++e) {
                                 const float2 k2 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&w[e]));
-                                w[e] = pack_bf16(fmaf(m.c, __uint_as_float(v[q * 8 + 2 * e]), k2.x), fmaf(m.c, __uint_as_float(v[q * 8 + 2 * e + 1]), k2.y));
+                                const float x0 = fmaf(m.c, __uint_as_float(v[q * 8 + 2 * e]), k2.x), x1 = fmaf(m.c, __uint_as_float(v[q * 8 + 2 * e + 1]), k2.y);
+                                w[e] = pack_bf16(x0, x1);
+                                if (SIDE) {        // the low parts: what the rounding above dropped
+                                    const float2 h2 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&w[e]));
+                                    l[e] = pack_bf16(x0 - h2.x, x1 - h2.y);
+                                }
                             }
                         }
 #pragma unroll
                         for (int q = 0; q < 4; ++q) *ptr[q] = kv[q];
+                    }
+                    if (side_lo) {
+                        uint4* dst = reinterpret_cast<uint4*>(xlo + c * 32);
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) dst[q] = lo4[q];
                     }
                     __syncwarp();      // all lanes together again before the next warp-wide load
                 }
@@ -516,9 +539,9 @@ edit_tiles_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
 #pragma unroll 1
             for (int i = 0; i < 16 / RPI; ++i) {
                 const int r = warp * 16 + i * RPI + lane / LPR, col = (lane % LPR) * 8;
-                if (fl[r]) {
+                if (SIDE ? r < m.nvalid : fl[r] != 0) {
                     const uint4 v = *reinterpret_cast<const uint4*>(sK + (col >> 6) * EBLK + sw128_offset(r, col & 63));
-                    *reinterpret_cast<uint4*>(K_out + ((size_t)(m.tok0 + r) * Hkv + m.h) * D + col) = v;
+                    *reinterpret_cast<uint4*>(K_out + ((size_t)(m.tok0 + r) * Hkv + m.h) * (SIDE ? 2 * D : D) + col) = v;
                 }
             }
             __syncwarp();
@@ -553,11 +576,11 @@ static seka_status launch_edit_tiles(const seka_shape* s, const WorkspaceLayout&
     if (!make_tile_map(&tk, K_in, D, Hkv, T) || !make_tile_map(&tp, P, D, 1, (long long)2 * M * Hkv * D, D)) return SEKA_ERR_CUDA;
     if (M == 1) {
         using PL = EpSmem<D>;
-        if (cudaFuncSetAttribute(edit_tiles_pipe_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PL::DYN_BYTES) != cudaSuccess)
+        if (cudaFuncSetAttribute(edit_tiles_pipe_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PL::DYN_BYTES) != cudaSuccess)
             return SEKA_ERR_CUDA;
         const long long work = (long long)s->batch * w.n_tiles * Hkv;
         const unsigned gridp = (unsigned)(work < (long long)n_sm ? work : (long long)n_sm);
-        edit_tiles_pipe_kernel<D><<<gridp, EP_THREADS, PL::DYN_BYTES, st>>>(tk, tp, static_cast<__nv_bfloat16*>(K_out), mask, alpha, gain, he,
+        edit_tiles_pipe_kernel<D, false><<<gridp, EP_THREADS, PL::DYN_BYTES, st>>>(tk, tp, static_cast<__nv_bfloat16*>(K_out), mask, alpha, gain, he,
                                                                           s->cu_seqlens, hot_list, status + 2, status, s->max_seqlen,
                                                                           Hkv, w.n_tiles);
         ++g_launches;
@@ -574,6 +597,40 @@ static seka_status launch_edit_tiles(const seka_shape* s, const WorkspaceLayout&
                                                          w.n_tiles, cols);
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? SEKA_OK : SEKA_ERR_CUDA;
+}
+
+template <int D>
+static seka_status stage_keys_pipe_t(const seka_shape* s, const WorkspaceLayout& w, const void* K16, void* X,
+                                     const uint8_t* mask, const float* U, const float* alpha, const float* gain,
+                                     const uint8_t* he, char* ws, cudaStream_t st) {
+    using PL = EpSmem<D>;
+    int n_sm = 0;
+    if (!device_info(&n_sm)) return SEKA_ERR_CUDA;
+    int* status = reinterpret_cast<int*>(ws);
+    void* P = ws + w.w_off;
+    uint8_t* tile_hot = reinterpret_cast<uint8_t*>(ws + w.hot_off);
+    int* hot_list = reinterpret_cast<int*>(ws + w.list_off);
+    launch_prep_edit(s, U, mask, P, tile_hot, w.n_tiles, hot_list, status + 2, st, reinterpret_cast<int*>(ws + w.first_off),
+                     reinterpret_cast<uint8_t*>(ws + w.info_off), gain, alpha, he);
+    const int T = shape_total_tokens(s), Hkv = s->n_kv_heads;
+    CUtensorMap tk, tp;
+    if (!make_tile_map(&tk, K16, D, Hkv, T) || !make_tile_map(&tp, P, D, 1, (long long)2 * Hkv * D, D)) return SEKA_ERR_CUDA;
+    if (cudaFuncSetAttribute(edit_tiles_pipe_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PL::DYN_BYTES) != cudaSuccess)
+        return SEKA_ERR_CUDA;
+    const long long work = (long long)s->batch * w.n_tiles * Hkv;
+    const unsigned grid = (unsigned)(work < (long long)n_sm ? work : (long long)n_sm);
+    edit_tiles_pipe_kernel<D, true><<<grid, EP_THREADS, PL::DYN_BYTES, st>>>(tk, tp, static_cast<__nv_bfloat16*>(X), mask, alpha, gain, he,
+                                                                           s->cu_seqlens, hot_list, status + 2, status, s->max_seqlen,
+                                                                           Hkv, w.n_tiles);
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? SEKA_OK : SEKA_ERR_CUDA;
+}
+
+seka_status launch_stage_keys_pipe(const seka_shape* s, const WorkspaceLayout& w, const void* K16, void* X,
+                                   const uint8_t* mask, const float* U, const float* alpha, const float* gain,
+                                   const uint8_t* head_enable, char* ws, cudaStream_t st) {
+    return s->head_dim == 128 ? stage_keys_pipe_t<128>(s, w, K16, X, mask, U, alpha, gain, head_enable, ws, st)
+                              : stage_keys_pipe_t<64>(s, w, K16, X, mask, U, alpha, gain, head_enable, ws, st);
 }
 
 }  // namespace seka

@@ -480,10 +480,16 @@ prep_steering_kernel(const __grid_constant__ CUtensorMap tmK, int* status, const
 //                      coefficients are applied per row when dK is added, so this does not depend on the batch;
 //   blocks [n_p, ...): one warp per (sequence, 128-key tile): flag, and the tiles that hold a highlighted token
 //                      appended to `hot_list` (any order).
+// (for the fused forward) also the first highlighted tile of every sequence (atomic minimum: `first_hot` starts large)
+// and the steering byte of every (sequence, KV head): bit 0 steered, bit 1 the fused kernel multiplies the low parts too
+struct SteerInfoArgs {
+    int* first_hot; uint8_t* bh_info; const float* gain; const float* alpha; const uint8_t* head_enable;
+};
+
 __global__ void prep_edit_kernel(const float* __restrict__ U, const uint8_t* __restrict__ mask,
                                  const int* __restrict__ cu_seqlens, __nv_bfloat16* __restrict__ P,
                                  uint8_t* __restrict__ tile_hot, int* __restrict__ hot_list, int* __restrict__ hot_count,
-                                 int B, int L, int Hkv, int D, int r, int M, int n_tiles, int n_p) {
+                                 int B, int L, int Hkv, int D, int r, int M, int n_tiles, int n_p, const SteerInfoArgs info) {
     const int tid = threadIdx.x;
     if ((int)blockIdx.x < n_p) {
         const int tiles = D / 32;
@@ -532,6 +538,15 @@ __global__ void prep_edit_kernel(const float* __restrict__ U, const uint8_t* __r
         if (lane == 0) {
             tile_hot[item] = any ? 1 : 0;
             if (any) hot_list[atomicAdd(hot_count, 1)] = item;
+            if (any && info.first_hot != nullptr) atomicMin(info.first_hot + b, t);
+        }
+        if (info.bh_info != nullptr && t == 0) {
+            const float g = info.gain[b];
+            for (int h = lane; h < Hkv; h += 32) {
+                const bool on = g != 0.f && (info.head_enable == nullptr || info.head_enable[h] != 0);
+                const float amax = alpha_max_of(info.alpha, (size_t)b * Hkv + h, M);
+                info.bh_info[(size_t)b * Hkv + h] = (on ? 1 : 0) | ((on && lo_needed(g, amax)) ? 2 : 0);
+            }
         }
     }
 }
@@ -644,14 +659,17 @@ seka_status launch_prep_steering(const seka_shape* sh, const SteerPlan& plan, co
 }
 
 void launch_prep_edit(const seka_shape* sh, const float* U, const uint8_t* mask, void* P, uint8_t* tile_hot, int n_tiles,
-                      int* hot_list, int* hot_count, cudaStream_t st) {
+                      int* hot_list, int* hot_count, cudaStream_t st, int* first_hot, uint8_t* bh_info, const float* gain,
+                      const float* alpha, const uint8_t* head_enable) {
     const int D = sh->head_dim, tiles = D / 32;
     const int n_p = sh->n_experts * sh->n_kv_heads * tiles * tiles;
     const int n_flag = (sh->batch * n_tiles + 7) / 8;
     cudaMemsetAsync(hot_count, 0, sizeof(int), st);
+    if (first_hot != nullptr) cudaMemsetAsync(first_hot, 0x7f, sizeof(int) * sh->batch, st);      // a large value per sequence
+    SteerInfoArgs info{first_hot, bh_info, gain, alpha, head_enable};
     prep_edit_kernel<<<n_p + n_flag, 256, 0, st>>>(U, mask, sh->cu_seqlens, static_cast<__nv_bfloat16*>(P), tile_hot, hot_list,
                                                   hot_count, sh->batch, sh->max_seqlen, sh->n_kv_heads, D, sh->rank,
-                                                  sh->n_experts, n_tiles, n_p);
+                                                  sh->n_experts, n_tiles, n_p, info);
     ++g_launches;
 }
 
