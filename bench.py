@@ -34,8 +34,8 @@ WORKLOAD = "C2: 8B-shaped prefill layer B=4 Hq=32 Hkv=8 d=128 L=4096 bf16, rank 
 # Counters of one fused-kernel launch on this workload, from the ncu capture of the current kernel (summary under
 # profiles/): dram__bytes_read.sum + dram__bytes_write.sum, and sm__pipe_tensor_cycles_active in per cent.
 # None means: no capture of the kernel as it stands.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 422682624     # 325.68 MB read + 97.00 MB written, steered launch
-NCU_TENSOR_PIPE_ACTIVE_PCT = 56.2
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 431451648     # 335.07 MB read + 96.38 MB written, steered launch
+NCU_TENSOR_PIPE_ACTIVE_PCT = 56.1
 NOMINAL_BF16_TFLOPS = 2250.0      # dense bf16, datasheet
 
 
