@@ -13,8 +13,9 @@
  *  - Pointers are DEVICE pointers unless the name starts with `h_`. The caller owns
  *    every buffer; the library keeps none and allocates no device memory.  Process state it
  *    does keep: the launch counter of seka_launch_count (atomic), the SM count of each
- *    device it has been called on, the driver entry point for tensor maps, and the
- *    per-device address of the built-in scratch of seka_edit_keys_static (all behind
+ *    device it has been called on, the driver entry point for tensor maps, the per-device
+ *    address of the built-in scratch of seka_edit_keys_static, and eight events per device
+ *    that order the staging buffer of seka_attention_fwd_host between calls (all behind
  *    mutexes; calls may come from several host threads and for several devices).
  *  - Tensors are packed token-major: Q [T, Hq, d], K and V [T, Hkv, d], O [T, Hq, d],
  *    mask [T] (non-zero = highlighted), T = total_tokens, rows contiguous, base
@@ -140,8 +141,15 @@ seka_status seka_attention_fwd_routed(const seka_shape* shape, const void* Q, co
  * is complete when the work queued on `cuda_stream` is.  A fixed-length batch is cut by
  * sequence into up to eight parts that are copied in, computed and copied out as a
  * pipeline (the call creates two more streams and a few events for its duration and
- * releases them before it returns); a packed batch goes through in one piece.  U, alpha,
- * gain, head_enable stay device pointers (they are per-model or per-prompt constants).
+ * releases them before it returns); a packed batch goes through in one piece.  The host
+ * input buffers are read from the moment of the call on: they must hold their data when
+ * the call is made, and the copies in do NOT wait for work queued on `cuda_stream`
+ * earlier (so the input copies of one call overlap the output copies of the call before
+ * it).  What they do wait for is the previous host-buffer call's kernels on this device,
+ * which may still be reading a staging buffer; the library keeps eight events per device
+ * for that.  `staging` belongs to the call until `cuda_stream` has passed it; two calls
+ * that overlap in time need a staging buffer and a workspace each.  U, alpha, gain,
+ * head_enable stay device pointers (they are per-model or per-prompt constants).
  */
 size_t seka_host_staging_bytes(const seka_shape* shape);
 seka_status seka_attention_fwd_host(const seka_shape* shape, const void* h_Q, const void* h_K,

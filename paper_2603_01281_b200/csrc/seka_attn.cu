@@ -896,6 +896,21 @@ extern "C" size_t seka_host_staging_bytes(const seka_shape* shape) {
     return 2 * nq + 2 * nk + align_up(T, 256) + align_up(T * shape->n_q_heads * 4, 256);
 }
 
+namespace seka {
+// Per device: events that mark the end of the compute of each part of the last host-buffer call, and that call's
+// geometry.  The next call's copies into the staging buffer wait for them instead of for the caller's stream, so its
+// input copies run while the previous call's output is still on its way back.
+struct HostPipeState {
+    cudaEvent_t cmp[8] = {};
+    bool made = false, valid = false;
+    const void* staging = nullptr;
+    int parts = 0;
+    size_t tok_per = 0;
+};
+static std::mutex g_host_pipe_mutex;
+static HostPipeState g_host_pipe[64];
+}  // namespace seka
+
 extern "C" seka_status seka_attention_fwd_host(const seka_shape* shape, const void* h_Q, const void* h_K,
                                                const void* h_V, void* h_O, float* h_lse, const uint8_t* h_mask,
                                                const float* U, const float* alpha, const float* gain,
@@ -930,17 +945,27 @@ extern "C" seka_status seka_attention_fwd_host(const seka_shape* shape, const vo
     const int seq_per = shape->batch / parts;
     const size_t tok_per = (size_t)seq_per * shape->max_seqlen;
     cudaStream_t s_in = nullptr, s_out = nullptr;
-    cudaEvent_t ev_start = nullptr, ev_in[8] = {}, ev_cmp[8] = {}, ev_out = nullptr;
+    cudaEvent_t ev_tail = nullptr, ev_in[8] = {}, ev_out = nullptr;
     bool okc = true;
     auto make_event = [&](cudaEvent_t* e) { okc = okc && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess; };
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SEKA_ERR_CUDA;
+    std::lock_guard<std::mutex> pipe_lock(g_host_pipe_mutex);
+    HostPipeState& hs = g_host_pipe[dev];
+    if (!hs.made) {
+        for (int i = 0; i < 8; ++i) make_event(&hs.cmp[i]);
+        if (!okc) return SEKA_ERR_CUDA;
+        hs.made = true;
+    }
+    // The staging buffer of the call before may still be read by its kernels.  Same buffer cut the same way: part i
+    // waits for that call's part i; anything else: for its last part.
+    const bool same_cut = hs.valid && hs.staging == staging && hs.parts == parts && hs.tok_per == tok_per;
+    const int prev_last = hs.valid ? hs.parts - 1 : -1;
     if (parts > 1) {
         okc = okc && cudaStreamCreateWithFlags(&s_in, cudaStreamNonBlocking) == cudaSuccess;
         okc = okc && cudaStreamCreateWithFlags(&s_out, cudaStreamNonBlocking) == cudaSuccess;
-        make_event(&ev_start); make_event(&ev_out);
-        for (int i = 0; i < parts; ++i) { make_event(&ev_in[i]); make_event(&ev_cmp[i]); }
-        // the copies start after whatever the caller queued before this call
-        okc = okc && cudaEventRecord(ev_start, st) == cudaSuccess && cudaStreamWaitEvent(s_in, ev_start, 0) == cudaSuccess &&
-              cudaStreamWaitEvent(s_out, ev_start, 0) == cudaSuccess;
+        make_event(&ev_tail); make_event(&ev_out);
+        for (int i = 0; i < parts; ++i) make_event(&ev_in[i]);
     } else {
         s_in = st; s_out = st;
     }
@@ -949,6 +974,8 @@ extern "C" seka_status seka_attention_fwd_host(const seka_shape* shape, const vo
     part.total_tokens = shape->cu_seqlens ? shape->total_tokens : 0;
     for (int i = 0; i < parts && okc && stc == SEKA_OK; ++i) {
         const size_t t0 = (size_t)i * tok_per, nt = parts > 1 ? tok_per : T;
+        if (parts > 1 && prev_last >= 0 && (same_cut || i == 0))
+            okc = okc && cudaStreamWaitEvent(s_in, hs.cmp[same_cut ? i : prev_last], 0) == cudaSuccess;
         okc = okc && cudaMemcpyAsync(dq + t0 * rq, static_cast<const char*>(h_Q) + t0 * rq, nt * rq, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
         okc = okc && cudaMemcpyAsync(dk + t0 * rk, static_cast<const char*>(h_K) + t0 * rk, nt * rk, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
         okc = okc && cudaMemcpyAsync(dv + t0 * rk, static_cast<const char*>(h_V) + t0 * rk, nt * rk, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
@@ -961,7 +988,8 @@ extern "C" seka_status seka_attention_fwd_host(const seka_shape* shape, const vo
                                  alpha ? alpha + (size_t)i * seq_per * shape->n_kv_heads * shape->n_experts : nullptr,
                                  gain ? gain + (size_t)i * seq_per : nullptr, head_enable, workspace, workspace_bytes, cuda_stream);
         if (stc != SEKA_OK) break;
-        if (parts > 1) okc = okc && cudaEventRecord(ev_cmp[i], st) == cudaSuccess && cudaStreamWaitEvent(s_out, ev_cmp[i], 0) == cudaSuccess;
+        okc = okc && cudaEventRecord(hs.cmp[i], st) == cudaSuccess;
+        if (parts > 1) okc = okc && cudaStreamWaitEvent(s_out, hs.cmp[i], 0) == cudaSuccess;
         okc = okc && cudaMemcpyAsync(static_cast<char*>(h_O) + t0 * rq, dO + t0 * rq, nt * rq, cudaMemcpyDeviceToHost, s_out) == cudaSuccess;
         if (h_lse) okc = okc && cudaMemcpyAsync(h_lse + t0 * shape->n_q_heads, reinterpret_cast<float*>(dl) + t0 * shape->n_q_heads,
                                                 nt * shape->n_q_heads * 4, cudaMemcpyDeviceToHost, s_out) == cudaSuccess;
@@ -969,14 +997,18 @@ extern "C" seka_status seka_attention_fwd_host(const seka_shape* shape, const vo
     if (parts > 1) {
         // the caller's stream ends behind the last copy out (and behind the copies in, if the loop stopped early)
         if (ev_out && s_out) { cudaEventRecord(ev_out, s_out); cudaStreamWaitEvent(st, ev_out, 0); }
-        if (ev_start && s_in) { cudaEventRecord(ev_start, s_in); cudaStreamWaitEvent(st, ev_start, 0); }
+        if (ev_tail && s_in) { cudaEventRecord(ev_tail, s_in); cudaStreamWaitEvent(st, ev_tail, 0); }
         // queued work keeps what it needs: destroying a stream or an event only drops the handle
-        for (int i = 0; i < parts; ++i) { if (ev_in[i]) cudaEventDestroy(ev_in[i]); if (ev_cmp[i]) cudaEventDestroy(ev_cmp[i]); }
-        if (ev_start) cudaEventDestroy(ev_start);
+        for (int i = 0; i < parts; ++i) if (ev_in[i]) cudaEventDestroy(ev_in[i]);
+        if (ev_tail) cudaEventDestroy(ev_tail);
         if (ev_out) cudaEventDestroy(ev_out);
         if (s_in) cudaStreamDestroy(s_in);
         if (s_out) cudaStreamDestroy(s_out);
     }
+    // a call that stopped early leaves the next one to wait for the whole stream instead
+    hs.valid = okc && stc == SEKA_OK;
+    hs.staging = staging; hs.parts = parts; hs.tok_per = tok_per;
+    if (!hs.valid) cudaStreamSynchronize(st);
     if (stc != SEKA_OK) return stc;
     return okc ? SEKA_OK : SEKA_ERR_CUDA;
 }

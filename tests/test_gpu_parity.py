@@ -182,6 +182,33 @@ def test_host_buffer_entry_point():
     assert np.array_equal(hO.double().numpy(), ref) and np.array_equal(hlse.double().numpy(), lse)
 
 
+def test_host_buffer_calls_back_to_back_share_a_staging_buffer():
+    """Calls through host buffers overlap: the input copies of one run while the output of the one before is still on
+    its way back, all through one staging buffer.  Different inputs, the same cut and then another cut (a batch of four,
+    a batch of two, a packed batch), queued without a synchronisation in between: each result equals the device path's."""
+    cases = []
+    for seed, lens in ((21, [384] * 4), (22, [384] * 4), (23, [768] * 2), (24, [384] * 4), (25, [300, 41, 384]), (26, [384] * 4)):
+        w = inputs.make_custom(seed=seed, dtype="bf16", lens=lens, n_q_heads=4, n_kv_heads=2, head_dim=128, rank=32,
+                               gain=1.0, highlight=0.2)
+        dev = H.device_tensors(w)
+        cases.append((w, dev, H.shape_of(w, dev)))
+    nbytes = max(binding.seka_host_staging_bytes(shp) for _, _, shp in cases)
+    staging = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    ws = torch.zeros(max(binding.seka_workspace_bytes(shp) for _, _, shp in cases), dtype=torch.uint8, device="cuda")
+    host = []
+    for w, dev, shp in cases:
+        hQ, hK, hV = (dev[k].cpu().pin_memory() for k in "QKV")
+        host.append((hQ, hK, hV, dev["mask"].cpu().pin_memory(), torch.empty_like(hQ).pin_memory()))
+    torch.cuda.synchronize()
+    for (w, dev, shp), (hQ, hK, hV, hm, hO) in zip(cases, host):
+        binding.seka_attention_fwd_host(shp, hQ, hK, hV, hO, None, hm, dev["U"], None, dev["gain"], None, staging, ws)
+    torch.cuda.synchronize()
+    assert binding.seka_poll_status(ws) == binding.SEKA_OK
+    for (w, dev, shp), (_, _, _, _, hO) in zip(cases, host):
+        ref, _ = H.run_fused(w, dev)
+        assert np.array_equal(hO.double().numpy(), ref)
+
+
 # ----------------------------------------------------------------- fused attention: the five configurations at full size
 
 @pytest.mark.parametrize("name,nrows,nseq", [("C2", 256, None), ("C3", 256, None), ("C4", 256, None), ("C5", None, 8), ("C2s70", 128, None)])
