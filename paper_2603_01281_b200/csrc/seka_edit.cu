@@ -293,7 +293,6 @@ edit_tiles_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
 //   warp 9   MMA issuer: K P (two bf16 parts) into one of two sets of tensor-memory columns;
 //   warps 0-7  drain: half a key row per thread, k' = k + c (K P)[row] into the staged tile for highlighted rows,
 //            then the highlighted rows go out 16 bytes per lane; the stage and the columns are handed back.
-constexpr int EP_NS = 4;                      // key tiles in flight per SM
 constexpr int EP_THREADS = 320;
 
 struct EpMeta { int tok0, h, valid, p_gen; float c; int nvalid, with_lo, pad; };     // per stage: first token, head, end marker, projector generation, g * alpha, rows inside the sequence, low parts wanted (side mode)
@@ -303,12 +302,13 @@ struct EpSmem {
     static constexpr uint32_t TILE = (D / 64) * EBLK;
     static constexpr uint32_t PBLK = D * 128;
     static constexpr uint32_t PMAT = (D / 64) * PBLK;
-    static constexpr uint32_t K = 0;                        // EP_NS stages
-    static constexpr uint32_t P = K + EP_NS * TILE;         // high part, then low part
-    static constexpr uint32_t FLAGS = P + 2 * PMAT;         // EP_NS x 128 bytes
-    static constexpr uint32_t META = FLAGS + EP_NS * 128;   // EP_NS x 32 bytes
-    static constexpr uint32_t BARS = META + EP_NS * 32;     // full[NS], free[NS], mma_done[2], cols_free[2], p_full, meet[2]
-    static constexpr uint32_t NBARS = 2 * EP_NS + 7;
+    static constexpr int NS = D == 128 ? 4 : 8;             // key tiles in flight per SM
+    static constexpr uint32_t K = 0;                        // NS stages
+    static constexpr uint32_t P = K + NS * TILE;            // high part, then low part
+    static constexpr uint32_t FLAGS = P + 2 * PMAT;         // NS x 128 bytes
+    static constexpr uint32_t META = FLAGS + NS * 128;      // NS x 32 bytes
+    static constexpr uint32_t BARS = META + NS * 32;        // full[NS], free[NS], mma_done[2], cols_free[2], p_full, meet[2]
+    static constexpr uint32_t NBARS = 2 * NS + 7;
     static constexpr uint32_t MISC = BARS + NBARS * 8;
     static constexpr uint32_t DYN_BYTES = MISC + 16 + 1024;
 };
@@ -324,6 +324,7 @@ edit_tiles_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
                        const int* __restrict__ cu_seqlens, const int* __restrict__ hot_list, const int* __restrict__ hot_count,
                        int* status, int L, int Hkv, int n_tiles) {
     using SL = EpSmem<D>;
+    constexpr int EP_NS = SL::NS;
     constexpr int NBLK = D / 64;
     constexpr uint32_t TMEM_COLS = 2 * D < 32 ? 32 : 2 * D;
     extern __shared__ uint8_t smem_raw[];
@@ -366,65 +367,105 @@ edit_tiles_pipe_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         uint32_t n_push = 0;      // stages filled so far
         int p_gen = 0, cur_h = -1;
         bool ok = true;
-        for (long long idx = w0; idx <= w1 && ok; ++idx) {
-            const bool last = idx >= w1;                    // one more stage after the work: the end marker
-            int h = 0, tile = 0, b = 0, t = 0, seq0 = 0, Lb = 0;
-            float c = 0.f;
-            if (!last) {
-                h = (int)(idx / n_hot); tile = hot_list[idx % n_hot];
-                b = tile / n_tiles; t = tile % n_tiles;
-                const float g = gain[b];
-                if (g == 0.f || (head_enable != nullptr && head_enable[h] == 0)) continue;
-                c = g * (alpha != nullptr ? alpha[(size_t)b * Hkv + h] : 1.f);
-                seq0 = cu_seqlens ? cu_seqlens[b] : b * L;
-                Lb = (cu_seqlens ? cu_seqlens[b + 1] : (b + 1) * L) - seq0;
-                if (h != cur_h) {
-                    // the projector changes: every tile of the old head must be through the tensor core (here: the
-                    // whole ring handed back), then the new one is loaded
-                    for (uint32_t q = n_push >= EP_NS ? n_push - EP_NS : 0; q < n_push && ok; ++q)
-                        ok = warp_wait(freeb + q % EP_NS, (q / EP_NS) & 1, abort_flag, status, 62);
-                    if (!ok) break;
-                    if (lane == 0) {
-                        mbar_expect_tx(p_full, 2 * SL::PMAT);
-#pragma unroll
-                        for (int part = 0; part < 2; ++part)
-#pragma unroll
-                            for (int cb = 0; cb < NBLK; ++cb)
-                                tma_load_3d(smem + SL::P + part * SL::PMAT + cb * SL::PBLK, &tmP, p_full, cb * 64, 0, (part * Hkv + h) * D);
-                    }
-                    __syncwarp();
-                    cur_h = h; ++p_gen;
+        // What a work unit needs from global memory (its entry of the list, the sequence bounds, gain, coefficient) is a
+        // chain of dependent loads; one lane per unit fetches it for 32 units at a time, and the highlight flags of a
+        // tile are requested one tile ahead, so that the ring is not fed at the pace of memory round trips.
+        uint8_t fl_next[4] = {0, 0, 0, 0};
+        bool have_next = false;
+        for (long long base = w0; base <= w1 && ok; base += 32) {
+            int h_l = 0, t_l = 0, seq0_l = 0, Lb_l = 0, lo_l = 0, skip_l = 1;
+            float c_l = 0.f;
+            {
+                const long long my = base + lane;
+                if (my < w1) {
+                    h_l = (int)(my / n_hot);
+                    const int tile = hot_list[my % n_hot];
+                    const int b = tile / n_tiles;
+                    t_l = tile % n_tiles;
+                    const float g = gain[b];
+                    const float a = alpha != nullptr ? alpha[(size_t)b * Hkv + h_l] : 1.f;
+                    skip_l = (g == 0.f || (head_enable != nullptr && head_enable[h_l] == 0)) ? 1 : 0;
+                    c_l = g * a;
+                    seq0_l = cu_seqlens ? cu_seqlens[b] : b * L;
+                    Lb_l = (cu_seqlens ? cu_seqlens[b + 1] : (b + 1) * L) - seq0_l;
+                    lo_l = (SIDE && (lo_needed(g, fabsf(a)) || t_l < kLoTiles)) ? 1 : 0;
                 }
             }
-            const uint32_t s = n_push % EP_NS;
-            if (n_push >= EP_NS) {
-                ok = warp_wait(freeb + s, ((n_push / EP_NS) - 1) & 1, abort_flag, status, 63);
-                if (!ok) break;
-            }
-            uint8_t* fl = smem + SL::FLAGS + s * 128;
-            if (!last) {
+            const int n_here = (int)((w1 - base + 1) < 32 ? (w1 - base + 1) : 32);      // units of this batch, end marker included
+            auto flags_of = [&](int k, uint8_t (&f)[4]) {      // highlight flags of unit k of the batch (4 rows per lane)
+                const int seq0 = __shfl_sync(0xffffffffu, seq0_l, k), t = __shfl_sync(0xffffffffu, t_l, k), Lb = __shfl_sync(0xffffffffu, Lb_l, k);
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
                     const int kpos = t * 128 + q * 32 + lane;
-                    fl[q * 32 + lane] = (kpos < Lb && mask[seq0 + kpos] != 0) ? 1 : 0;
+                    f[q] = (kpos < Lb && mask[seq0 + kpos] != 0) ? 1 : 0;
                 }
-            }
-            if (lane == 0) {
-                EpMeta* m = reinterpret_cast<EpMeta*>(smem + SL::META + s * 32);
-                m->tok0 = seq0 + t * 128; m->h = h; m->valid = last ? 0 : 1; m->p_gen = p_gen; m->c = c;
-                m->nvalid = Lb - t * 128 < 128 ? Lb - t * 128 : 128;
-                m->with_lo = (SIDE && !last && (lo_needed(gain[b], alpha != nullptr ? fabsf(alpha[(size_t)b * Hkv + h]) : 1.f) || t < kLoTiles)) ? 1 : 0;
+            };
+            for (int k = 0; k < n_here && ok; ++k) {
+                const long long idx = base + k;
+                const bool last = idx >= w1;                    // one more stage after the work: the end marker
+                const int h = __shfl_sync(0xffffffffu, h_l, k), t = __shfl_sync(0xffffffffu, t_l, k);
+                const int seq0 = __shfl_sync(0xffffffffu, seq0_l, k), Lb = __shfl_sync(0xffffffffu, Lb_l, k);
+                const int with_lo = __shfl_sync(0xffffffffu, lo_l, k), skip = __shfl_sync(0xffffffffu, skip_l, k);
+                const float c = __shfl_sync(0xffffffffu, c_l, k);
+                uint8_t fl_cur[4] = {0, 0, 0, 0};
                 if (!last) {
-                    mbar_expect_tx(full + s, SL::TILE);
+                    if (have_next) {
 #pragma unroll
-                    for (int cb = 0; cb < NBLK; ++cb) tma_load_3d(smem + SL::K + s * SL::TILE + cb * EBLK, &tmK, full + s, cb * 64, h, seq0 + t * 128);
-                } else {
-                    mbar_arrive(full + s);
+                        for (int q = 0; q < 4; ++q) fl_cur[q] = fl_next[q];
+                    } else {
+                        flags_of(k, fl_cur);
+                    }
                 }
+                // the flags of the next unit of the batch are requested now and used in the next trip
+                have_next = k + 1 < n_here && base + k + 1 < w1;
+                if (have_next) flags_of(k + 1, fl_next);
+                if (!last) {
+                    if (skip) continue;
+                    if (h != cur_h) {
+                        // the projector changes: every tile of the old head must be through the tensor core (here: the
+                        // whole ring handed back), then the new one is loaded
+                        for (uint32_t q = n_push >= EP_NS ? n_push - EP_NS : 0; q < n_push && ok; ++q)
+                            ok = warp_wait(freeb + q % EP_NS, (q / EP_NS) & 1, abort_flag, status, 62);
+                        if (!ok) break;
+                        if (lane == 0) {
+                            mbar_expect_tx(p_full, 2 * SL::PMAT);
+#pragma unroll
+                            for (int part = 0; part < 2; ++part)
+#pragma unroll
+                                for (int cb = 0; cb < NBLK; ++cb)
+                                    tma_load_3d(smem + SL::P + part * SL::PMAT + cb * SL::PBLK, &tmP, p_full, cb * 64, 0, (part * Hkv + h) * D);
+                        }
+                        __syncwarp();
+                        cur_h = h; ++p_gen;
+                    }
+                }
+                const uint32_t s = n_push % EP_NS;
+                if (n_push >= EP_NS) {
+                    ok = warp_wait(freeb + s, ((n_push / EP_NS) - 1) & 1, abort_flag, status, 63);
+                    if (!ok) break;
+                }
+                uint8_t* fl = smem + SL::FLAGS + s * 128;
+                if (!last) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) fl[q * 32 + lane] = fl_cur[q];
+                }
+                if (lane == 0) {
+                    EpMeta* m = reinterpret_cast<EpMeta*>(smem + SL::META + s * 32);
+                    m->tok0 = seq0 + t * 128; m->h = h; m->valid = last ? 0 : 1; m->p_gen = p_gen; m->c = c;
+                    m->nvalid = Lb - t * 128 < 128 ? Lb - t * 128 : 128;
+                    m->with_lo = last ? 0 : with_lo;
+                    if (!last) {
+                        mbar_expect_tx(full + s, SL::TILE);
+#pragma unroll
+                        for (int cb = 0; cb < NBLK; ++cb) tma_load_3d(smem + SL::K + s * SL::TILE + cb * EBLK, &tmK, full + s, cb * 64, h, seq0 + t * 128);
+                    } else {
+                        mbar_arrive(full + s);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(full + s);       // second arrival: flags and coordinates are in place
+                ++n_push;
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(full + s);       // second arrival: flags and coordinates are in place
-            ++n_push;
         }
     } else if (warp == 9) {
         // ------------------------------------------------------------ MMA issuer
