@@ -144,6 +144,7 @@ struct WorkspaceLayout {
     size_t list_off, list_bytes;      // int32 [total_tokens]
     size_t cvt_off, cvt_bytes;        // bf16 copies of Q, K, V (fp32 inputs only)
     size_t x_off, x_bytes;            // edited keys of the fused kernel
+    size_t alpha_off;                 // fp32 [B, Hkv, M]: routing coefficients of a routed call that does not ask for them
     size_t edit_total;                // what the stand-alone edit needs (everything before the edited keys)
     size_t total;
     int n_tiles;                      // key tiles per sequence = ceil(max_seqlen / 128)
@@ -173,7 +174,8 @@ static inline WorkspaceLayout workspace_layout(const seka_shape* s) {
     w.edit_total = w.cvt_off + w.cvt_bytes;
     w.x_off = align_up(w.edit_total, 1024);
     w.x_bytes = align_up(T * s->n_kv_heads * plan.xcols * 2, 1024);
-    w.total = w.x_off + w.x_bytes;
+    w.alpha_off = w.x_off + w.x_bytes;
+    w.total = w.alpha_off + align_up((size_t)s->batch * s->n_kv_heads * s->n_experts * 4 + 4, 256);
     return w;
 }
 

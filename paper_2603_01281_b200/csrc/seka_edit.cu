@@ -122,7 +122,9 @@ struct EditSmem {
     static constexpr uint32_t DYN_BYTES = MISC + 16 + 1024;
 };
 
-template <int D>
+// SIDE: as in the pipelined kernel below, k' of every row of the tile that lies inside its sequence goes to the side
+// buffer of the fused forward (rows of 2 D bf16: high parts, then low parts where the fused kernel reads them).
+template <int D, bool SIDE>
 __global__ void __launch_bounds__(EDIT_THREADS)
 edit_tiles_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmP,
                   __nv_bfloat16* __restrict__ K_out, const uint8_t* __restrict__ mask, const float* __restrict__ alpha,
@@ -177,6 +179,8 @@ edit_tiles_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         const int kpos = t * 128 + row;
         const bool hl = kpos < Lb && mask[seq0 + kpos] != 0;
         if (half == 0) flags[row] = hl ? 1 : 0;
+        const int nvalid = Lb - t * 128 < 128 ? Lb - t * 128 : 128;
+        const bool with_lo = SIDE && (lo_needed(g, alpha_max_of(alpha, (size_t)b * Hkv + h, M)) || t < kLoTiles);
         for (int m = 0; m < M && ok; ++m) {
             const bool load_p = resident != m * Hkv + h;
             if (m == 0 || load_p) {
@@ -223,19 +227,27 @@ edit_tiles_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         // this thread's half row: k' = k + g sum_m alpha_m (K P_m)[row]
         // (the tensor-memory loads are warp-wide instructions: every lane of a warp that has a highlighted row
         // takes part in them, only the update of the row itself depends on the lane's own flag)
-        if (__any_sync(0xffffffffu, hl)) {
+        const bool warp_hl = __any_sync(0xffffffffu, hl);
+        if (warp_hl || with_lo) {
+            const bool side_lo = with_lo && row < nvalid;
+            __nv_bfloat16* xlo = K_out + ((size_t)(seq0 + t * 128 + (row < nvalid ? row : 0)) * Hkv + h) * (2 * D) + D;
 #pragma unroll 1
             for (int c = half * (D / 64); c < (half + 1) * (D / 64); ++c) {
                 float dk[32];
 #pragma unroll
                 for (int e = 0; e < 32; ++e) dk[e] = 0.f;
-                for (int m = 0; m < M; ++m) {
+                for (int m = 0; m < M && warp_hl; ++m) {
                     const float cm = g * (alpha != nullptr ? alpha[((size_t)b * Hkv + h) * M + m] : 1.f);
                     uint32_t v[32];
                     tmem_ld32(t_lane + (uint32_t)m * D + c * 32, v);
                     tmem_wait_ld_on(v);
 #pragma unroll
                     for (int e = 0; e < 32; ++e) dk[e] = fmaf(cm, __uint_as_float(v[e]), dk[e]);
+                }
+                uint4 lo4[4];
+                if (SIDE) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) lo4[q] = make_uint4(0u, 0u, 0u, 0u);
                 }
                 if (hl) {
                     uint4* ptr[4];
@@ -249,14 +261,25 @@ edit_tiles_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                         uint32_t* w = reinterpret_cast<uint32_t*>(&kv[q]);
+                        uint32_t* l = reinterpret_cast<uint32_t*>(&lo4[q]);
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const float2 k2 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&w[e]));
-                            w[e] = pack_bf16(k2.x + dk[q * 8 + 2 * e], k2.y + dk[q * 8 + 2 * e + 1]);
+                            const float x0 = k2.x + dk[q * 8 + 2 * e], x1 = k2.y + dk[q * 8 + 2 * e + 1];
+                            w[e] = pack_bf16(x0, x1);
+                            if (SIDE) {        // the low parts: what the rounding above dropped
+                                const float2 h2 = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&w[e]));
+                                l[e] = pack_bf16(x0 - h2.x, x1 - h2.y);
+                            }
                         }
                     }
 #pragma unroll
                     for (int q = 0; q < 4; ++q) *ptr[q] = kv[q];
+                }
+                if (SIDE && side_lo) {
+                    uint4* dst = reinterpret_cast<uint4*>(xlo + c * 32);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) dst[q] = lo4[q];
                 }
                 __syncwarp();      // all lanes together again before the next warp-wide load
             }
@@ -268,9 +291,9 @@ edit_tiles_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
 #pragma unroll 1
         for (int i = 0; i < 16 / RPI; ++i) {
             const int r = warp * 16 + i * RPI + lane / LPR, col = (lane % LPR) * 8;
-            if (flags[r]) {
+            if (SIDE ? r < nvalid : flags[r] != 0) {
                 const uint4 v = *reinterpret_cast<const uint4*>(sK + (col >> 6) * EBLK + sw128_offset(r, col & 63));
-                *reinterpret_cast<uint4*>(K_out + ((size_t)(seq0 + t * 128 + r) * Hkv + h) * D + col) = v;
+                *reinterpret_cast<uint4*>(K_out + ((size_t)(seq0 + t * 128 + r) * Hkv + h) * (SIDE ? 2 * D : D) + col) = v;
             }
         }
         __syncthreads();        // the tile and the flags are reused by the next step
@@ -605,7 +628,7 @@ static seka_status launch_edit_tiles(const seka_shape* s, const WorkspaceLayout&
     // per-device facts: looked up per device; function attributes set on every call (they belong to the current device)
     int n_sm = 0;
     if (!device_info(&n_sm)) return SEKA_ERR_CUDA;
-    if (cudaFuncSetAttribute(edit_tiles_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SL::DYN_BYTES) != cudaSuccess)
+    if (cudaFuncSetAttribute(edit_tiles_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SL::DYN_BYTES) != cudaSuccess)
         return SEKA_ERR_CUDA;
     int* status = reinterpret_cast<int*>(ws);
     void* P = ws + w.w_off;
@@ -633,7 +656,7 @@ static seka_status launch_edit_tiles(const seka_shape* s, const WorkspaceLayout&
     const long long work_max = (long long)s->batch * w.n_tiles * Hkv;
     const long long want = (long long)n_sm * per_sm;
     const unsigned grid = (unsigned)(work_max < want ? work_max : want);
-    edit_tiles_kernel<D><<<grid, EDIT_THREADS, SL::DYN_BYTES, st>>>(tk, tp, static_cast<__nv_bfloat16*>(K_out), mask, alpha, gain, he,
+    edit_tiles_kernel<D, false><<<grid, EDIT_THREADS, SL::DYN_BYTES, st>>>(tk, tp, static_cast<__nv_bfloat16*>(K_out), mask, alpha, gain, he,
                                                          s->cu_seqlens, hot_list, status + 2, status, s->max_seqlen, Hkv, M,
                                                          w.n_tiles, cols);
     ++g_launches;
@@ -653,9 +676,25 @@ static seka_status stage_keys_pipe_t(const seka_shape* s, const WorkspaceLayout&
     int* hot_list = reinterpret_cast<int*>(ws + w.list_off);
     launch_prep_edit(s, U, mask, P, tile_hot, w.n_tiles, hot_list, status + 2, st, reinterpret_cast<int*>(ws + w.first_off),
                      reinterpret_cast<uint8_t*>(ws + w.info_off), gain, alpha, he);
-    const int T = shape_total_tokens(s), Hkv = s->n_kv_heads;
+    const int T = shape_total_tokens(s), Hkv = s->n_kv_heads, M = s->n_experts;
     CUtensorMap tk, tp;
-    if (!make_tile_map(&tk, K16, D, Hkv, T) || !make_tile_map(&tp, P, D, 1, (long long)2 * Hkv * D, D)) return SEKA_ERR_CUDA;
+    if (!make_tile_map(&tk, K16, D, Hkv, T) || !make_tile_map(&tp, P, D, 1, (long long)2 * M * Hkv * D, D)) return SEKA_ERR_CUDA;
+    if (M > 1) {
+        // a bank of experts: one product pair per expert into its own tensor-memory columns, two CTAs per SM
+        using SL = EditSmem<D>;
+        if (cudaFuncSetAttribute(edit_tiles_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SL::DYN_BYTES) != cudaSuccess)
+            return SEKA_ERR_CUDA;
+        uint32_t cols = 32;
+        while (cols < (uint32_t)(M * D)) cols *= 2;
+        const int per_sm = (int)(512 / cols) < 2 ? (int)(512 / cols) : 2;
+        const long long work_max = (long long)s->batch * w.n_tiles * Hkv, want = (long long)n_sm * per_sm;
+        const unsigned grid_b = (unsigned)(work_max < want ? work_max : want);
+        edit_tiles_kernel<D, true><<<grid_b, EDIT_THREADS, SL::DYN_BYTES, st>>>(tk, tp, static_cast<__nv_bfloat16*>(X), mask, alpha, gain, he,
+                                                                              s->cu_seqlens, hot_list, status + 2, status, s->max_seqlen,
+                                                                              Hkv, M, w.n_tiles, cols);
+        ++g_launches;
+        return cudaGetLastError() == cudaSuccess ? SEKA_OK : SEKA_ERR_CUDA;
+    }
     if (cudaFuncSetAttribute(edit_tiles_pipe_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PL::DYN_BYTES) != cudaSuccess)
         return SEKA_ERR_CUDA;
     const long long work = (long long)s->batch * w.n_tiles * Hkv;

@@ -28,9 +28,14 @@ void launch_prep_edit(const seka_shape* s, const float* U, const uint8_t* mask, 
                       int* hot_list, int* hot_count, cudaStream_t st, int* first_hot = nullptr, uint8_t* bh_info = nullptr,
                       const float* gain = nullptr, const float* alpha = nullptr, const uint8_t* head_enable = nullptr);
 
-// One expert: the edited keys of the tiles that hold a highlighted token into the side buffer X [T, Hkv, 2 d] of the
-// fused forward (high | low parts), by the pipelined tile kernel of the stand-alone edit (two launches with its
-// preparation).  K16 is the bf16 key tensor; workspace regions as in workspace_layout.
+// Eq. 6 for every (sequence, KV head): the launch behind adaseka_route
+seka_status launch_route(const seka_shape* s, const void* Q, const float* U, const float* sigma, int k_route,
+                         float* alpha_out, cudaStream_t st);
+
+// The edited keys of the tiles that hold a highlighted token into the side buffer X [T, Hkv, 2 d] of the fused forward
+// (high | low parts), by the tile kernels of the stand-alone edit in their side mode (two launches with the
+// preparation): the pipelined kernel for one expert, the bank kernel for several (n_experts * d <= 512).
+// K16 is the bf16 key tensor; workspace regions as in workspace_layout.
 seka_status launch_stage_keys_pipe(const seka_shape* s, const WorkspaceLayout& w, const void* K16, void* X,
                                    const uint8_t* mask, const float* U, const float* alpha, const float* gain,
                                    const uint8_t* head_enable, char* ws, cudaStream_t st);
