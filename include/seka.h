@@ -120,12 +120,11 @@ seka_status seka_attention_fwd(const seka_shape* shape, const void* Q, const voi
                                void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
- * AdaSEKA in one call (Algorithm 2): the routing coefficients of Eq. 6, then seka_attention_fwd with them, queued on
- * the stream by one call.  Banks that fit tensor memory (n_experts * head_dim <= 512) run the launch of adaseka_route
- * ahead of the preparation of the forward; wider banks evaluate Eq. 6 inside a one-launch preparation kernel.
- * sigma and k_route are those of adaseka_route; either way the result equals adaseka_route followed by
- * seka_attention_fwd bit for bit.  alpha_out, if not NULL, receives the coefficients (fp32 [B, Hkv, M]); without it
- * they live in the workspace.  mask, U and sigma are required.
+ * AdaSEKA in one call (Algorithm 2): seka_attention_fwd with the routing coefficients of Eq. 6 computed by further
+ * blocks of the library's operand-preparation launch instead of by a separate adaseka_route call (one launch fewer).
+ * sigma and k_route are those of adaseka_route; the result equals adaseka_route followed by seka_attention_fwd bit
+ * for bit.  alpha_out, if not NULL, receives the coefficients (fp32 [B, Hkv, M]); without it they live in the
+ * workspace.  mask, U and sigma are required.
  */
 seka_status seka_attention_fwd_routed(const seka_shape* shape, const void* Q, const void* K,
                                       const void* V, void* O, float* lse,

@@ -830,18 +830,14 @@ static seka_status attention_fwd_impl(const seka_shape* shape, const void* Q, co
     int* first_hot = reinterpret_cast<int*>(ws + w.first_off);
     uint8_t* bh_info = reinterpret_cast<uint8_t*>(ws + w.info_off);
     if (steer) {
-        // The tile kernels of the stand-alone edit write the side buffer (two small launches; a routed call first runs the
-        // launch of adaseka_route, so that it computes exactly what route-then-forward computes).  Banks too wide for
-        // tensor memory (n_experts * head_dim > 512) take the one-launch preparation kernel.
+        // The tile kernels of the stand-alone edit write the side buffer (two small launches; in a routed call further
+        // blocks of the first one evaluate Eq. 6 with the routine of adaseka_route, so the coefficients, and with them
+        // everything after, are those of route-then-forward bit for bit).  Banks too wide for tensor memory
+        // (n_experts * head_dim > 512) take the one-launch preparation kernel.
         if ((long long)shape->n_experts * D <= 512) {
             const float* a = alpha;
-            if (sigma != nullptr) {
-                float* ar = alpha_out != nullptr ? alpha_out : reinterpret_cast<float*>(ws + w.alpha_off);
-                stc = launch_route(shape, Q, U, sigma, k_route, ar, st);
-                if (stc != SEKA_OK) return stc;
-                a = ar;
-            }
-            stc = launch_stage_keys_pipe(shape, w, k16, X, mask, U, a, gain, head_enable, ws, st);
+            if (sigma != nullptr) a = alpha_out != nullptr ? alpha_out : reinterpret_cast<float*>(ws + w.alpha_off);
+            stc = launch_stage_keys_pipe(shape, w, k16, X, mask, U, a, gain, head_enable, ws, st, Q, sigma, k_route);
         } else {
             stc = launch_prep_steering(shape, p.plan, k16, U, alpha, gain, head_enable, mask, X, tile_hot, first_hot, bh_info,
                                        reinterpret_cast<int*>(ws), w.n_tiles, st, Q, sigma, k_route, alpha_out);

@@ -634,7 +634,7 @@ static seka_status launch_edit_tiles(const seka_shape* s, const WorkspaceLayout&
     void* P = ws + w.w_off;
     uint8_t* tile_hot = reinterpret_cast<uint8_t*>(ws + w.hot_off);
     int* hot_list = reinterpret_cast<int*>(ws + w.list_off);
-    launch_prep_edit(s, U, mask, P, tile_hot, w.n_tiles, hot_list, status + 2, st);
+    if (launch_prep_edit(s, U, mask, P, tile_hot, w.n_tiles, hot_list, status + 2, st) != SEKA_OK) return SEKA_ERR_CUDA;
     const int T = shape_total_tokens(s), Hkv = s->n_kv_heads, M = s->n_experts;
     CUtensorMap tk, tp;
     if (!make_tile_map(&tk, K_in, D, Hkv, T) || !make_tile_map(&tp, P, D, 1, (long long)2 * M * Hkv * D, D)) return SEKA_ERR_CUDA;
@@ -666,7 +666,8 @@ static seka_status launch_edit_tiles(const seka_shape* s, const WorkspaceLayout&
 template <int D>
 static seka_status stage_keys_pipe_t(const seka_shape* s, const WorkspaceLayout& w, const void* K16, void* X,
                                      const uint8_t* mask, const float* U, const float* alpha, const float* gain,
-                                     const uint8_t* he, char* ws, cudaStream_t st) {
+                                     const uint8_t* he, char* ws, cudaStream_t st, const void* Q_route, const float* sigma,
+                                     int k_route) {
     using PL = EpSmem<D>;
     int n_sm = 0;
     if (!device_info(&n_sm)) return SEKA_ERR_CUDA;
@@ -674,8 +675,11 @@ static seka_status stage_keys_pipe_t(const seka_shape* s, const WorkspaceLayout&
     void* P = ws + w.w_off;
     uint8_t* tile_hot = reinterpret_cast<uint8_t*>(ws + w.hot_off);
     int* hot_list = reinterpret_cast<int*>(ws + w.list_off);
-    launch_prep_edit(s, U, mask, P, tile_hot, w.n_tiles, hot_list, status + 2, st, reinterpret_cast<int*>(ws + w.first_off),
-                     reinterpret_cast<uint8_t*>(ws + w.info_off), gain, alpha, he);
+    // routed call: `alpha` is where the preparation launch writes the coefficients (read by the tile kernel after it)
+    if (launch_prep_edit(s, U, mask, P, tile_hot, w.n_tiles, hot_list, status + 2, st, reinterpret_cast<int*>(ws + w.first_off),
+                         reinterpret_cast<uint8_t*>(ws + w.info_off), gain, alpha, he, Q_route, sigma, k_route,
+                         const_cast<float*>(alpha)) != SEKA_OK)
+        return SEKA_ERR_CUDA;
     const int T = shape_total_tokens(s), Hkv = s->n_kv_heads, M = s->n_experts;
     CUtensorMap tk, tp;
     if (!make_tile_map(&tk, K16, D, Hkv, T) || !make_tile_map(&tp, P, D, 1, (long long)2 * M * Hkv * D, D)) return SEKA_ERR_CUDA;
@@ -708,9 +712,10 @@ static seka_status stage_keys_pipe_t(const seka_shape* s, const WorkspaceLayout&
 
 seka_status launch_stage_keys_pipe(const seka_shape* s, const WorkspaceLayout& w, const void* K16, void* X,
                                    const uint8_t* mask, const float* U, const float* alpha, const float* gain,
-                                   const uint8_t* head_enable, char* ws, cudaStream_t st) {
-    return s->head_dim == 128 ? stage_keys_pipe_t<128>(s, w, K16, X, mask, U, alpha, gain, head_enable, ws, st)
-                              : stage_keys_pipe_t<64>(s, w, K16, X, mask, U, alpha, gain, head_enable, ws, st);
+                                   const uint8_t* head_enable, char* ws, cudaStream_t st, const void* Q_route,
+                                   const float* sigma, int k_route) {
+    return s->head_dim == 128 ? stage_keys_pipe_t<128>(s, w, K16, X, mask, U, alpha, gain, head_enable, ws, st, Q_route, sigma, k_route)
+                              : stage_keys_pipe_t<64>(s, w, K16, X, mask, U, alpha, gain, head_enable, ws, st, Q_route, sigma, k_route);
 }
 
 }  // namespace seka

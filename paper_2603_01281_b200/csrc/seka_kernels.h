@@ -23,10 +23,13 @@ void launch_compact_mask(const uint8_t* mask, int T, int* list, int* count, cuda
 void launch_convert_bf16(const float* in, void* out, size_t n, cudaStream_t st);
 
 // Preparation of the tile-wise edit: P[m][h] = U_m U_m^T (two bf16 parts), tile flags, list of the tiles that hold a
-// highlighted token; with `first_hot` / `bh_info` set also what the fused forward needs (see prep_edit_kernel).
-void launch_prep_edit(const seka_shape* s, const float* U, const uint8_t* mask, void* P, uint8_t* tile_hot, int n_tiles,
-                      int* hot_list, int* hot_count, cudaStream_t st, int* first_hot = nullptr, uint8_t* bh_info = nullptr,
-                      const float* gain = nullptr, const float* alpha = nullptr, const uint8_t* head_enable = nullptr);
+// highlighted token; with `first_hot` / `bh_info` set also what the fused forward needs (see prep_edit_kernel); with
+// `sigma` set also the routing coefficients of Eq. 6 into `alpha_out` (further blocks of the same launch).
+seka_status launch_prep_edit(const seka_shape* s, const float* U, const uint8_t* mask, void* P, uint8_t* tile_hot, int n_tiles,
+                             int* hot_list, int* hot_count, cudaStream_t st, int* first_hot = nullptr, uint8_t* bh_info = nullptr,
+                             const float* gain = nullptr, const float* alpha = nullptr, const uint8_t* head_enable = nullptr,
+                             const void* Q_route = nullptr, const float* sigma = nullptr, int k_route = 0,
+                             float* alpha_out = nullptr);
 
 // Eq. 6 for every (sequence, KV head): the launch behind adaseka_route
 seka_status launch_route(const seka_shape* s, const void* Q, const float* U, const float* sigma, int k_route,
@@ -38,7 +41,8 @@ seka_status launch_route(const seka_shape* s, const void* Q, const float* U, con
 // K16 is the bf16 key tensor; workspace regions as in workspace_layout.
 seka_status launch_stage_keys_pipe(const seka_shape* s, const WorkspaceLayout& w, const void* K16, void* X,
                                    const uint8_t* mask, const float* U, const float* alpha, const float* gain,
-                                   const uint8_t* head_enable, char* ws, cudaStream_t st);
+                                   const uint8_t* head_enable, char* ws, cudaStream_t st, const void* Q_route = nullptr,
+                                   const float* sigma = nullptr, int k_route = 0);
 
 // bf16 tensor [T, H, d] viewed as (d, H, T) for TMA: tiles of 64 x 1 x box_rows with the 128-byte swizzle.
 bool make_tile_map(CUtensorMap* m, const void* base, int d, int H, long long T, int box_rows = 128);

@@ -489,8 +489,26 @@ struct SteerInfoArgs {
 __global__ void prep_edit_kernel(const float* __restrict__ U, const uint8_t* __restrict__ mask,
                                  const int* __restrict__ cu_seqlens, __nv_bfloat16* __restrict__ P,
                                  uint8_t* __restrict__ tile_hot, int* __restrict__ hot_list, int* __restrict__ hot_count,
-                                 int B, int L, int Hkv, int D, int r, int M, int n_tiles, int n_p, const SteerInfoArgs info) {
+                                 int B, int L, int Hkv, int D, int r, int M, int n_tiles, int n_p, int n_flag,
+                                 const SteerInfoArgs info, const RouteArgs route) {
     const int tid = threadIdx.x;
+    if ((int)blockIdx.x >= n_p + n_flag) {
+        // ------------------------------------------------------------ (routed call) Eq. 6 for one (sequence, KV head), with the
+        // routine adaseka_route uses; the block also writes the steering byte of its pair, which needs the coefficients
+        extern __shared__ double route_sm[];
+        const int bh = (int)blockIdx.x - n_p - n_flag, b = bh / Hkv, h = bh % Hkv;
+        const double* a = route_group(route.Q, route.q_is_f32, U, route.sigma, cu_seqlens, L, route.Hq, Hkv, D, r, M,
+                                      route.k_route, b, h, route_sm);
+        for (int m = tid; m < M; m += blockDim.x) route.alpha_out[(size_t)bh * M + m] = (float)a[m];
+        if (tid == 0 && info.bh_info != nullptr) {
+            const float g = info.gain[b];
+            const bool on = g != 0.f && (info.head_enable == nullptr || info.head_enable[h] != 0);
+            float amax = 0.f;
+            for (int m = 0; m < M; ++m) amax = fmaxf(amax, fabsf((float)a[m]));
+            info.bh_info[bh] = (on ? 1 : 0) | ((on && lo_needed(g, amax)) ? 2 : 0);
+        }
+        return;
+    }
     if ((int)blockIdx.x < n_p) {
         const int tiles = D / 32;
         const int mh = blockIdx.x / (tiles * tiles), t = blockIdx.x % (tiles * tiles);
@@ -540,7 +558,7 @@ __global__ void prep_edit_kernel(const float* __restrict__ U, const uint8_t* __r
             if (any) hot_list[atomicAdd(hot_count, 1)] = item;
             if (any && info.first_hot != nullptr) atomicMin(info.first_hot + b, t);
         }
-        if (info.bh_info != nullptr && t == 0) {
+        if (info.bh_info != nullptr && t == 0 && route.sigma == nullptr) {
             const float g = info.gain[b];
             for (int h = lane; h < Hkv; h += 32) {
                 const bool on = g != 0.f && (info.head_enable == nullptr || info.head_enable[h] != 0);
@@ -658,19 +676,27 @@ seka_status launch_prep_steering(const seka_shape* sh, const SteerPlan& plan, co
     return cudaGetLastError() == cudaSuccess ? SEKA_OK : SEKA_ERR_CUDA;
 }
 
-void launch_prep_edit(const seka_shape* sh, const float* U, const uint8_t* mask, void* P, uint8_t* tile_hot, int n_tiles,
-                      int* hot_list, int* hot_count, cudaStream_t st, int* first_hot, uint8_t* bh_info, const float* gain,
-                      const float* alpha, const uint8_t* head_enable) {
+seka_status launch_prep_edit(const seka_shape* sh, const float* U, const uint8_t* mask, void* P, uint8_t* tile_hot, int n_tiles,
+                             int* hot_list, int* hot_count, cudaStream_t st, int* first_hot, uint8_t* bh_info, const float* gain,
+                             const float* alpha, const uint8_t* head_enable, const void* Q_route, const float* sigma,
+                             int k_route, float* alpha_out) {
     const int D = sh->head_dim, tiles = D / 32;
     const int n_p = sh->n_experts * sh->n_kv_heads * tiles * tiles;
     const int n_flag = (sh->batch * n_tiles + 7) / 8;
+    const int n_r = sigma != nullptr ? sh->batch * sh->n_kv_heads : 0;
+    const size_t smem = sigma != nullptr ? route_smem_bytes(D, sh->n_experts, k_route) : 0;
+    if (smem > 40 * 1024 &&      // beside 8 KB of static shared memory; very wide banks of rank-1 experts: up to 66 KB
+        cudaFuncSetAttribute(prep_edit_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return SEKA_ERR_CUDA;
     cudaMemsetAsync(hot_count, 0, sizeof(int), st);
     if (first_hot != nullptr) cudaMemsetAsync(first_hot, 0x7f, sizeof(int) * sh->batch, st);      // a large value per sequence
     SteerInfoArgs info{first_hot, bh_info, gain, alpha, head_enable};
-    prep_edit_kernel<<<n_p + n_flag, 256, 0, st>>>(U, mask, sh->cu_seqlens, static_cast<__nv_bfloat16*>(P), tile_hot, hot_list,
-                                                  hot_count, sh->batch, sh->max_seqlen, sh->n_kv_heads, D, sh->rank,
-                                                  sh->n_experts, n_tiles, n_p, info);
+    RouteArgs route{Q_route, sh->dtype == SEKA_F32 ? 1 : 0, sigma, k_route, sh->n_q_heads, alpha_out};
+    prep_edit_kernel<<<n_p + n_flag + n_r, 256, smem, st>>>(U, mask, sh->cu_seqlens, static_cast<__nv_bfloat16*>(P), tile_hot, hot_list,
+                                                            hot_count, sh->batch, sh->max_seqlen, sh->n_kv_heads, D, sh->rank,
+                                                            sh->n_experts, n_tiles, n_p, n_flag, info, route);
     ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? SEKA_OK : SEKA_ERR_CUDA;
 }
 
 void launch_build_items(const Sched& sc, const int* cu, const uint8_t* bh_info, ItemRecord* items, int* count,

@@ -346,7 +346,7 @@ def test_fused_output_is_repeatable(name):
     assert binding.seka_poll_status(ws) == binding.SEKA_OK
 
 
-# ----------------------------------------------------------------- AdaSEKA in one call (routing ahead of the preparation, same stream)
+# ----------------------------------------------------------------- AdaSEKA in one call (routing inside the preparation launch)
 
 @pytest.mark.parametrize("case", ["C3", "small_f32", "small_varlen", "wide_bank"])
 def test_routed_forward_equals_route_then_forward(case):
@@ -380,7 +380,7 @@ def test_routed_forward_equals_route_then_forward(case):
                                       k_route, alpha1, dev["gain"], hed, ws1)
     launches_one = binding.seka_launch_count() - launches0 - launches_two
     assert binding.seka_poll_status(ws1) == binding.SEKA_OK
-    assert launches_one <= launches_two          # the one call runs the same launches (banks too wide for tensor memory: one fewer)
+    assert launches_one == launches_two - 1      # Eq. 6 runs in blocks of the preparation launch
     assert torch.equal(alpha1, alpha)
     assert torch.equal(O1.view(torch.int16 if O1.dtype == torch.bfloat16 else torch.int32),
                        O2.view(torch.int16 if O2.dtype == torch.bfloat16 else torch.int32))
