@@ -148,7 +148,9 @@ seka_status seka_attention_fwd_routed(const seka_shape* shape, const void* Q, co
  * it).  What they do wait for is the previous host-buffer call's kernels on this device,
  * which may still be reading a staging buffer; the library keeps eight events per device
  * for that.  `staging` belongs to the call until `cuda_stream` has passed it; two calls
- * that overlap in time need a staging buffer and a workspace each.  U, alpha, gain,
+ * that overlap in time need a staging buffer and a workspace each.  Because its copies
+ * run on streams of its own that do not start from `cuda_stream`, this entry point must
+ * not be called while `cuda_stream` is being captured into a graph.  U, alpha, gain,
  * head_enable stay device pointers (they are per-model or per-prompt constants).
  */
 size_t seka_host_staging_bytes(const seka_shape* shape);
