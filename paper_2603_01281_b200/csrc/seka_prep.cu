@@ -569,40 +569,79 @@ __global__ void prep_edit_kernel(const float* __restrict__ U, const uint8_t* __r
     }
 }
 
-// Item table of the fused kernel for packed variable-length batches: items (see decode_item) whose tiles lie beyond
-// their sequence are dropped, order kept (one CTA scans).
-__global__ void build_items_varlen_kernel(const Sched sc, const int* __restrict__ cu, const uint8_t* __restrict__ bh_info,
-                                          ItemRecord* __restrict__ items, int* __restrict__ count) {
+// Item table of the fused kernel for packed variable-length batches: the items of decode_item whose tiles lie beyond
+// their sequence are dropped, order kept.  One block per row slot (block 0: the last, heaviest row); where a block's
+// items start follows from the sequence lengths alone, so the blocks do not talk to each other: a sequence of n_t row
+// tiles has R = n_t (tiles A and B are two heads) or ceil(n_t / 2) (two row tiles) row slots, row slot `row` keeps the
+// sequences with R > row, and the rows before it in the table hold hs * sum_b max(0, R_b - row - 1) items.
+__global__ void __launch_bounds__(1024)
+build_items_varlen_kernel(const Sched sc, const int* __restrict__ cu, const uint8_t* __restrict__ bh_info,
+                          ItemRecord* __restrict__ items, int* __restrict__ count) {
+    __shared__ long long red_s[32];
+    __shared__ int pre_s[1024];
     __shared__ int warp_tot[32];
-    __shared__ int base_s;
+    __shared__ long long base_s;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nw = blockDim.x >> 5;
-    if (tid == 0) base_s = 0;
+    const int row = sc.rs - 1 - (int)blockIdx.x;
+    auto rows_of = [&](int b) -> int {
+        const int n_t = (cu[b + 1] - cu[b] + 127) / 128;
+        return sc.pair_heads ? n_t : (n_t + 1) / 2;
+    };
+    // items of the rows above this one (they come first), and, in block 0, of all rows
+    long long before = 0, all = 0;
+    for (int b = tid; b < sc.B; b += blockDim.x) {
+        const int R = rows_of(b);
+        before += R > row + 1 ? R - row - 1 : 0;
+        all += R;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        before += __shfl_xor_sync(0xffffffffu, before, o);
+        all += __shfl_xor_sync(0xffffffffu, all, o);
+    }
+    if (lane == 0) red_s[wid] = before;
     __syncthreads();
-    const long long n = sc.n_items_max;
-    for (long long start = 0; start < n; start += blockDim.x) {
-        const long long idx = start + tid;
-        ItemRecord r;
-        bool keep = false;
-        if (idx < n) {
-            keep = decode_item(sc, idx, cu, r);
-            const int b = r.bh & 0xffff, hkv = r.bh >> 16;
-            r.steer = bh_info != nullptr ? (int)bh_info[b * sc.Hkv + hkv] : 0;
+    if (tid == 0) {
+        long long t = 0;
+        for (int q = 0; q < nw; ++q) t += red_s[q];
+        base_s = t * sc.hs;
+    }
+    __syncthreads();
+    if (blockIdx.x == 0) {
+        if (lane == 0) red_s[wid] = all;
+        __syncthreads();
+        if (tid == 0) {
+            long long t = 0;
+            for (int q = 0; q < nw; ++q) t += red_s[q];
+            *count = (int)(t * sc.hs);
         }
+    }
+    // this row: the sequences that reach it, 1024 at a time, keep their order
+    for (int b0 = 0; b0 < sc.B; b0 += blockDim.x) {
+        const int b = b0 + tid;
+        const bool keep = b < sc.B && rows_of(b) > row;
         const unsigned bal = __ballot_sync(0xffffffffu, keep);
         if (lane == 0) warp_tot[wid] = __popc(bal);
         __syncthreads();
-        int off = base_s;
-        for (int q = 0; q < wid; ++q) off += warp_tot[q];
-        if (keep) items[off + __popc(bal & ((1u << lane) - 1))] = r;
+        int off = 0, tot = 0;
+        for (int q = 0; q < nw; ++q) { if (q < wid) off += warp_tot[q]; tot += warp_tot[q]; }
+        pre_s[tid] = keep ? off + __popc(bal & ((1u << lane) - 1)) : -1;
+        const long long base = base_s;
         __syncthreads();
-        if (tid == 0) {
-            int tot = 0;
-            for (int q = 0; q < nw; ++q) tot += warp_tot[q];
-            base_s += tot;
+        const int n_b = sc.B - b0 < (int)blockDim.x ? sc.B - b0 : (int)blockDim.x;
+        for (int c = tid; c < n_b * sc.hs; c += blockDim.x) {
+            const int bi = c / sc.hs, slot = c - bi * sc.hs;
+            const int pos = pre_s[bi];
+            if (pos < 0) continue;
+            ItemRecord r;
+            decode_item(sc, (long long)blockIdx.x * sc.per + (long long)(b0 + bi) * sc.hs + slot, cu, r);
+            r.steer = bh_info != nullptr ? (int)bh_info[(r.bh & 0xffff) * sc.Hkv + (r.bh >> 16)] : 0;
+            items[base + (long long)pos * sc.hs + slot] = r;
         }
         __syncthreads();
+        if (tid == 0) base_s = base + (long long)tot * sc.hs;
+        __syncthreads();
     }
-    if (tid == 0) *count = base_s;
 }
 
 // Appends the indices of highlighted tokens to `list` (order within a warp preserved).
@@ -701,7 +740,8 @@ seka_status launch_prep_edit(const seka_shape* sh, const float* U, const uint8_t
 
 void launch_build_items(const Sched& sc, const int* cu, const uint8_t* bh_info, ItemRecord* items, int* count,
                         cudaStream_t st) {
-    build_items_varlen_kernel<<<1, 1024, 0, st>>>(sc, cu, bh_info, items, count);
+    if (sc.rs <= 0) return;
+    build_items_varlen_kernel<<<(unsigned)sc.rs, 1024, 0, st>>>(sc, cu, bh_info, items, count);
     ++g_launches;
 }
 
