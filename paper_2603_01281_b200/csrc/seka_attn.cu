@@ -817,9 +817,7 @@ static seka_status attention_fwd_impl(const seka_shape* shape, const void* Q, co
         char* cq = ws + w.cvt_off;
         char* ck = cq + align_up(nq * 2, 256);
         char* cv = ck + align_up(nk * 2, 256);
-        launch_convert_bf16(static_cast<const float*>(Q), cq, nq, st);
-        launch_convert_bf16(static_cast<const float*>(K), ck, nk, st);
-        launch_convert_bf16(static_cast<const float*>(V), cv, nk, st);
+        launch_convert_bf16(static_cast<const float*>(Q), cq, nq, static_cast<const float*>(K), ck, static_cast<const float*>(V), cv, nk, st);
         q16 = cq; k16 = ck; v16 = cv;
     }
     AttnParams p;

@@ -20,7 +20,8 @@ seka_status launch_prep_steering(const seka_shape* s, const SteerPlan& plan, con
 void launch_build_items(const Sched& sc, const int* cu, const uint8_t* bh_info, ItemRecord* items, int* count,
                         cudaStream_t st);
 void launch_compact_mask(const uint8_t* mask, int T, int* list, int* count, cudaStream_t st);
-void launch_convert_bf16(const float* in, void* out, size_t n, cudaStream_t st);
+void launch_convert_bf16(const float* Q, void* q16, size_t nq, const float* K, void* k16, const float* V, void* v16, size_t nk,
+                         cudaStream_t st);
 
 // Preparation of the tile-wise edit: P[m][h] = U_m U_m^T (two bf16 parts), tile flags, list of the tiles that hold a
 // highlighted token; with `first_hot` / `bh_info` set also what the fused forward needs (see prep_edit_kernel); with

@@ -658,11 +658,19 @@ __global__ void compact_mask_kernel(const uint8_t* __restrict__ mask, int T, int
     if (hl) list[base + __popc(b & ((1u << lane) - 1))] = t;
 }
 
-__global__ void convert_f32_bf16_kernel(const float4* __restrict__ in, uint2* __restrict__ out, size_t n4) {
-    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= n4) return;
-    const float4 v = in[i];
-    out[i] = make_uint2(pack_bf16(v.x, v.y), pack_bf16(v.z, v.w));
+// fp32 -> bf16 copies of Q, K and V in one launch (groups of four values; the three tensors one after another)
+struct ConvertArgs { const float4* in[3]; uint2* out[3]; size_t n4[3]; };
+__global__ void convert_f32_bf16_kernel(const ConvertArgs a) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+#pragma unroll
+    for (int t = 0; t < 3; ++t) {
+        if (i < a.n4[t]) {
+            const float4 v = a.in[t][i];
+            a.out[t][i] = make_uint2(pack_bf16(v.x, v.y), pack_bf16(v.z, v.w));
+            return;
+        }
+        i -= a.n4[t];
+    }
 }
 
 static size_t route_bytes_aligned(int D, int M, int k_route) { return align_up(route_smem_bytes(D, M, k_route), 16); }
@@ -752,11 +760,15 @@ void launch_compact_mask(const uint8_t* mask, int T, int* list, int* count, cuda
     ++g_launches;
 }
 
-void launch_convert_bf16(const float* in, void* out, size_t n, cudaStream_t st) {
-    const size_t n4 = n / 4;   // head_dim is a multiple of 4, so n is too
+void launch_convert_bf16(const float* Q, void* q16, size_t nq, const float* K, void* k16, const float* V, void* v16, size_t nk,
+                         cudaStream_t st) {
+    ConvertArgs a;      // head_dim is a multiple of 4, so the element counts are too
+    a.in[0] = reinterpret_cast<const float4*>(Q); a.out[0] = reinterpret_cast<uint2*>(q16); a.n4[0] = nq / 4;
+    a.in[1] = reinterpret_cast<const float4*>(K); a.out[1] = reinterpret_cast<uint2*>(k16); a.n4[1] = nk / 4;
+    a.in[2] = reinterpret_cast<const float4*>(V); a.out[2] = reinterpret_cast<uint2*>(v16); a.n4[2] = nk / 4;
+    const size_t n4 = a.n4[0] + a.n4[1] + a.n4[2];
     if (n4 == 0) return;
-    convert_f32_bf16_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(
-        reinterpret_cast<const float4*>(in), reinterpret_cast<uint2*>(out), n4);
+    convert_f32_bf16_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(a);
     ++g_launches;
 }
 
