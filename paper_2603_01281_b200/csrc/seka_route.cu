@@ -19,7 +19,7 @@ seka_status launch_route(const seka_shape* shape, const void* Q, const float* U,
     if (smem > 48 * 1024 &&      // very wide banks of rank-1 experts: up to 66 KB
         cudaFuncSetAttribute(route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return SEKA_ERR_CUDA;
-    route_kernel<<<shape->batch * shape->n_kv_heads, 256, smem, stream>>>(
+    route_kernel<<<shape->batch * shape->n_kv_heads, 1024, smem, stream>>>(
         Q, shape->dtype == SEKA_F32 ? 1 : 0, U, sigma, shape->cu_seqlens, shape->max_seqlen, shape->n_q_heads,
         shape->n_kv_heads, shape->head_dim, shape->rank, shape->n_experts, k_route, alpha_out);
     ++g_launches;
